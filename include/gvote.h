@@ -1,0 +1,189 @@
+/*
+ * gvote.h — C ABI of the GVote per-request KV-cache compression pass for NVIDIA B200 (sm_100a).
+ *
+ * The pass is Algorithm 1 of "Adaptive KV-Cache Compression without Manually Setting Budget"
+ * (GVote), run once per layer at the end of prefill, per request and per KV head
+ * (Section 3.2): fit a diagonal Gaussian to the hidden states (Step 2), draw S synthetic
+ * hidden states (Step 3), project them through W_q and rotate them with the RoPE cos/sin
+ * averaged over n_f future positions (Step 3), score them against all cached keys, let each
+ * synthetic query pick its keys (top-k with k = |C0|, where C0 is the top-p set of the
+ * current query, Step 1), OR the picks into one keep-mask per KV head (Step 4) and prune K
+ * and V to that set (Algorithm 1, line 11).
+ *
+ * Conventions, valid for every entry point unless it says otherwise
+ *  - Every pointer named below is a DEVICE pointer unless its comment says "host".
+ *  - The caller owns every buffer.  The library allocates nothing, frees nothing and keeps
+ *    no pointer after a call returns (gvote_compress_host is the one exception, see there).
+ *  - Work is enqueued on the given CUDA stream (passed as void* = cudaStream_t); calls return
+ *    without synchronising.
+ *  - Return value: GVOTE_OK (0) or a negative GVOTE_ERR_* code.  On an error detected on the
+ *    host nothing has been enqueued.  A bounded device-side wait that ran out is reported
+ *    through the status word at the start of the workspace: read it with gvote_poll_status.
+ *  - Pointers must be 16-byte aligned; d_h must be a multiple of 8, d_k a multiple of 8.
+ *  - A ragged batch packs its requests along the token axis; cu_seqlens [batch+1] int32
+ *    (device) holds the prefix sums of the request lengths N_r (request r owns tokens
+ *    cu_seqlens[r] .. cu_seqlens[r+1]-1).  `total_tokens` = cu_seqlens[batch] and `max_N` =
+ *    the longest request are passed from the host so that no call has to read the device.
+ *  - bf16 tensors: W_q [n_q_heads*d_k, d_h], one row per output feature (the paper's W_q
+ *    stored transposed, as linear layers keep it), row stride wq_ld elements;
+ *    K and V [n_kv_heads, total_tokens, d_k] with element strides (head_stride, tok_stride),
+ *    inner dimension contiguous; keys are stored as the model stores them (already rotated).
+ *  - Positions: request r's keys sit at positions 0..N_r-1, its current query at N_r-1 and the
+ *    n_f future positions are N_r .. N_r+n_f-1.
+ *  - Keep-mask: uint32 words, bit (n mod 32) of word (n div 32) is key n of the request; each
+ *    request's bit row starts on a word boundary at word gvote_mask_word_offset(cu_seqlens[r], r)
+ *    of its head's row; a head's row has gvote_mask_row_words(total_tokens, batch) words;
+ *    padding bits are zero.
+ */
+#ifndef GVOTE_H_
+#define GVOTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define GVOTE_API __attribute__((visibility("default")))
+#else
+#define GVOTE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  GVOTE_OK = 0,
+  GVOTE_ERR_INVALID_ARG = -1,
+  GVOTE_ERR_UNALIGNED = -2,
+  GVOTE_ERR_WORKSPACE_TOO_SMALL = -3,
+  GVOTE_ERR_UNSUPPORTED_SHAPE = -4,
+  GVOTE_ERR_CUDA = -5,
+  GVOTE_ERR_TIMEOUT = -6
+};
+
+enum { GVOTE_SEL_TOPK_C0 = 0, GVOTE_SEL_TOPP = 1 };
+enum { GVOTE_DTYPE_F32 = 0, GVOTE_DTYPE_BF16 = 1 };
+
+/* Hyper-parameters and model shape (Algorithm 1, "Require" line, plus what it uses implicitly). */
+typedef struct {
+  int32_t d_h;          /* hidden size */
+  int32_t n_q_heads;    /* query heads */
+  int32_t n_kv_heads;   /* KV heads; n_q_heads must be a multiple */
+  int32_t d_k;          /* head dimension */
+  double  rope_theta;   /* RoPE base; rotate-half pairing (j, j+d_k/2), w_j = theta^(-2j/d_k) */
+  int32_t S;            /* synthetic queries per request (Section 3.5: S >= 8 advised) */
+  float   p_nuc;        /* nucleus mass threshold in (0,1] (Section 3.5: 0.95 advised) */
+  int32_t n_f;          /* future positions whose cos/sin are averaged (Step 3) */
+  int32_t n_s;          /* leading sink tokens the fit ignores (Step 2) */
+  int32_t sel_mode;     /* GVOTE_SEL_TOPK_C0: Algorithm 1 line 9.  GVOTE_SEL_TOPP: the top-p rule
+                           of Section 3.1 applied to every synthetic query instead. */
+  int32_t include_c0;   /* non-zero: the current query's set C0 joins the union (line 10 unions
+                           the synthetic sets only; default 0) */
+  uint64_t seed;        /* Philox key */
+  uint32_t layer_id;    /* Philox counter word: gives every layer its own stream */
+  int32_t h_dtype;      /* GVOTE_DTYPE_F32 or GVOTE_DTYPE_BF16: element type of h and h_last */
+} gvote_params;
+
+/* Words per head in the keep-mask, and the word where request r's bits start. */
+static inline int64_t gvote_mask_row_words(int64_t total_tokens, int32_t batch) {
+  return (total_tokens >> 5) + batch;
+}
+static inline int64_t gvote_mask_word_offset(int64_t cu_seqlens_r, int32_t r) {
+  return (cu_seqlens_r >> 5) + r;
+}
+
+/* Bytes of scratch every entry point below accepts as `ws` for a batch of this size.  The
+ * first 256 bytes hold the status word; a workspace must be zero-filled once after
+ * allocation (the library keeps it consistent afterwards).  Returns 0 on invalid params. */
+GVOTE_API size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
+
+/* Step 2 / Algorithm 1 line 4.  mu[r][c], var[r][c] = mean and unbiased variance over rows
+ * cu_seqlens[r]+n_s .. cu_seqlens[r+1]-1 of h [total_tokens, d_h] (row stride h_row_stride
+ * elements).  Every request needs N_r - n_s >= 2 (the result is NaN otherwise; the host cannot
+ * check device-resident lengths, it checks max_N only).  mu, var: [batch, d_h] float. */
+GVOTE_API int32_t gvote_fit(const gvote_params* p, const void* h, int64_t h_row_stride,
+                  const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                  float* mu, float* var, void* ws, size_t ws_bytes, void* stream);
+
+/* Step 3 / Algorithm 1 line 5.  H_tilde[r][s][c] = mu[r][c] + sqrt(var[r][c]) * z, z a standard
+ * normal drawn by Box-Muller from Philox4x32-10 with key = (seed low, seed high) and counter
+ * = (c div 4, s, layer_id, r); word pairs (0,1) and (2,3) of a block give channels 4b..4b+3;
+ * u = ((x >> 9) + 0.5) * 2^-23.  H_tilde: [batch, S, d_h] float.  raw_u32_or_null, when given,
+ * receives the Philox words [batch, S, d_h] (bit-exact by definition). */
+GVOTE_API int32_t gvote_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch,
+                     float* H_tilde, uint32_t* raw_u32_or_null, void* stream);
+
+/* Algorithm 1 lines 1 (Q0), 6 and 7.  X = [h_last[r]; H_tilde[r]] is rounded to bf16, multiplied
+ * by W_q (fp32 accumulation), b_q added when given ([n_q_heads*d_k] float), then rotated: row 0
+ * exactly at position N_r-1, rows 1..S with the mean cos/sin of positions N_r..N_r+n_f-1.
+ * Q: [batch, n_q_heads, S+1, d_k] bf16.  h_last: [batch, d_h] of p->h_dtype. */
+GVOTE_API int32_t gvote_project(const gvote_params* p, const float* H_tilde, const void* h_last,
+                      const void* W_q, int64_t wq_ld, const float* b_q_or_null,
+                      const int32_t* cu_seqlens, int32_t batch,
+                      void* Q, void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 lines 1-3 and 8-10, given the rotated queries.  Per query head g: logits of its
+ * S+1 rows against the N_r keys of KV head g div G, scaled by 1/sqrt(d_k); row 0 -> softmax ->
+ * top-p -> b_step[r][g] = |C0|; rows 1..S -> top-k(b_step) on logits (or top-p on their softmax
+ * in GVOTE_SEL_TOPP); mask[h] = OR over the rows of the head's group; budget[r][h] = popcount.
+ * Ties at a selection boundary go to the lower key index.  mask: [n_kv_heads, row_words] is
+ * overwritten.  dbg_probs_or_null: [sum_r n_q_heads*(S+1)*N_r] float, request-major, receives the
+ * softmax rows (small cases only). */
+GVOTE_API int32_t gvote_vote(const gvote_params* p, const void* Q,
+                   const void* K, int64_t k_tok_stride, int64_t k_head_stride,
+                   const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                   uint32_t* mask, int32_t* budget, int32_t* b_step,
+                   float* dbg_probs_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/* gvote_project followed by gvote_vote (Algorithm 1 lines 1-3 and 6-10); Q lives in ws. */
+GVOTE_API int32_t gvote_select(const gvote_params* p, const float* H_tilde, const void* h_last,
+                     const void* W_q, int64_t wq_ld, const float* b_q_or_null,
+                     const void* K, int64_t k_tok_stride, int64_t k_head_stride,
+                     const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                     uint32_t* mask, int32_t* budget, int32_t* b_step,
+                     float* dbg_probs_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 line 11.  In place: for every request r and KV head h the kept rows of K and V
+ * move, in ascending key order, to rows cu_seqlens[r] .. cu_seqlens[r]+budget[r][h]-1 of the
+ * head's slab; rows behind them are left as they are.  budget [batch, n_kv_heads] is written
+ * (popcount of the mask).  Rows are d_k bf16 values, moved in 16-byte pieces. */
+GVOTE_API int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t tok_stride, int64_t head_stride,
+                      const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch,
+                      int64_t total_tokens, int64_t max_N, int32_t* budget,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1, whole: fit, sample, project, vote, compact for one layer.  The current query's
+ * hidden state is the last row of each request in h unless h_last_or_null is given.
+ * Outputs: mask, budget, b_step as in gvote_vote; K and V compacted in place. */
+GVOTE_API int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_stride, const void* h_last_or_null,
+                       const void* W_q, int64_t wq_ld, const float* b_q_or_null,
+                       void* K, void* V, int64_t tok_stride, int64_t head_stride,
+                       const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                       uint32_t* mask, int32_t* budget, int32_t* b_step,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/* The same pass for a caller whose tensors live in HOST memory (pinned memory gives full copy
+ * speed): all pointers are host pointers, K and V are dense ([n_kv_heads, total_tokens, d_k]),
+ * h is dense [total_tokens, d_h].  The call copies the inputs to device buffers it keeps in a
+ * grow-only per-device arena (released by gvote_host_arena_release), runs gvote_compress on an
+ * internal stream, copies mask, budget, b_step and the compacted K and V back, and returns after
+ * everything has completed.  This is the only entry point that allocates or synchronises. */
+GVOTE_API int32_t gvote_compress_host(const gvote_params* p, const void* h, const void* W_q, const float* b_q_or_null,
+                            void* K, void* V, const int32_t* cu_seqlens_host, int32_t batch,
+                            uint32_t* mask, int32_t* budget, int32_t* b_step);
+GVOTE_API void gvote_host_arena_release(void);
+
+/* Reads the status word of a workspace (synchronises the stream): GVOTE_OK or GVOTE_ERR_TIMEOUT. */
+GVOTE_API int32_t gvote_poll_status(void* ws, void* stream);
+
+/* Number of kernel launches the library has enqueued in this process (all entry points). */
+GVOTE_API int64_t gvote_launch_count(void);
+
+GVOTE_API const char* gvote_status_string(int32_t status);
+/* Text of the last CUDA error seen by the calling thread's last failing call ("" if none). */
+GVOTE_API const char* gvote_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GVOTE_H_ */

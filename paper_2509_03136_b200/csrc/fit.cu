@@ -1,0 +1,147 @@
+// Step 2 of the GVote scheme (Algorithm 1, line 4): per-channel mean and unbiased variance of the
+// hidden states along the sequence axis, skipping the first n_s sink tokens of every request.
+//
+// The hidden-state matrix is the largest tensor the pass touches (16 KiB per token at d_h = 4096
+// in fp32), so this is a pure HBM stream: each CTA owns a strip of 256 channels and a chunk of
+// rows, every thread keeps shifted first and second moments of four channels in registers, and
+// one (mean, M2) pair per channel and chunk goes to scratch.  A second, tiny kernel merges the
+// chunks with Chan's parallel-variance update in fp64.
+#include "common.cuh"
+
+namespace gvote {
+namespace {
+
+constexpr int kFitTx = 64;   // column threads (x4 channels each)
+constexpr int kFitTy = 4;    // row lanes
+
+template <typename T>
+__device__ __forceinline__ float4 load4(const T* p);
+template <>
+__device__ __forceinline__ float4 load4<float>(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+template <>
+__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
+  uint2 u = __ldcs(reinterpret_cast<const uint2*>(p));
+  float4 r;
+  r.x = __uint_as_float(u.x << 16);
+  r.y = __uint_as_float(u.x & 0xffff0000u);
+  r.z = __uint_as_float(u.y << 16);
+  r.w = __uint_as_float(u.y & 0xffff0000u);
+  return r;
+}
+
+__device__ __forceinline__ void acc4(float4& s1, float4& s2, const float4& v, const float4& sh) {
+  float dx = v.x - sh.x, dy = v.y - sh.y, dz = v.z - sh.z, dw = v.w - sh.w;
+  s1.x += dx; s1.y += dy; s1.z += dz; s1.w += dw;
+  s2.x = fmaf(dx, dx, s2.x); s2.y = fmaf(dy, dy, s2.y);
+  s2.z = fmaf(dz, dz, s2.z); s2.w = fmaf(dw, dw, s2.w);
+}
+
+// Rows of chunk `c` of a request whose fitted rows are [first, last): [a, b).
+__device__ __forceinline__ void chunk_rows(int first, int last, int chunks, int c, int& a, int& b) {
+  int n = max(last - first, 0);
+  int per = (n + chunks - 1) / chunks;
+  a = min(first + c * per, last);
+  b = min(a + per, last);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kFitTx* kFitTy)
+fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restrict__ cu, int n_s, int d_h,
+                   int chunks, float2* __restrict__ partial) {
+  const int r = blockIdx.z, c = blockIdx.y;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int col = (blockIdx.x * kFitTx + tx) * 4;
+  const bool active = col < d_h;
+  int a, b;
+  chunk_rows(cu[r] + n_s, cu[r + 1], chunks, c, a, b);
+
+  float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1, sh = s1;
+  if (active && a < b) {
+    const T* base = h + col;
+    sh = load4<T>(base + (int64_t)a * ld);   // shift: the chunk's first row (same for all row lanes)
+    int i = a + ty;
+    for (; i + 3 * kFitTy < b; i += 4 * kFitTy) {
+      float4 v0 = load4<T>(base + (int64_t)i * ld);
+      float4 v1 = load4<T>(base + (int64_t)(i + kFitTy) * ld);
+      float4 v2 = load4<T>(base + (int64_t)(i + 2 * kFitTy) * ld);
+      float4 v3 = load4<T>(base + (int64_t)(i + 3 * kFitTy) * ld);
+      acc4(s1, s2, v0, sh); acc4(s1, s2, v1, sh); acc4(s1, s2, v2, sh); acc4(s1, s2, v3, sh);
+    }
+    for (; i < b; i += kFitTy) {
+      float4 v = load4<T>(base + (int64_t)i * ld);
+      acc4(s1, s2, v, sh);
+    }
+  }
+  __shared__ float4 sm1[kFitTy][kFitTx], sm2[kFitTy][kFitTx];
+  sm1[ty][tx] = s1;
+  sm2[ty][tx] = s2;
+  __syncthreads();
+  if (ty == 0 && active) {
+    double t1[4] = {0, 0, 0, 0}, t2[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < kFitTy; ++j) {
+      float4 u = sm1[j][tx], w = sm2[j][tx];
+      t1[0] += u.x; t1[1] += u.y; t1[2] += u.z; t1[3] += u.w;
+      t2[0] += w.x; t2[1] += w.y; t2[2] += w.z; t2[3] += w.w;
+    }
+    const int n = b - a;
+    const float shv[4] = {sh.x, sh.y, sh.z, sh.w};
+    float2* out = partial + ((int64_t)(r * chunks + c)) * d_h + col;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      double mean = 0.0, m2 = 0.0;
+      if (n > 0) {
+        mean = (double)shv[j] + t1[j] / n;
+        m2 = t2[j] - t1[j] * t1[j] / n;
+      }
+      out[j] = make_float2((float)mean, (float)fmax(m2, 0.0));
+    }
+  }
+}
+
+// Chan et al. pairwise update over the chunks of a request, in fp64; one thread per channel.
+__global__ void fit_finalize_kernel(const float2* __restrict__ partial, const int32_t* __restrict__ cu, int n_s,
+                                    int d_h, int chunks, float* __restrict__ mu, float* __restrict__ var) {
+  const int r = blockIdx.y;
+  const int col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= d_h) return;
+  const int first = cu[r] + n_s, last = cu[r + 1];
+  double n = 0.0, mean = 0.0, m2 = 0.0;
+  for (int c = 0; c < chunks; ++c) {
+    int a, b;
+    chunk_rows(first, last, chunks, c, a, b);
+    const double nc = (double)(b - a);
+    if (nc <= 0.0) continue;
+    const float2 pc = partial[((int64_t)(r * chunks + c)) * d_h + col];
+    const double delta = (double)pc.x - mean;
+    const double tot = n + nc;
+    mean += delta * nc / tot;
+    m2 += (double)pc.y + delta * delta * n * nc / tot;
+    n = tot;
+  }
+  mu[(int64_t)r * d_h + col] = (float)mean;
+  var[(int64_t)r * d_h + col] = (float)(m2 / (n - 1.0));   // NaN/inf when fewer than 2 rows
+}
+
+}  // namespace
+
+int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                   int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st) {
+  const int strips = (int)ceil_div(p->d_h, kFitStripCols);
+  dim3 grid(strips, fit_chunks, batch), block(kFitTx, kFitTy);
+  if (p->h_dtype == GVOTE_DTYPE_F32) {
+    fit_partial_kernel<float><<<grid, block, 0, st>>>((const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks, partial);
+  } else {
+    fit_partial_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)h, ld, cu, p->n_s, p->d_h,
+                                                              fit_chunks, partial);
+  }
+  GVOTE_LAUNCH_CHECK("fit_partial_kernel");
+  dim3 g2((unsigned)ceil_div(p->d_h, 128), batch);
+  fit_finalize_kernel<<<g2, 128, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
+  GVOTE_LAUNCH_CHECK("fit_finalize_kernel");
+  return GVOTE_OK;
+}
+
+}  // namespace gvote

@@ -1,0 +1,420 @@
+// Algorithm 1 lines 1-3 and 8-10: attention logits of the current query and of the S synthetic
+// queries against all cached keys, the current query's top-p set size |C0| (the step budget),
+// each synthetic query's selection (top-k with k = |C0|, or top-p in the alternative mode), and
+// the union of the selections as one keep bit-mask per KV head.
+//
+// Selection never sorts.  A row's threshold is found by a most-significant-digit radix search
+// over an order-preserving 32-bit image of the fp32 logit: three histogram passes (11, 11 and 10
+// bits) in shared memory narrow the threshold to one exact value; counts are integers and
+// softmax mass is accumulated in 2^-40 fixed point, so the search is order independent and two
+// runs give the same bits.  Ties at the threshold go to the lower key index.  The union is a
+// warp ballot per 32 keys OR-ed into the mask word.
+#include "common.cuh"
+
+namespace gvote {
+namespace {
+
+constexpr int kSelThreads = 256;
+constexpr float kFixScale = 1099511627776.0f;   // 2^40
+
+// ---------------------------------------------------------------------------------- logits (SIMT)
+// logits[row][n] = (Q[row] . K[n]) / sqrt(d_k) for the rows of one KV head's group.
+// CTA: 64 keys x all group rows; thread: 2 keys x 8 rows.
+constexpr int kScoreKeys = 64;
+constexpr int kScoreRowChunk = 64;
+
+__global__ void __launch_bounds__(256)
+score_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K, int64_t k_tok,
+                  int64_t k_head, const int32_t* __restrict__ cu, int Hq, int G, int S1, int d_k, float scale,
+                  float* __restrict__ logits) {
+  extern __shared__ __align__(16) uint32_t smem_u32[];
+  const int r = blockIdx.z, kh = blockIdx.y;
+  const int start = cu[r], N = cu[r + 1] - start;
+  const int n0 = blockIdx.x * kScoreKeys;
+  if (n0 >= N) return;
+  const int half = d_k / 2;               // bf16 pairs per row
+  const int kpitch = half + 1;            // odd pitch: conflict-free across keys
+  uint32_t* Ks = smem_u32;                              // [64][kpitch]
+  uint32_t* Qs = smem_u32 + kScoreKeys * kpitch;        // [64][half]
+  const int tid = threadIdx.x, lane = tid & 31, rg = tid >> 5;   // 8 row groups of 8 rows
+
+  const __nv_bfloat16* Kbase = K + (int64_t)kh * k_head + (int64_t)(start + n0) * k_tok;
+  for (int idx = tid; idx < kScoreKeys * half; idx += blockDim.x) {
+    const int key = idx / half, d2 = idx % half;
+    uint32_t v = 0;
+    if (n0 + key < N) v = *reinterpret_cast<const uint32_t*>(Kbase + (int64_t)key * k_tok + 2 * d2);
+    Ks[key * kpitch + d2] = v;
+  }
+  const int R = G * S1;
+  const __nv_bfloat16* Qbase = Q + ((int64_t)r * Hq + (int64_t)kh * G) * S1 * d_k;   // rows of the group are contiguous
+  float* Lbase = logits + (int64_t)Hq * S1 * start + (int64_t)kh * G * S1 * N;
+
+  for (int c0 = 0; c0 < R; c0 += kScoreRowChunk) {
+    __syncthreads();
+    for (int idx = tid; idx < kScoreRowChunk * half; idx += blockDim.x) {
+      const int row = idx / half, d2 = idx % half;
+      uint32_t v = 0;
+      if (c0 + row < R) v = *reinterpret_cast<const uint32_t*>(Qbase + (int64_t)(c0 + row) * d_k + 2 * d2);
+      Qs[row * half + d2] = v;
+    }
+    __syncthreads();
+    float acc0[8], acc1[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+    for (int d2 = 0; d2 < half; ++d2) {
+      const float2 ka = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&Ks[lane * kpitch + d2]));
+      const float2 kb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&Ks[(lane + 32) * kpitch + d2]));
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&Qs[(rg * 8 + j) * half + d2]));
+        acc0[j] = fmaf(q.x, ka.x, acc0[j]); acc0[j] = fmaf(q.y, ka.y, acc0[j]);
+        acc1[j] = fmaf(q.x, kb.x, acc1[j]); acc1[j] = fmaf(q.y, kb.y, acc1[j]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int row = c0 + rg * 8 + j;
+      if (row < R) {
+        if (n0 + lane < N) Lbase[(int64_t)row * N + n0 + lane] = acc0[j] * scale;
+        if (n0 + lane + 32 < N) Lbase[(int64_t)row * N + n0 + lane + 32] = acc1[j] * scale;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------- block helpers
+struct SelShared {
+  uint32_t cnt[2048];
+  unsigned long long mass[2048];
+  unsigned long long red64[kSelThreads / 32];
+  uint32_t red32[kSelThreads / 32];
+  float redf[kSelThreads / 32];
+  // results of a digit search
+  int bin;
+  uint32_t cnt_above;
+  unsigned long long mass_above;
+  int tie_base;
+};
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float m = red[0];
+#pragma unroll
+  for (int i = 1; i < kSelThreads / 32; ++i) m = fmaxf(m, red[i]);
+  __syncthreads();
+  return m;
+}
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* red) {
+  v = warp_sum_u64(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long s = 0;
+#pragma unroll
+  for (int i = 0; i < kSelThreads / 32; ++i) s += red[i];
+  __syncthreads();
+  return s;
+}
+__device__ __forceinline__ uint32_t block_sum_u32(uint32_t v, uint32_t* red) {
+  v = (uint32_t)warp_sum_i((int)v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  uint32_t s = 0;
+#pragma unroll
+  for (int i = 0; i < kSelThreads / 32; ++i) s += red[i];
+  __syncthreads();
+  return s;
+}
+
+// exp(l - max) in 2^-40 fixed point (l <= max, so the value is in [0, 2^40]).
+__device__ __forceinline__ unsigned long long mass_fix(float l, float mx) {
+  return __float2ull_rn(expf(l - mx) * kFixScale);
+}
+
+// Find the highest bin b of hist[0..nbins) whose suffix sum (bins >= b) reaches `need`;
+// publish b and the sum of the bins above it.  MASS selects which histogram decides; the count
+// of elements above is always published too.  Requires total >= need (else bin 0 is returned).
+template <bool MASS>
+__device__ void find_bin(SelShared& sh, int nbins, unsigned long long need) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = nbins / kSelThreads;
+  unsigned long long w = 0;
+  uint32_t c = 0;
+  for (int i = 0; i < per; ++i) {
+    const int b = tid * per + i;
+    c += sh.cnt[b];
+    w += MASS ? sh.mass[b] : (unsigned long long)sh.cnt[b];
+  }
+  // suffix sums over threads (exclusive): warp shuffle scan from the top lane down
+  unsigned long long ws = w;
+  uint32_t cs = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long tw = __shfl_down_sync(0xffffffffu, ws, o);
+    const uint32_t tc = __shfl_down_sync(0xffffffffu, cs, o);
+    if (lane + o < 32) { ws += tw; cs += tc; }
+  }
+  if (lane == 0) { sh.red64[warp] = ws; sh.red32[warp] = cs; }
+  if (tid == 0) { sh.bin = 0; sh.cnt_above = 0; sh.mass_above = 0; }
+  __syncthreads();
+  unsigned long long hi_w = 0;
+  uint32_t hi_c = 0;
+  for (int i = warp + 1; i < kSelThreads / 32; ++i) { hi_w += sh.red64[i]; hi_c += sh.red32[i]; }
+  const unsigned long long excl_w = ws - w + hi_w;   // weight in bins of higher threads
+  const uint32_t excl_c = cs - c + hi_c;
+  if (excl_w < need && excl_w + w >= need) {
+    unsigned long long aw = excl_w;
+    uint32_t ac = excl_c;
+    int b = tid * per + per - 1;
+    for (; b > tid * per; --b) {
+      const unsigned long long bw = MASS ? sh.mass[b] : (unsigned long long)sh.cnt[b];
+      if (aw + bw >= need) break;
+      aw += bw;
+      ac += sh.cnt[b];
+    }
+    sh.bin = b;
+    sh.cnt_above = ac;
+    sh.mass_above = aw;
+  }
+  __syncthreads();
+}
+
+// Radix search for the threshold key of one row.
+//   MASS = false: largest t with #(key >= t) >= need            (top-k, need = k)
+//   MASS = true : largest t with mass(key >= t) >= need          (top-p, need = p * Z in fixed point)
+// Outputs (same in every thread): t, number of keys above t, their mass (MASS only: mass above
+// in fixed point), number of keys equal to t.
+template <bool MASS>
+__device__ void radix_threshold(const float* __restrict__ row, int N, float mx, unsigned long long need,
+                                SelShared& sh, uint32_t& t_out, uint32_t& above_cnt,
+                                unsigned long long& above_mass, uint32_t& eq_cnt) {
+  const int tid = threadIdx.x;
+  uint32_t prefix = 0;          // digits fixed so far, left aligned
+  uint32_t cnt_acc = 0;
+  unsigned long long mass_acc = 0;
+  const int shifts[3] = {21, 10, 0};
+  const int bits[3] = {11, 11, 10};
+  uint32_t known_mask = 0;
+  for (int pass = 0; pass < 3; ++pass) {
+    const int nb = 1 << bits[pass];
+    for (int b = tid; b < nb; b += kSelThreads) { sh.cnt[b] = 0; if (MASS) sh.mass[b] = 0; }
+    __syncthreads();
+    for (int n = tid; n < N; n += kSelThreads) {
+      const float l = row[n];
+      const uint32_t key = ordered_key(l);
+      if ((key & known_mask) == prefix) {
+        const int b = (key >> shifts[pass]) & (nb - 1);
+        atomicAdd(&sh.cnt[b], 1u);
+        if (MASS) atomicAdd(&sh.mass[b], mass_fix(l, mx));
+      }
+    }
+    __syncthreads();
+    const unsigned long long remaining = need - (MASS ? mass_acc : (unsigned long long)cnt_acc);
+    find_bin<MASS>(sh, nb, remaining);
+    const int b = sh.bin;
+    cnt_acc += sh.cnt_above;
+    mass_acc += sh.mass_above;
+    if (pass == 2) eq_cnt = sh.cnt[b];
+    prefix |= ((uint32_t)b) << shifts[pass];
+    known_mask |= ((uint32_t)(nb - 1)) << shifts[pass];
+    __syncthreads();
+  }
+  t_out = prefix;
+  above_cnt = cnt_acc;
+  above_mass = mass_acc;
+}
+
+// OR the row's selection into the mask: keys above t, plus the first `ties` keys equal to t.
+__device__ void emit_row(const float* __restrict__ row, int N, uint32_t t, uint32_t ties, uint32_t eq_cnt,
+                         uint32_t* __restrict__ mask_row, SelShared& sh) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool all_ties = ties >= eq_cnt;
+  uint32_t taken = 0;   // ties taken so far (ordered path only)
+  for (int base = 0; base < N; base += kSelThreads) {
+    const int n = base + tid;
+    uint32_t key = 0;
+    bool valid = n < N;
+    if (valid) key = ordered_key(row[n]);
+    bool sel = valid && key > t;
+    const bool tie = valid && key == t;
+    if (all_ties) {
+      sel |= tie;
+    } else if (ties > 0) {
+      // ordered: rank of this tie among all ties of the row, by index
+      const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+      if (lane == 0) sh.red32[warp] = __popc(tb);
+      __syncthreads();
+      uint32_t before = taken;
+      for (int w = 0; w < warp; ++w) before += sh.red32[w];
+      uint32_t total = 0;
+      for (int w = 0; w < kSelThreads / 32; ++w) total += sh.red32[w];
+      const uint32_t rank = before + __popc(tb & ((1u << lane) - 1u));
+      sel |= tie && rank < ties;
+      taken += total;
+      __syncthreads();
+    }
+    const uint32_t bal = __ballot_sync(0xffffffffu, sel);
+    if (lane == 0 && bal) atomicOr(&mask_row[n >> 5], bal);
+  }
+}
+
+// ---------------------------------------------------------------------------------- top-p rows
+// One CTA per row.  rows_per_head = 1: only the current query's row of every head (row 0);
+// rows_per_head = S+1: every row (top-p mode).  Row 0 always publishes b_step = |C0|.
+__global__ void __launch_bounds__(kSelThreads)
+topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
+                 int rows_per_head, float p_nuc, int include_c0, int64_t row_words, uint32_t* __restrict__ mask,
+                 int32_t* __restrict__ b_step) {
+  __shared__ SelShared sh;
+  const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x;   // row < rows_per_head
+  const int start = cu[r], N = cu[r + 1] - start;
+  if (N <= 0) { if (row == 0 && threadIdx.x == 0) b_step[r * Hq + g] = 0; return; }
+  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  const int tid = threadIdx.x;
+
+  float mx = -INFINITY;
+  for (int n = tid; n < N; n += kSelThreads) mx = fmaxf(mx, L[n]);
+  mx = block_max(mx, sh.redf);
+  unsigned long long z = 0;
+  for (int n = tid; n < N; n += kSelThreads) z += mass_fix(L[n], mx);
+  z = block_sum_u64(z, sh.red64);
+  // smallest integer mass that is >= p * Z
+  unsigned long long need = (unsigned long long)ceil((double)p_nuc * (double)z);
+  if (need > z) need = z;
+  if (need == 0) need = 1;
+
+  uint32_t t, above_cnt, eq_cnt;
+  unsigned long long above_mass;
+  radix_threshold<true>(L, N, mx, need, sh, t, above_cnt, above_mass, eq_cnt);
+  // every key equal to t has the same logit, hence the same mass e_t: take the fewest that reach p
+  float lt;
+  {
+    const uint32_t u = (t & 0x80000000u) ? (t & 0x7fffffffu) : ~t;
+    lt = __uint_as_float(u);
+  }
+  const unsigned long long e_t = mass_fix(lt, mx);
+  uint32_t ties = eq_cnt;
+  if (e_t > 0) {
+    const unsigned long long lack = need - above_mass;             // > 0 by construction
+    const unsigned long long j = (lack + e_t - 1) / e_t;
+    ties = (uint32_t)(j < (unsigned long long)eq_cnt ? j : eq_cnt);
+  }
+  if (ties == 0) ties = 1;
+  if (row == 0 && tid == 0) b_step[r * Hq + g] = (int32_t)(above_cnt + ties);
+  const bool emit = (row == 0) ? (include_c0 != 0) : true;
+  if (emit) {
+    uint32_t* mrow = mask + (int64_t)(g / G) * row_words + mask_word_offset(start, r);
+    emit_row(L, N, t, ties, eq_cnt, mrow, sh);
+  }
+}
+
+// ---------------------------------------------------------------------------------- top-k rows
+// One CTA per synthetic row: the b_step[g] largest logits, ties to the lower index.
+__global__ void __launch_bounds__(kSelThreads)
+topk_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
+                 const int32_t* __restrict__ b_step, int64_t row_words, uint32_t* __restrict__ mask) {
+  __shared__ SelShared sh;
+  const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x + 1;
+  const int start = cu[r], N = cu[r + 1] - start;
+  if (N <= 0) return;
+  int k = b_step[r * Hq + g];
+  if (k <= 0) return;
+  if (k > N) k = N;
+  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  uint32_t t, above_cnt, eq_cnt;
+  unsigned long long above_mass;
+  radix_threshold<false>(L, N, 0.f, (unsigned long long)k, sh, t, above_cnt, above_mass, eq_cnt);
+  const uint32_t ties = (uint32_t)k - above_cnt;
+  uint32_t* mrow = mask + (int64_t)(g / G) * row_words + mask_word_offset(start, r);
+  emit_row(L, N, t, ties, eq_cnt, mrow, sh);
+}
+
+// ---------------------------------------------------------------------------------- softmax dump
+__global__ void __launch_bounds__(kSelThreads)
+softmax_dump_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int S1,
+                    float* __restrict__ probs) {
+  __shared__ float red[kSelThreads / 32];
+  __shared__ double redd[kSelThreads / 32];
+  const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x;
+  const int start = cu[r], N = cu[r + 1] - start;
+  const int64_t off = (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  const float* L = logits + off;
+  const int tid = threadIdx.x;
+  float mx = -INFINITY;
+  for (int n = tid; n < N; n += kSelThreads) mx = fmaxf(mx, L[n]);
+  mx = block_max(mx, red);
+  double z = 0.0;
+  for (int n = tid; n < N; n += kSelThreads) z += (double)expf(L[n] - mx);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+  if ((tid & 31) == 0) redd[tid >> 5] = z;
+  __syncthreads();
+  double zt = 0.0;
+  for (int i = 0; i < kSelThreads / 32; ++i) zt += redd[i];
+  const float inv = (float)(1.0 / zt);
+  for (int n = tid; n < N; n += kSelThreads) probs[off + n] = expf(L[n] - mx) * inv;
+}
+
+// ---------------------------------------------------------------------------------- budgets
+__global__ void __launch_bounds__(256)
+budget_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu, int Hkv, int64_t row_words,
+              int32_t* __restrict__ budget) {
+  __shared__ uint32_t red[8];
+  const int r = blockIdx.y, h = blockIdx.x;
+  const int start = cu[r], N = cu[r + 1] - start;
+  const int words = (N + 31) >> 5;
+  const uint32_t* m = mask + (int64_t)h * row_words + mask_word_offset(start, r);
+  uint32_t c = 0;
+  for (int w = threadIdx.x; w < words; w += blockDim.x) c += __popc(m[w]);
+  c = block_sum_u32(c, red);
+  if (threadIdx.x == 0) budget[r * Hkv + h] = (int32_t)c;
+}
+
+}  // namespace
+
+int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                    int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                    uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs, const WorkspaceMap& m,
+                    char* ws, cudaStream_t st) {
+  const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
+  float* logits = reinterpret_cast<float*>(ws + m.logits);
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(mask, 0, (size_t)Hkv * m.row_words * sizeof(uint32_t), st));
+
+  {
+    const int half = d_k / 2;
+    const size_t smem = ((size_t)kScoreKeys * (half + 1) + (size_t)kScoreRowChunk * half) * sizeof(uint32_t);
+    if (smem > 48 * 1024) {
+      GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    dim3 grid((unsigned)ceil_div(max_N, kScoreKeys), Hkv, batch);
+    score_simt_kernel<<<grid, 256, smem, st>>>(Q, K, k_tok, k_head, cu, Hq, G, S1, d_k,
+                                               (float)(1.0 / sqrt((double)d_k)), logits);
+    GVOTE_LAUNCH_CHECK("score_simt_kernel");
+  }
+  if (dbg_probs) {
+    dim3 grid(S1, Hq, batch);
+    softmax_dump_kernel<<<grid, kSelThreads, 0, st>>>(logits, cu, Hq, S1, dbg_probs);
+    GVOTE_LAUNCH_CHECK("softmax_dump_kernel");
+  }
+  if (p->sel_mode == GVOTE_SEL_TOPK_C0) {
+    dim3 g1(1, Hq, batch);
+    topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0, m.row_words,
+                                                 mask, b_step);
+    GVOTE_LAUNCH_CHECK("topp_rows_kernel");
+    dim3 g2(p->S, Hq, batch);
+    topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask);
+    GVOTE_LAUNCH_CHECK("topk_rows_kernel");
+  } else {
+    dim3 g1(S1, Hq, batch);
+    topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0, m.row_words,
+                                                 mask, b_step);
+    GVOTE_LAUNCH_CHECK("topp_rows_kernel");
+  }
+  dim3 gb(Hkv, batch);
+  budget_kernel<<<gb, 256, 0, st>>>(mask, cu, Hkv, m.row_words, budget);
+  GVOTE_LAUNCH_CHECK("budget_kernel");
+  return GVOTE_OK;
+}
+
+}  // namespace gvote

@@ -1,0 +1,374 @@
+"""Parity of the CUDA library against the CPU oracle, stage by stage and end to end, through the
+C ABI.  Tolerances (stated where used): Philox words and compaction bit-exact; fit 1e-5 relative;
+normal draws 1e-5 absolute on z; rotated queries within one bf16 step; softmax rows 2e-2 relative
+where the weight is >= 1e-6; masks identical outside the 1e-3 band around each selection
+threshold; budgets within 0.5 % of N."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gvote_oracle as o
+from paper_2509_03136_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gv():
+    from paper_2509_03136_b200 import build as gbuild
+    gbuild.build()
+    from paper_2509_03136_b200 import gvote
+    gvote.load()
+    return gvote
+
+
+def _geom(cfg):
+    return (cfg.batch, cfg.total_tokens, max(cfg.seq_lens))
+
+
+def _small_cfgs():
+    return [
+        synth.make_small(1, seq_lens=(40,), S=4),
+        synth.make_small(2, seq_lens=(33, 64, 17), S=5, d_h=72, d_k=16),
+        synth.make_small(3, seq_lens=(129, 31, 257), S=7, d_h=256, n_q_heads=6, n_kv_heads=2, d_k=64, n_f=16),
+        synth.make_small(4, seq_lens=(1000,), S=9, d_h=128, n_q_heads=2, n_kv_heads=2, d_k=128, p_nuc=0.99),
+    ]
+
+
+# ----------------------------------------------------------------------------- sample
+@pytest.mark.parametrize("d_h,S,batch", [(512, 16, 1), (72, 3, 4), (4096, 32, 2)])
+def test_sample_philox_bit_exact_and_normals(gv, d_h, S, batch):
+    seed, layer = 0x0123456789ABCDEF, 11
+    p = gv.make_params(d_h=d_h, n_q_heads=8, n_kv_heads=2, d_k=64, rope_theta=1e4, S=S, p_nuc=0.95, n_f=8, n_s=0,
+                       seed=seed, layer_id=layer)
+    rng = np.random.default_rng(5)
+    mu = rng.normal(size=(batch, d_h)).astype(np.float32)
+    var = rng.uniform(0.1, 10, size=(batch, d_h)).astype(np.float32)
+    H = torch.empty(batch, S, d_h, device="cuda")
+    raw = torch.empty(batch, S, d_h, dtype=torch.int32, device="cuda")
+    gv.gvote_sample(p, torch.from_numpy(mu).cuda(), torch.from_numpy(var).cuda(), batch, H, raw)
+    H, raw = H.cpu().numpy(), raw.cpu().numpy().view(np.uint32)
+    for r in range(batch):
+        Ho, rawo = o.sample(mu[r].astype(np.float64), var[r].astype(np.float64), S, seed, layer, r)
+        assert np.array_equal(raw[r], rawo[:, :d_h])                                   # bit-exact
+        sig = np.sqrt(var[r].astype(np.float64))
+        z_gpu = (H[r] - mu[r]) / sig
+        z_or = (Ho - mu[r]) / sig
+        assert np.abs(z_gpu - z_or).max() < 1e-5 + 2e-6 * np.abs(mu[r] / sig).max()    # 1e-5 abs on z
+
+
+# ----------------------------------------------------------------------------- fit
+@pytest.mark.parametrize("name,lens,d_h,n_s", [("a", (40,), 64, 2), ("b", (33, 64, 17), 72, 4),
+                                               ("c", (5000, 700), 1024, 4), ("d", (6,), 8, 4)])
+def test_fit_matches_oracle(gv, name, lens, d_h, n_s):
+    rng = np.random.default_rng(7)
+    T = sum(lens)
+    h = (rng.normal(size=(T, d_h)) * rng.uniform(0.3, 3, size=d_h) + rng.normal(size=d_h) * 5).astype(np.float32)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    p = gv.make_params(d_h=d_h, n_q_heads=2, n_kv_heads=1, d_k=16, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=n_s,
+                       seed=0)
+    geom = (len(lens), T, max(lens))
+    ws = gv.alloc_workspace(p, *geom)
+    mu = torch.empty(len(lens), d_h, device="cuda")
+    var = torch.empty_like(mu)
+    gv.gvote_fit(p, torch.from_numpy(h).cuda(), torch.from_numpy(cu).cuda(), geom, mu, var, ws)
+    for r in range(len(lens)):
+        m, v = o.fit(h[cu[r]:cu[r + 1]], n_s)
+        assert np.allclose(var[r].cpu().numpy(), v, rtol=1e-5, atol=0)
+        assert np.abs(mu[r].cpu().numpy() - m).max() <= 1e-5 * np.sqrt(v).max() + 1e-6 * np.abs(m).max()
+
+
+def test_fit_bf16_hidden_states(gv):
+    rng = np.random.default_rng(8)
+    h = torch.from_numpy(rng.normal(size=(300, 128)).astype(np.float32)).bfloat16()
+    cu = np.array([0, 300], dtype=np.int32)
+    p = gv.make_params(d_h=128, n_q_heads=2, n_kv_heads=1, d_k=16, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=4,
+                       seed=0, h_dtype=gv.DTYPE_BF16)
+    geom = (1, 300, 300)
+    ws = gv.alloc_workspace(p, *geom)
+    mu = torch.empty(1, 128, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p, h.cuda(), torch.from_numpy(cu).cuda(), geom, mu, var, ws)
+    m, v = o.fit(h.double().numpy(), 4)
+    assert np.allclose(var[0].cpu().numpy(), v, rtol=1e-5) and np.allclose(mu[0].cpu().numpy(), m, atol=1e-5)
+
+
+# ----------------------------------------------------------------------------- project
+@pytest.mark.parametrize("idx", range(4))
+@pytest.mark.parametrize("bias", [False, True])
+def test_project_matches_oracle(gv, idx, bias):
+    cfg = _small_cfgs()[idx]
+    li = synth.make_layer(cfg, 0, with_bias=bias)
+    p = gv.params_from_config(cfg)
+    rng = np.random.default_rng(9)
+    Ht = rng.normal(size=(cfg.batch, cfg.S, cfg.d_h)).astype(np.float32) * 2
+    hl = rng.normal(size=(cfg.batch, cfg.d_h)).astype(np.float32)
+    d = pu.upload_layer(li, gv, torch)
+    ws = gv.alloc_workspace(p, *_geom(cfg))
+    Q = torch.empty(cfg.batch, cfg.n_q_heads, cfg.S + 1, cfg.d_k, dtype=torch.bfloat16, device="cuda")
+    gv.gvote_project(p, torch.from_numpy(Ht).cuda(), torch.from_numpy(hl).cuda(), d["W_q"], d["b_q"], d["cu"],
+                     cfg.batch, Q, ws)
+    Qg = Q.float().cpu().numpy().astype(np.float64)
+    W = o.bf16_bits_to_f64(li.W_q)
+    for r in range(cfg.batch):
+        Qo = o.queries_for_request(Ht[r].astype(np.float64), hl[r].astype(np.float64), W, li.b_q, cfg.seq_lens[r],
+                                   n_q_heads=cfg.n_q_heads, d_k=cfg.d_k, theta=cfg.rope_theta, n_f=cfg.n_f)
+        diff = np.abs(Qg[r] - Qo)
+        assert np.all(diff <= 2.0 ** -7 * np.abs(Qo) + 1e-6)            # at most one bf16 step
+        assert (diff == 0).mean() > 0.98
+
+
+# ----------------------------------------------------------------------------- vote (given the oracle's queries)
+def _run_vote(gv, cfg, li, Q_or, sel_mode, include_c0, want_probs):
+    p = gv.params_from_config(cfg, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0,
+                              include_c0=include_c0)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    K = gv.bf16_from_bits(li.K)
+    cu = torch.from_numpy(li.cu_seqlens).cuda()
+    Qd = torch.from_numpy(np.ascontiguousarray(np.stack(Q_or))).to(torch.bfloat16).contiguous().cuda()      # values are on the bf16 grid already
+    mask = torch.full((cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch)), -1, dtype=torch.int32,
+                      device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    probs = None
+    if want_probs:
+        probs = torch.empty(cfg.n_q_heads * (cfg.S + 1) * cfg.total_tokens, device="cuda")
+    gv.gvote_vote(p, Qd, K, cu, geom, mask, budget, b_step, ws, probs)
+    assert gv.gvote_poll_status(ws) == 0
+    return mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), None if probs is None else probs.cpu().numpy()
+
+
+def _oracle_queries(cfg, li, seed=None):
+    W = o.bf16_bits_to_f64(li.W_q)
+    out = []
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        h = li.h[a:b].astype(np.float64)
+        mu, var = o.fit(h, cfg.n_s)
+        Ht, _ = o.sample(mu, var, cfg.S, cfg.seed if seed is None else seed, 0, r)
+        out.append(o.queries_for_request(Ht, h[-1], W, li.b_q, b - a, n_q_heads=cfg.n_q_heads, d_k=cfg.d_k,
+                                         theta=cfg.rope_theta, n_f=cfg.n_f))
+    return out
+
+
+def _check_vote(gv, cfg, li, sel_mode, include_c0=False, want_probs=True):
+    Q_or = _oracle_queries(cfg, li)
+    mask, budget, b_step, probs = _run_vote(gv, cfg, li, Q_or, sel_mode, include_c0, want_probs)
+    pf = float(np.float32(cfg.p_nuc))
+    poff = 0
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        N = b - a
+        Kr = o.bf16_bits_to_f64(li.K[:, a:b])
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N) for h in range(cfg.n_kv_heads)])
+        pu.check_vote_against_oracle(Q_or[r], Kr, pf, sel_mode, include_c0, gm, b_step[r])
+        om, ob, obs, _, op = o.vote(Q_or[r], Kr, p_nuc=pf, sel_mode=sel_mode, include_c0=include_c0,
+                                    keep_probs=want_probs)
+        assert np.array_equal(budget[r], gm.sum(axis=1))                     # budget = popcount
+        assert np.all(np.abs(budget[r] - ob) <= max(1, 0.005 * N))           # within 0.5 % of N
+        assert (gm != om).sum() <= max(2, 0.005 * N * cfg.n_kv_heads)
+        if want_probs:
+            pg = probs[poff:poff + cfg.n_q_heads * (cfg.S + 1) * N].reshape(cfg.n_q_heads, cfg.S + 1, N)
+            big = op >= 1e-6
+            assert np.abs(pg[big] / op[big] - 1.0).max() < 2e-2              # stated score tolerance
+            poff += cfg.n_q_heads * (cfg.S + 1) * N
+        # padding bits of the request's last word stay zero
+        if N % 32:
+            last = mask[:, gv.mask_word_offset(a, r) + N // 32].view(np.uint32)
+            assert np.all(last >> np.uint32(N % 32) == 0)
+
+
+@pytest.mark.parametrize("idx", range(4))
+@pytest.mark.parametrize("mode", ["topk", "topp"])
+def test_vote_small(gv, idx, mode):
+    cfg = _small_cfgs()[idx]
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode)
+
+
+def test_vote_include_c0(gv):
+    cfg = _small_cfgs()[2]
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", include_c0=True)
+
+
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c1", "topp")])
+def test_vote_configs(gv, name, mode):
+    cfg = synth.make_config(name)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode)
+
+
+def test_vote_degenerate_all_keys_equal(gv):
+    """Every logit ties: top-p keeps ceil(p N) keys and top-k keeps exactly k, lowest indices first."""
+    cfg = synth.make_small(5, seq_lens=(100,), S=3, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=32, p_nuc=0.5)
+    li = synth.make_layer(cfg, 0)
+    li.K[:] = li.K[:, :1, :]                                                 # one key repeated
+    Q_or = _oracle_queries(cfg, li)
+    mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    assert b_step.tolist() == [[50, 50]] and budget.tolist() == [[50]]
+    gm = gv.unpack_mask(mask[0], 0, 100)
+    assert gm[:50].all() and not gm[50:].any()
+
+
+def test_vote_single_dominant_key(gv):
+    cfg = synth.make_small(6, seq_lens=(77,), S=4, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=32, p_nuc=0.95)
+    li = synth.make_layer(cfg, 0)
+    Q_or = _oracle_queries(cfg, li)
+    Kf = np.zeros((1, 77, 32), dtype=np.float32)
+    # key 13 lines up with every row of every head by construction: sum of the sign patterns
+    qsum = np.sign(np.concatenate([Q_or[0][g] for g in range(2)]).sum(axis=0))
+    Kf[0, 13] = 40.0 * qsum
+    li.K = synth.f32_to_bf16_bits(Kf)
+    Kr = o.bf16_bits_to_f64(li.K)
+    om, ob, obs, _, _ = o.vote(Q_or[0], Kr, p_nuc=float(np.float32(0.95)))
+    mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    assert b_step[0].tolist() == obs.tolist()
+    assert np.array_equal(gv.unpack_mask(mask[0], 0, 77), om[0])
+
+
+# ----------------------------------------------------------------------------- compact
+@pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
+                                                  ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
+                                                  ((1000,), 1, 8, 1.0), ((1000,), 1, 16, 0.0)])
+def test_compact_bit_exact(gv, lens, Hkv, d_k, density):
+    rng = np.random.default_rng(12)
+    T, B = sum(lens), len(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    K = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
+    V = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
+    keep = rng.random((Hkv, T)) < density
+    if density == 0.7:
+        keep[0, :1500] = True                                                 # long fully-kept prefix
+    words = np.zeros((Hkv, gv.mask_row_words(T, B)), dtype=np.uint32)
+    for r in range(B):
+        for h in range(Hkv):
+            w = o.pack_mask_bits(keep[h, cu[r]:cu[r + 1]])
+            off = gv.mask_word_offset(int(cu[r]), r)
+            words[h, off:off + len(w)] = w
+    p = gv.make_params(d_h=64, n_q_heads=Hkv, n_kv_heads=Hkv, d_k=d_k, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=0,
+                       seed=0)
+    geom = (B, T, max(lens))
+    ws = gv.alloc_workspace(p, *geom)
+    Kd, Vd = gv.bf16_from_bits(K), gv.bf16_from_bits(V)
+    budget = torch.empty(B, Hkv, dtype=torch.int32, device="cuda")
+    md = torch.from_numpy(words.view(np.int32)).cuda()
+    for rep in range(2):                                                      # second run: same flags reused
+        Kd.copy_(gv.bf16_from_bits(K)); Vd.copy_(gv.bf16_from_bits(V))
+        gv.gvote_compact(p, Kd, Vd, md, torch.from_numpy(cu).cuda(), geom, budget, ws)
+        assert gv.gvote_poll_status(ws) == 0
+        Kg, Vg, bg = gv.bits_from_bf16(Kd), gv.bits_from_bf16(Vd), budget.cpu().numpy()
+        for r in range(B):
+            a, b = int(cu[r]), int(cu[r + 1])
+            Kc, Vc = o.compact(K[:, a:b], V[:, a:b], keep[:, a:b])
+            for h in range(Hkv):
+                n = Kc[h].shape[0]
+                assert bg[r, h] == n
+                assert np.array_equal(Kg[h, a:a + n], Kc[h]) and np.array_equal(Vg[h, a:a + n], Vc[h])
+
+
+def test_compact_strided_heads(gv):
+    """K and V as views of a [T, Hkv, d_k] cache (token-major), not dense per head."""
+    rng = np.random.default_rng(13)
+    T, Hkv, d_k = 700, 2, 64
+    base = rng.integers(0, 65536, size=(2, T, Hkv, d_k)).astype(np.uint16)
+    keep = rng.random((Hkv, T)) < 0.3
+    words = np.stack([o.pack_mask_bits(keep[h]) for h in range(Hkv)])
+    words = np.concatenate([words, np.zeros((Hkv, gv.mask_row_words(T, 1) - words.shape[1]), np.uint32)], axis=1)
+    p = gv.make_params(d_h=64, n_q_heads=Hkv, n_kv_heads=Hkv, d_k=d_k, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=0,
+                       seed=0)
+    geom = (1, T, T)
+    ws = gv.alloc_workspace(p, *geom)
+    KV = gv.bf16_from_bits(base)
+    Kd, Vd = KV[0].permute(1, 0, 2), KV[1].permute(1, 0, 2)                   # [Hkv, T, d_k] strided
+    budget = torch.empty(1, Hkv, dtype=torch.int32, device="cuda")
+    gv.gvote_compact(p, Kd, Vd, torch.from_numpy(words.view(np.int32)).cuda(),
+                     torch.tensor([0, T], dtype=torch.int32, device="cuda"), geom, budget, ws)
+    out = gv.bits_from_bf16(KV)
+    for h in range(Hkv):
+        n = int(keep[h].sum())
+        assert np.array_equal(out[0, :n, h], base[0, keep[h], h]) and np.array_equal(out[1, :n, h], base[1, keep[h], h])
+
+
+# ----------------------------------------------------------------------------- whole pass
+def _run_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
+    p = gv.params_from_config(cfg, layer_id=layer_id, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget, b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
+            gv.bits_from_bf16(d["V"]))
+
+
+def _check_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
+    """End to end.  The GPU draws its own samples (fp32 fit and Box-Muller), so a few query values
+    land on the neighbouring bf16 step; masks are compared inside the score tolerance (2e-2) band
+    and budgets to 0.5 % of N.  Compaction is checked bit-exactly against the GPU's own mask."""
+    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li, sel_mode, layer_id)
+    kw = pu.oracle_kwargs(cfg, layer_id)
+    res, _, _ = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, sel_mode=sel_mode, **kw)
+    pf = kw["p_nuc"]
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        N = b - a
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N) for h in range(cfg.n_kv_heads)])
+        Kr = o.bf16_bits_to_f64(li.K[:, a:b])
+        pu.check_vote_against_oracle(res[r].Q, Kr, pf, sel_mode, False, gm, b_step[r], mass_band=2e-2, logit_band=2e-2)
+        assert np.all(np.abs(budget[r] - res[r].budget) <= max(2, 0.005 * N)), (budget[r], res[r].budget)
+        Kc, Vc = o.compact(li.K[:, a:b], li.V[:, a:b], gm)
+        for h in range(cfg.n_kv_heads):
+            n = int(gm[h].sum())
+            assert budget[r, h] == n
+            assert np.array_equal(Kg[h, a:a + n], Kc[h]) and np.array_equal(Vg[h, a:a + n], Vc[h])
+
+
+@pytest.mark.parametrize("idx", range(4))
+def test_compress_small(gv, idx):
+    cfg = _small_cfgs()[idx]
+    _check_compress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx % 2 == 1)))
+
+
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c1", "topp"), ("c3", "topk")])
+def test_compress_configs(gv, name, mode):
+    cfg = synth.make_config(name)
+    _check_compress(gv, cfg, synth.make_layer(cfg, 0), mode)
+
+
+def test_compress_is_deterministic(gv):
+    cfg = synth.make_config("c1")
+    li = synth.make_layer(cfg, 0)
+    a = _run_compress(gv, cfg, li)
+    b = _run_compress(gv, cfg, li)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
+def test_compress_full_size_c2_layer(gv):
+    """One layer of the 32K workload, in the launch configuration the benchmark times."""
+    cfg = synth.make_config("c2")
+    _check_compress(gv, cfg, synth.make_layer(cfg, 3), layer_id=3)
+
+
+def test_compress_host_variant_matches_device_variant(gv):
+    cfg = synth.make_config("c0")
+    li = synth.make_layer(cfg, 0)
+    mask_d, budget_d, b_step_d, Kd, Vd = _run_compress(gv, cfg, li)
+    p = gv.params_from_config(cfg)
+    h = torch.from_numpy(li.h).pin_memory()
+    W = gv.bf16_from_bits(li.W_q, "cpu", pin=True)
+    K = gv.bf16_from_bits(li.K, "cpu", pin=True).clone()
+    V = gv.bf16_from_bits(li.V, "cpu", pin=True).clone()
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, 1), dtype=torch.int32)
+    budget = torch.empty(1, cfg.n_kv_heads, dtype=torch.int32)
+    b_step = torch.empty(1, cfg.n_q_heads, dtype=torch.int32)
+    for _ in range(2):
+        K.copy_(gv.bf16_from_bits(li.K, "cpu")); V.copy_(gv.bf16_from_bits(li.V, "cpu"))
+        gv.gvote_compress_host(p, h, W, None, K, V, torch.from_numpy(li.cu_seqlens), mask, budget, b_step)
+        assert np.array_equal(mask.numpy(), mask_d) and np.array_equal(budget.numpy(), budget_d)
+        assert np.array_equal(gv.bits_from_bf16(K), Kd) and np.array_equal(gv.bits_from_bf16(V), Vd)
+    gv.gvote_host_arena_release()
