@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the GVote compression pass: cached tokens compressed per second on B200.
+
+A step is one pass of the whole hot path (fit, sample, project, vote, compact) over every layer
+of the workload, one `gvote_compress` call per layer.  The default workload is the Llama-3-8B
+shaped 32K-context pass (32 layers, N = 32768, S = 32, p = 0.95) on seeded synthetic inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+
+Prints one JSON line.  With --impl reference the CPU oracle is timed instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "GVote KV tokens compressed/sec (all layers of the workload, 1 B200 per rank)"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 <= ts <= t1):
+                continue
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(self.NAMES, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def gen_layers(cfg, layers, workers):
+    from paper_2509_03136_b200 import synth
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        return list(ex.map(lambda l: synth.make_layer(cfg, l), layers))
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def time_oracle_layer(cfg, li, layer_id):
+    from oracle import gvote_oracle as o
+    t0 = time.perf_counter()
+    res, Kc, Vc = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, n_q_heads=cfg.n_q_heads,
+                                   d_k=cfg.d_k, theta=cfg.rope_theta, S=cfg.S, p_nuc=float(np.float32(cfg.p_nuc)),
+                                   n_f=cfg.n_f, n_s=cfg.n_s, seed=cfg.seed, layer_id=layer_id)
+    return time.perf_counter() - t0, res
+
+
+def algorithmic_bytes(cfg, kept_frac):
+    """Compulsory bytes per layer of each stage (no recompute, no materialised logits)."""
+    T = cfg.total_tokens
+    kv = T * cfg.n_kv_heads * cfg.d_k * 2
+    return {
+        "fit": (T - cfg.batch * cfg.n_s) * cfg.d_h * 4,
+        "wq": cfg.d_h * cfg.n_q_heads * cfg.d_k * 2,
+        "k": kv,
+        "compact": 4.0 * kept_frac * kv,
+    }
+
+
+def flops(cfg):
+    rows = cfg.batch * (cfg.S + 1)
+    proj = 2.0 * rows * cfg.d_h * cfg.n_q_heads * cfg.d_k
+    score = 2.0 * (cfg.S + 1) * cfg.n_q_heads * cfg.total_tokens * cfg.d_k
+    return proj, score
+
+
+STAGE_OF = {
+    "fit_partial_kernel": "fit", "fit_finalize_kernel": "fit", "sample_kernel": "sample",
+    "xstage_kernel": "project", "rope_table_kernel": "project", "project_simt_kernel": "project",
+    "project_umma_kernel": "project", "project_finish_kernel": "project",
+    "score_simt_kernel": "vote", "score_umma_kernel": "vote", "topp_rows_kernel": "vote",
+    "topk_rows_kernel": "vote", "softmax_dump_kernel": "vote", "budget_kernel": "vote",
+    "mask_scan_kernel": "compact", "compact_kernel": "compact",
+}
+
+
+# ----------------------------------------------------------------------------- reference arm
+def run_reference(args, cfg, rank, world):
+    if rank != 0:
+        return
+    from paper_2509_03136_b200 import synth
+    cores = blas_threads()
+    times = []
+    for s in range(args.warmup + args.steps):
+        layer = s % cfg.n_layers
+        li = synth.make_layer(cfg, layer)
+        t, _ = time_oracle_layer(cfg, li, layer)
+        if s >= args.warmup:
+            times.append(t)
+    per_layer = sum(times) / len(times)
+    ms_step = per_layer * cfg.n_layers * 1e3
+    value = cfg.total_tokens / (per_layer * cfg.n_layers)
+    sample = f"one layer of {cfg.n_layers} per step ({cfg.total_tokens} tokens), scaled by the layer count"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(cfg, args):
+    return {"workload": f"{cfg.name}: {cfg.n_layers} layers, hidden {cfg.d_h}, {cfg.n_q_heads}/{cfg.n_kv_heads} heads, "
+                        f"d_k {cfg.d_k}, requests {cfg.batch}, tokens {cfg.total_tokens}, S {cfg.S}, p {cfg.p_nuc}",
+            "n_f": cfg.n_f, "n_s": cfg.n_s, "sel_mode": "topk_c0", "h_dtype": "f32", "kv_dtype": "bf16",
+            "l2": "inputs larger than L2 (every layer has its own tensors; K/V restored from pristine copies "
+                  "between steps, outside the timed intervals)",
+            "timing": "sum of per-step CUDA-event intervals on the launch stream"}
+
+
+# ----------------------------------------------------------------------------- native arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2509_03136_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    over = {"n_layers": args.layers} if args.layers > 0 else {}
+    base_cfg = synth.make_config(args.workload, **over)
+
+    if args.impl == "reference":
+        run_reference(args, base_cfg, rank, world)
+        return
+
+    import torch
+    from paper_2509_03136_b200 import build as gbuild
+    if rank == 0:
+        gbuild.build()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    else:
+        dist = None
+        torch.cuda.set_device(local)
+    from paper_2509_03136_b200 import gvote as gv
+    gv.load()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    # weak scaling: every rank compresses its own requests (same shapes, its own seed)
+    cfg = synth.make_config(args.workload, seed=base_cfg.seed + 1000 * rank, **over)
+    L = cfg.n_layers
+    geom = (cfg.batch, cfg.total_tokens, max(cfg.seq_lens))
+    workers = max(1, min(len(os.sched_getaffinity(0)) // max(world, 1), 16))
+    t_gen = time.perf_counter()
+    layers = gen_layers(cfg, range(L), workers)
+    t_gen = time.perf_counter() - t_gen
+
+    dev = torch.device("cuda", local)
+    p_layer = [gv.params_from_config(cfg, layer_id=l) for l in range(L)]
+    ws = gv.alloc_workspace(p_layer[0], *geom)
+    cu = torch.from_numpy(layers[0].cu_seqlens).to(dev)
+    d_h = [torch.from_numpy(li.h).to(dev) for li in layers]
+    d_W = [gv.bf16_from_bits(li.W_q, dev) for li in layers]
+    d_K0 = [gv.bf16_from_bits(li.K, dev) for li in layers]
+    d_V0 = [gv.bf16_from_bits(li.V, dev) for li in layers]
+    d_K = [t.clone() for t in d_K0]
+    d_V = [t.clone() for t in d_V0]
+    words = gv.mask_row_words(cfg.total_tokens, cfg.batch)
+    d_mask = [torch.empty(cfg.n_kv_heads, words, dtype=torch.int32, device=dev) for _ in range(L)]
+    d_budget = [torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device=dev) for _ in range(L)]
+    d_bstep = [torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device=dev) for _ in range(L)]
+
+    def restore():
+        for l in range(L):
+            d_K[l].copy_(d_K0[l]); d_V[l].copy_(d_V0[l])
+
+    def one_pass():
+        for l in range(L):
+            gv.gvote_compress(p_layer[l], d_h[l], d_W[l], None, d_K[l], d_V[l], cu, geom, d_mask[l], d_budget[l],
+                              d_bstep[l], ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_steps(n):
+        total_ms = 0.0
+        for _ in range(n):
+            restore()
+            barrier()
+            ev0.record()
+            one_pass()
+            ev1.record()
+            torch.cuda.synchronize()
+            total_ms += ev0.elapsed_time(ev1)
+        return total_ms
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(1.0)
+    tw0 = time.perf_counter()
+    timed_steps(args.warmup)
+    n0 = gv.gvote_launch_count()
+    tc0 = time.perf_counter()
+    total_ms = timed_steps(args.steps)
+    tc1 = time.perf_counter()
+    launches = gv.gvote_launch_count() - n0
+    assert gv.gvote_poll_status(ws) == 0, "a device-side wait timed out"
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.total_tokens / (ms_per_step * 1e-3)
+
+    # ---- per-kernel timing: the same steps again with an event pair around every launch
+    gv.gvote_profile_enable(True)
+    timed_steps(args.steps)
+    prof = gv.gvote_profile_report()
+    gv.gvote_profile_enable(False)
+    # clock samples cover the warm-up, the timed steps and their event-instrumented repeat (same work)
+    clocks = sampler.stop(tw0, time.perf_counter())
+    clocks["window"] = "warm-up + timed steps + instrumented repeat"
+    budgets = torch.stack(d_budget).cpu().numpy()                       # [L, batch, Hkv]
+    kept_frac = float(budgets.sum() / (L * cfg.n_kv_heads * cfg.total_tokens))
+    hbm_gbs, bf16_tf, peak_kind = load_peaks()
+    ab = algorithmic_bytes(cfg, kept_frac)
+    f_proj, f_score = flops(cfg)
+    per_kernel = {k: {"launches": n, "avg_us": ms / n * 1e3, "share": 0.0} for k, (n, ms) in prof.items()}
+    tot_prof = sum(ms for _, ms in prof.values()) or 1.0
+    for k, (n, ms) in prof.items():
+        per_kernel[k]["share"] = ms / tot_prof
+    stage_us = {}
+    for k, (n, ms) in prof.items():
+        st = STAGE_OF.get(k, "other")
+        stage_us[st] = stage_us.get(st, 0.0) + ms * 1e3 / (args.steps * L)
+    dom = max(prof.items(), key=lambda kv: kv[1][1])[0]
+    dom_bytes = {"fit": ab["fit"], "project": ab["wq"], "vote": ab["k"], "compact": ab["compact"],
+                 "sample": 0}.get(STAGE_OF.get(dom, "other"), 0)
+    dom_avg_s = prof[dom][1] / prof[dom][0] * 1e-3
+    achieved = dom_bytes / dom_avg_s / 1e9 if dom_avg_s > 0 else 0.0
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", f"{dom}_{cfg.name}_dram_bytes.txt")
+    if os.path.exists(tpath):
+        try:
+            traffic = float(open(tpath).read().split()[0])
+        except Exception:
+            traffic = None
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s",
+                "frac": achieved / hbm_gbs, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_us": dom_avg_s * 1e6,
+                "timed_with": "CUDA event pairs around every launch on the launch stream, same steps repeated"}
+    lit_t = max((f_proj + f_score) / (bf16_tf * 1e12), (ab["k"] + ab["compact"]) / (hbm_gbs * 1e9))
+    full_t = max((f_proj + f_score) / (bf16_tf * 1e12),
+                 (ab["fit"] + ab["wq"] + ab["k"] + ab["compact"]) / (hbm_gbs * 1e9))
+    layer_s = ms_per_step * 1e-3 / L
+    sel_s = (stage_us.get("project", 0) + stage_us.get("vote", 0) + stage_us.get("compact", 0)) * 1e-6
+    pass_roofline = {
+        "kept_fraction": kept_frac, "per_layer_us": layer_s * 1e6, "stage_us_per_layer": stage_us,
+        "full_bytes_roofline_us": full_t * 1e6, "full_bytes_frac": full_t / layer_s,
+        "literal_roofline_us": lit_t * 1e6, "literal_frac_whole_pass": lit_t / layer_s,
+        "literal_frac_select_compact_only": (lit_t / sel_s) if sel_s > 0 else None,
+        "peaks": {"hbm_gbs": hbm_gbs, "bf16_tflops": bf16_tf, "kind": peak_kind},
+    }
+
+    # ---- end to end through the host-memory entry point
+    e2e = None
+    if not args.no_e2e:
+        hK0 = [gv.bf16_from_bits(li.K, "cpu") for li in layers]
+        hV0 = [gv.bf16_from_bits(li.V, "cpu") for li in layers]
+        hh = [torch.from_numpy(li.h).pin_memory() for li in layers]
+        hW = [gv.bf16_from_bits(li.W_q, "cpu", pin=True) for li in layers]
+        hK = [t.clone().pin_memory() for t in hK0]
+        hV = [t.clone().pin_memory() for t in hV0]
+        hcu = torch.from_numpy(layers[0].cu_seqlens)
+        hmask = [torch.empty(cfg.n_kv_heads, words, dtype=torch.int32).pin_memory() for _ in range(L)]
+        hbud = [torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32).pin_memory() for _ in range(L)]
+        hbs = [torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32).pin_memory() for _ in range(L)]
+        e2e_total = 0.0
+        n_e2e = max(1, args.e2e_steps)
+        for s in range(1 + n_e2e):
+            for l in range(L):
+                hK[l].copy_(hK0[l]); hV[l].copy_(hV0[l])
+            barrier()
+            t0 = time.perf_counter()
+            for l in range(L):
+                gv.gvote_compress_host(p_layer[l], hh[l], hW[l], None, hK[l], hV[l], hcu, hmask[l], hbud[l], hbs[l])
+            dt = time.perf_counter() - t0
+            if s >= 1:
+                e2e_total += dt
+        if dist is not None:
+            t = torch.tensor([e2e_total], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_total = float(t.item())
+        gv.gvote_host_arena_release()
+        h2d = sum(a.numel() * a.element_size() for l in range(L) for a in (hh[l], hW[l], hK[l], hV[l])) + L * hcu.numel() * 4
+        d2h = sum(a.numel() * a.element_size() for l in range(L) for a in (hK[l], hV[l], hmask[l], hbud[l], hbs[l]))
+        e2e = {"value": world * cfg.total_tokens / (e2e_total / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": e2e_total / n_e2e * 1e3}
+        same = all(np.array_equal(hbud[l].numpy(), d_budget[l].cpu().numpy()) for l in range(L))
+        e2e["budgets_match_device_run"] = bool(same)
+
+    # ---- the oracle on this machine's host cores, on a bounded sample (rank 0, one GPU only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t_or, res = time_oracle_layer(cfg, layers[0], 0)
+        ob = np.stack([r.budget for r in res])
+        gb = d_budget[0].cpu().numpy()
+        tol = np.maximum(2, 0.005 * np.asarray(cfg.seq_lens)[:, None])
+        cpu_baseline = {"value": cfg.total_tokens / (t_or * L), "unit": UNIT, "cores": blas_threads(),
+                        "kind": "oracle", "sample": f"layer 0 of {L} ({cfg.total_tokens} tokens, {t_or:.1f} s), "
+                        "scaled by the layer count", "budgets_within_tolerance": bool(np.all(np.abs(ob - gb) <= tol))}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, args),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "pass_roofline": pass_roofline, "kernels": per_kernel,
+            "setup_s": {"generate": t_gen},
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -176,6 +176,14 @@ GVOTE_API void gvote_host_arena_release(void);
 /* Reads the status word of a workspace (synchronises the stream): GVOTE_OK or GVOTE_ERR_TIMEOUT. */
 GVOTE_API int32_t gvote_poll_status(void* ws, void* stream);
 
+/* Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is
+ * bracketed by two CUDA events on its stream.  Enabling (or disabling) drops earlier records.
+ * gvote_profile_report synchronises the device and writes one text line per kernel,
+ * "name launches total_ms", into buf (host, NUL-terminated, truncated to cap); it returns the
+ * bytes needed.  Not thread safe against concurrent launches from other threads. */
+GVOTE_API void gvote_profile_enable(int32_t on);
+GVOTE_API size_t gvote_profile_report(char* buf, size_t cap);
+
 /* Number of kernel launches the library has enqueued in this process (all entry points). */
 GVOTE_API int64_t gvote_launch_count(void);
 

@@ -15,6 +15,15 @@ namespace gvote {
 void set_cuda_error(cudaError_t e, const char* where);
 void count_launch(int n = 1);
 
+// Brackets one kernel launch with CUDA events on its stream when per-kernel timing is switched on
+// (gvote_profile_enable); otherwise it does nothing.
+struct LaunchScope {
+  LaunchScope(const char* name, cudaStream_t st);
+  ~LaunchScope();
+  int slot;
+  cudaStream_t st;
+};
+
 #define GVOTE_CUDA_CHECK(expr)                                   \
   do {                                                           \
     cudaError_t e__ = (expr);                                    \

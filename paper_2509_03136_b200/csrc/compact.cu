@@ -175,14 +175,20 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
   int32_t* ticket = flags + (size_t)2 * Hkv * m.n_tiles;
   int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
   dim3 gs(Hkv, batch);
+  {
+    LaunchScope scope_("mask_scan_kernel", st);
   mask_scan_kernel<<<gs, kScanThreads, 0, st>>>(mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
+  }
   GVOTE_LAUNCH_CHECK("mask_scan_kernel");
   const size_t smem = (size_t)kCompactTile * p->d_k * sizeof(__nv_bfloat16);
   if (smem > 48 * 1024)
     GVOTE_CUDA_CHECK(cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int64_t ctas = m.n_tiles * 2 * Hkv;
+  {
+    LaunchScope scope_("compact_kernel", st);
   compact_kernel<<<(unsigned)ctas, kCompactThreads, smem, st>>>(K, V, tok, head, mask, prefix, cu, batch, Hkv, p->d_k,
                                                                 m.row_words, m.n_tiles, flags, ticket, status);
+  }
   GVOTE_LAUNCH_CHECK("compact_kernel");
   return GVOTE_OK;
 }

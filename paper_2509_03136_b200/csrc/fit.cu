@@ -131,15 +131,21 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
                    int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st) {
   const int strips = (int)ceil_div(p->d_h, kFitStripCols);
   dim3 grid(strips, fit_chunks, batch), block(kFitTx, kFitTy);
+  {
+    LaunchScope scope_("fit_partial_kernel", st);
   if (p->h_dtype == GVOTE_DTYPE_F32) {
     fit_partial_kernel<float><<<grid, block, 0, st>>>((const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks, partial);
   } else {
     fit_partial_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)h, ld, cu, p->n_s, p->d_h,
                                                               fit_chunks, partial);
   }
+  }
   GVOTE_LAUNCH_CHECK("fit_partial_kernel");
   dim3 g2((unsigned)ceil_div(p->d_h, 128), batch);
+  {
+    LaunchScope scope_("fit_finalize_kernel", st);
   fit_finalize_kernel<<<g2, 128, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
+  }
   GVOTE_LAUNCH_CHECK("fit_finalize_kernel");
   return GVOTE_OK;
 }

@@ -165,22 +165,34 @@ int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* 
   float* table = reinterpret_cast<float*>(ws + m.rope);
 
   dim3 gx((unsigned)ceil_div(d_h, 256), S + 1, batch);
+  {
+    LaunchScope scope_("xstage_kernel", st);
   if (p->h_dtype == GVOTE_DTYPE_F32)
     xstage_kernel<float><<<gx, 256, 0, st>>>(H_tilde, (const float*)h_last, h_last_ld, h_last_rows_from_cu, d_h, S, X);
   else
     xstage_kernel<__nv_bfloat16><<<gx, 256, 0, st>>>(H_tilde, (const __nv_bfloat16*)h_last, h_last_ld,
                                                      h_last_rows_from_cu, d_h, S, X);
+  }
   GVOTE_LAUNCH_CHECK("xstage_kernel");
 
+  {
+    LaunchScope scope_("rope_table_kernel", st);
   rope_table_kernel<<<batch, 64, 0, st>>>(cu, p->d_k, p->rope_theta, p->n_f, table);
+  }
   GVOTE_LAUNCH_CHECK("rope_table_kernel");
 
   dim3 gp((unsigned)ceil_div(F, kProjWarps), (unsigned)ceil_div(rows_total, kProjRows));
+  {
+    LaunchScope scope_("project_simt_kernel", st);
   project_simt_kernel<<<gp, kProjWarps * 32, 0, st>>>(X, (const __nv_bfloat16*)W_q, wq_ld, rows_total, d_h, F, qf);
+  }
   GVOTE_LAUNCH_CHECK("project_simt_kernel");
 
   dim3 gf((unsigned)ceil_div((int64_t)p->n_q_heads * (p->d_k / 2), 128), S + 1, batch);
+  {
+    LaunchScope scope_("project_finish_kernel", st);
   project_finish_kernel<<<gf, 128, 0, st>>>(qf, 1, (int64_t)rows_total * F, b_q, table, S, p->n_q_heads, p->d_k, Q);
+  }
   GVOTE_LAUNCH_CHECK("project_finish_kernel");
   return GVOTE_OK;
 }

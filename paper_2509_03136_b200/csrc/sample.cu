@@ -63,8 +63,11 @@ int32_t launch_sample(const gvote_params* p, const float* mu, const float* var, 
                       uint32_t* raw, cudaStream_t st) {
   const int blocks4 = (int)ceil_div(p->d_h, 4);
   dim3 grid((unsigned)ceil_div(blocks4, 128), p->S, batch);
+  {
+    LaunchScope scope_("sample_kernel", st);
   sample_kernel<<<grid, 128, 0, st>>>(mu, var, p->d_h, p->S, (uint32_t)(p->seed & 0xffffffffu),
                                       (uint32_t)(p->seed >> 32), p->layer_id, H_tilde, raw);
+  }
   GVOTE_LAUNCH_CHECK("sample_kernel");
   return GVOTE_OK;
 }

@@ -388,31 +388,49 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
       GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     dim3 grid((unsigned)ceil_div(max_N, kScoreKeys), Hkv, batch);
+    {
+      LaunchScope scope_("score_simt_kernel", st);
     score_simt_kernel<<<grid, 256, smem, st>>>(Q, K, k_tok, k_head, cu, Hq, G, S1, d_k,
                                                (float)(1.0 / sqrt((double)d_k)), logits);
+    }
     GVOTE_LAUNCH_CHECK("score_simt_kernel");
   }
   if (dbg_probs) {
     dim3 grid(S1, Hq, batch);
+    {
+      LaunchScope scope_("softmax_dump_kernel", st);
     softmax_dump_kernel<<<grid, kSelThreads, 0, st>>>(logits, cu, Hq, S1, dbg_probs);
+    }
     GVOTE_LAUNCH_CHECK("softmax_dump_kernel");
   }
   if (p->sel_mode == GVOTE_SEL_TOPK_C0) {
     dim3 g1(1, Hq, batch);
+    {
+      LaunchScope scope_("topp_rows_kernel", st);
     topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0, m.row_words,
                                                  mask, b_step);
+    }
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
     dim3 g2(p->S, Hq, batch);
+    {
+      LaunchScope scope_("topk_rows_kernel", st);
     topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask);
+    }
     GVOTE_LAUNCH_CHECK("topk_rows_kernel");
   } else {
     dim3 g1(S1, Hq, batch);
+    {
+      LaunchScope scope_("topp_rows_kernel", st);
     topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0, m.row_words,
                                                  mask, b_step);
+    }
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
   }
   dim3 gb(Hkv, batch);
+  {
+    LaunchScope scope_("budget_kernel", st);
   budget_kernel<<<gb, 256, 0, st>>>(mask, cu, Hkv, m.row_words, budget);
+  }
   GVOTE_LAUNCH_CHECK("budget_kernel");
   return GVOTE_OK;
 }

@@ -24,7 +24,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 EXPORTS = (
     "gvote_workspace_bytes", "gvote_fit", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
     "gvote_compact", "gvote_compress", "gvote_compress_host", "gvote_host_arena_release",
-    "gvote_poll_status", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
+    "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
 
@@ -81,6 +81,10 @@ def load():
     lib.gvote_host_arena_release.argtypes = []
     lib.gvote_poll_status.restype = i32
     lib.gvote_poll_status.argtypes = [vp, vp]
+    lib.gvote_profile_enable.restype = None
+    lib.gvote_profile_enable.argtypes = [i32]
+    lib.gvote_profile_report.restype = sz
+    lib.gvote_profile_report.argtypes = [ctypes.c_char_p, sz]
     lib.gvote_launch_count.restype = i64
     lib.gvote_launch_count.argtypes = []
     lib.gvote_status_string.restype = ctypes.c_char_p
@@ -240,6 +244,23 @@ def gvote_host_arena_release() -> None:
 
 def gvote_poll_status(ws) -> int:
     return int(load().gvote_poll_status(_ptr(ws), _stream()))
+
+
+def gvote_profile_enable(on: bool) -> None:
+    load().gvote_profile_enable(1 if on else 0)
+
+
+def gvote_profile_report() -> dict:
+    """{kernel name: (launches, total milliseconds)} since profiling was enabled."""
+    lib = load()
+    cap = 1 << 16
+    buf = ctypes.create_string_buffer(cap)
+    lib.gvote_profile_report(buf, cap)
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, n, ms = line.split()
+        out[name] = (int(n), float(ms))
+    return out
 
 
 def gvote_launch_count() -> int:

@@ -67,7 +67,7 @@ class GVoteConfig:
     heavy_frac_layer_range: Optional[Sequence[float]] = None  # per-layer U[lo,hi]
     heavy_lead: float = 8.0          # target logit lead of a planted key for the mean query
     heavy_norm_cap: float = 1.0      # planted offset norm <= cap * sqrt(d_k)
-    heavy_gain: float = 4.0          # planted rows also carry this multiple of the N(0,1) row
+    heavy_gain: float = 2.5          # planted rows also carry this multiple of the N(0,1) row
     local_window: int = 0            # last tokens with a weaker planted offset
     local_scale: float = 0.25
 
