@@ -98,6 +98,7 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   m.q_bf16 = take((size_t)batch * S1 * F * sizeof(__nv_bfloat16));
   m.rope = take((size_t)batch * 4 * (p->d_k / 2) * sizeof(float));
   m.logits = take((size_t)p->n_q_heads * S1 * (size_t)total_tokens * sizeof(float));
+  m.keys16 = take(keys16_elems(p, batch, total_tokens) * sizeof(uint16_t));
   m.prefix = take((size_t)p->n_kv_heads * m.row_words * sizeof(int32_t));
   m.flags = take(((size_t)2 * p->n_kv_heads * m.n_tiles + 4) * sizeof(int32_t));
   m.total = off;
@@ -238,7 +239,7 @@ int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_strid
     PROPAGATE(launch_project(p, Ht, h, h_row_stride, cu_seqlens, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q,
                              st));
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, budget, b_step, nullptr, m, w, st));
+                        max_N, mask, nullptr, b_step, nullptr, m, w, st));   // budgets come from the scan below
   return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
                         total_tokens, max_N, budget, m, w, st);
 }

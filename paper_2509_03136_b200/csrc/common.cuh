@@ -65,6 +65,7 @@ struct WorkspaceMap {
   size_t q_bf16;        // bf16 [batch][Hq][S+1][d_k]
   size_t rope;          // float [batch][4][d_k/2]  (cos0, sin0, cbar, sbar)
   size_t logits;        // float [Hq*(S+1) * total_tokens], request-major
+  size_t keys16;        // uint16 [Hq*S * (padded tokens)]: 16-bit logit keys of the synthetic rows
   size_t prefix;        // int32 [Hkv][row_words]  exclusive popcount prefix per mask word
   size_t flags;         // int32 [2*Hkv*n_tiles + 4]  compaction "tile loaded" flags + ticket
   size_t total;
@@ -74,6 +75,7 @@ struct WorkspaceMap {
   int64_t row_words;    // mask words per head
 };
 
+size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens);
 WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
 // ---------------------------------------------------------------------------------- stage launchers
