@@ -75,6 +75,10 @@ struct WorkspaceMap {
   int64_t row_words;    // mask words per head
 };
 
+// Row tiling of the tensor-core score kernel: the (S+1)*G rows of a head group are split into
+// `row_chunks` chunks of RC rows (RC a multiple of 16, at most 240).
+struct ScoreGeometry { int RC; int row_chunks; };
+ScoreGeometry score_geometry(const gvote_params* p);
 size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens);
 WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 

@@ -9,15 +9,19 @@
 // One persistent CTA walks the key tiles x, x+X, x+2X, ... of one (request, KV head, row chunk):
 //   warp 0   : TMA producer - the group's query rows once, then a ring of key tiles
 //   warp 1   : allocates tensor memory, issues tcgen05.mma, commits to the ring and to the read-out
-//   warps 2-5: read-out - tcgen05.ld 32 rows at a time; thread = one key; scale; store
-// The read-out never writes the S x N logits as fp32 in the default mode: rows of the current
-// query (needed with full precision for the softmax mass) go out as fp32, rows of synthetic
-// queries go out as the upper 16 bits of an order-preserving image of the logit, which is all the
-// top-k search needs to bracket its threshold.
+//   warps 2-9: read-out - tcgen05.ld 32 rows at a time; thread = one key; two warps per lane quadrant
+//
+// Read-out, default mode.  The S x N logits never reach HBM as fp32.  Every logit is scaled and
+// turned into the upper 16 bits of an order-preserving image of its fp32 pattern (all the top-k
+// search needs to bracket its threshold), staged in shared memory as a [row][128 keys] tile and
+// written with one bulk copy per tile into a tile-blocked buffer keys16[head][tile][chunk][row][128].
+// Only the rows of the current query (one per query head) are also written as fp32, because the
+// softmax mass of line 2 needs them exactly.  In the all-fp32 mode (per-sample top-p, softmax dump)
+// every row is written as fp32 instead.
 //
 // Every wait on an mbarrier is bounded.  When one runs out the CTA raises a shared abort flag,
-// records GVOTE_ERR_TIMEOUT in the workspace status word, leaves its loops, frees its tensor
-// memory and returns.
+// records GVOTE_ERR_TIMEOUT in the workspace status word, leaves its loops, waits for its bulk
+// copies, frees its tensor memory and returns.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -25,8 +29,10 @@ namespace gvote {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kStages = 4;
-constexpr int kUmmaThreads = 192;
+constexpr int kStages = 3;
+constexpr int kEpiWarps = 8;
+constexpr int kUmmaThreads = 64 + 32 * kEpiWarps;
+constexpr int kMaxChunks32 = 8;   // RC <= 256
 
 struct ScoreSmemTail {
   uint64_t full[kStages];
@@ -36,6 +42,8 @@ struct ScoreSmemTail {
   uint64_t tmem_empty[2];
   uint32_t tmem_slot;
   volatile int abort_flag;
+  volatile int epi_go;                // read-out warps continue (decided by their leader, read after a barrier)
+  uint32_t real_mask[kMaxChunks32];   // per 32-row chunk: rows that belong to the current query
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -47,12 +55,17 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
+__device__ __forceinline__ uint32_t key16_of(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u ^ (uint32_t)(((int32_t)u >> 31) | (int32_t)0x80000000)) >> 16;
+}
+
 template <bool ALL_F32>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                   const int32_t* __restrict__ cu, int Hq, int G, int S1, int d_k, int RC, int row_chunks,
-                  int acc_cols, float scale, float* __restrict__ logits, uint16_t* __restrict__ keys16,
-                  int32_t* __restrict__ status) {
+                  int acc_cols, int n_out, float scale, int64_t n_tiles_total, float* __restrict__ logits,
+                  uint16_t* __restrict__ keys16, int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int r = blockIdx.z;
   const int kh = blockIdx.y / row_chunks, chunk = blockIdx.y % row_chunks;
@@ -67,29 +80,34 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t q_bytes = (uint32_t)kchunks * RC * 128;
   const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
+  const uint32_t out_bytes = (uint32_t)RC * kTileKeys * 2;
   uint8_t* Qs = base;
   uint8_t* Ks = base + q_bytes;
-  int64_t* row_meta = reinterpret_cast<int64_t*>(Ks + (size_t)kStages * stage_bytes);   // [RC]
-  ScoreSmemTail* tail = reinterpret_cast<ScoreSmemTail*>(row_meta + RC);
+  uint8_t* Os = Ks + (size_t)kStages * stage_bytes;                                        // [n_out][RC][128] u16
+  int64_t* row_meta = reinterpret_cast<int64_t*>(Os + (ALL_F32 ? 0 : (size_t)n_out * out_bytes));   // [RC] (all-fp32 mode)
+  ScoreSmemTail* tail = reinterpret_cast<ScoreSmemTail*>(row_meta + (ALL_F32 ? RC : 0));
 
-  // per-row output offsets (relative to the request's block): bit 0 = "fp32 row"; -1 = padding row
-  const int S = S1 - 1;
-  const int64_t pitch16 = (N + 7) & ~7;
-  for (int i = threadIdx.x; i < RC; i += blockDim.x) {
-    const int row = row0 + i;
-    int64_t meta = -1;
-    if (row < R) {
-      const int gl = row / S1, s = row % S1;
-      const int g = kh * G + gl;
-      if (ALL_F32 || s == 0) meta = ((((int64_t)g * S1 + s) * N) << 1) | 1;
-      else meta = (((int64_t)g * S + (s - 1)) * pitch16) << 1;
+  if (ALL_F32) {
+    // fp32 offset of every row (relative to the request's block); -1 = padding row
+    for (int i = threadIdx.x; i < RC; i += blockDim.x) {
+      const int row = row0 + i;
+      int64_t meta = -1;
+      if (row < R) meta = ((int64_t)(kh * G + row / S1) * S1 + row % S1) * N;
+      row_meta[i] = meta;
     }
-    row_meta[i] = meta;
+  }
+  if (threadIdx.x < kMaxChunks32) {
+    uint32_t m = 0;
+    for (int i = 0; i < 32; ++i) {
+      const int row = row0 + (int)threadIdx.x * 32 + i;
+      if ((int)threadIdx.x * 32 + i < RC && row < R && row % S1 == 0) m |= 1u << i;
+    }
+    tail->real_mask[threadIdx.x] = m;
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
     ptx::mbar_init(&tail->q_full, 1);
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&tail->tmem_full[a], 1); ptx::mbar_init(&tail->tmem_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&tail->tmem_full[a], 1); ptx::mbar_init(&tail->tmem_empty[a], kEpiWarps); }
     tail->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmK);
@@ -151,53 +169,91 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
     }
   } else {
-    // ------------------------------------------------------------------ read-out (4 warps = 128 lanes)
+    // ------------------------------------------------------------------ read-out (8 warps)
+    const int e = warp - 2;                      // 0..7
     const int q = warp & 3;                      // tensor-memory lane quadrant this warp may read
+    const int half = e >> 2;                     // which 32-row chunks this warp takes (even / odd)
+    const int m = q * 32 + lane;                 // key within the tile
+    const bool leader = (e == 0 && lane == 0);
     float* Lreq = logits + (int64_t)Hq * S1 * start;
-    uint16_t* Kreq = keys16 + (int64_t)Hq * S * (((int64_t)(start + 7) & ~7) + 16 * (int64_t)r);
+    const int64_t tile_base = ((int64_t)kh * n_tiles_total + tile_offset(start, r)) * row_chunks + chunk;
     int it = 0;
-    bool ok = true;
-    for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++it) {
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
       const int a = it & 1;
       const uint32_t aph = (uint32_t)(it >> 1) & 1u;
-      if (!wait_or_abort(&tail->tmem_full[a], aph, abort_flag)) { ok = false; break; }
+      const bool got = wait_or_abort(&tail->tmem_full[a], aph, abort_flag);
+      if (ALL_F32 && !got) break;               // no CTA-wide barriers in this mode: a warp may leave alone
       ptx::tc_fence_after_sync();
-      const int n = t * kTileKeys + q * 32 + lane;
+      const int n = t * kTileKeys + m;
       const bool valid = n < N;
       const uint32_t taddr = tmem_base + (uint32_t)(a * acc_cols) + ((uint32_t)(q * 32) << 16);
-      for (int c0 = 0; c0 < RC; c0 += 32) {
-        if (RC - c0 >= 32) {
-          uint32_t v[32];
+      uint8_t* obuf = Os + (size_t)(it % n_out) * out_bytes;
+      if (!ALL_F32) {
+        // All eight warps reach this barrier in every iteration, so the decision to stop is uniform.
+        // The staging buffer about to be overwritten must have been read by its bulk copy.
+        if (leader) {
+          if (n_out == 2) ptx::bulk_wait_read<1>(); else ptx::bulk_wait_read<0>();
+          tail->epi_go = *abort_flag ? 0 : 1;
+        }
+        ptx::named_barrier_sync(1, kEpiWarps * 32);
+        if (!tail->epi_go) break;
+      }
+      for (int c0 = half * 32; c0 < RC; c0 += 64) {
+        uint32_t v[32];
+        const bool wide = RC - c0 >= 32;
+        if (wide) {
           ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
-          ptx::tmem_wait_ld();
+        } else {
+          uint32_t w[16];
+          ptx::tmem_ld_32x16(taddr + (uint32_t)c0, w);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { v[i] = w[i]; v[16 + i] = 0; }
+        }
+        ptx::tmem_wait_ld();
+        const int nrows = wide ? 32 : 16;
+        if (ALL_F32) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const int64_t meta = row_meta[c0 + i];
-            if (meta >= 0 && valid) {
-              const float x = __uint_as_float(v[i]) * scale;
-              if (meta & 1) Lreq[(meta >> 1) + n] = x;
-              else Kreq[(meta >> 1) + n] = (uint16_t)(ordered_key(x) >> 16);
+            if (i < nrows) {
+              const int64_t meta = row_meta[c0 + i];
+              if (meta >= 0 && valid) Lreq[meta + n] = __uint_as_float(v[i]) * scale;
             }
           }
         } else {
-          uint32_t v[16];
-          ptx::tmem_ld_32x16(taddr + (uint32_t)c0, v);
-          ptx::tmem_wait_ld();
+          uint8_t* dst = obuf + (size_t)c0 * (kTileKeys * 2) + (size_t)m * 2;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int64_t meta = row_meta[c0 + i];
-            if (meta >= 0 && valid) {
-              const float x = __uint_as_float(v[i]) * scale;
-              if (meta & 1) Lreq[(meta >> 1) + n] = x;
-              else Kreq[(meta >> 1) + n] = (uint16_t)(ordered_key(x) >> 16);
+          for (int i = 0; i < 32; ++i) {
+            if (i < nrows)
+              *reinterpret_cast<uint16_t*>(dst + i * (kTileKeys * 2)) =
+                  (uint16_t)key16_of(__uint_as_float(v[i]) * scale);
+          }
+          const uint32_t rm = tail->real_mask[c0 >> 5];
+          if (rm != 0 && valid) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              if (rm & (1u << i)) {
+                const int row = row0 + c0 + i;     // s == 0 here
+                Lreq[((int64_t)(kh * G + row / S1) * S1) * N + n] = __uint_as_float(v[i]) * scale;
+              }
             }
           }
         }
       }
+      // accumulator drained: hand it back to the MMA warp
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&tail->tmem_empty[a]);
+      if (!ALL_F32) {
+        ptx::fence_proxy_async();                // staged tile visible to the bulk-copy engine
+        ptx::named_barrier_sync(2, kEpiWarps * 32);
+        if (leader) {
+          uint16_t* gdst = keys16 + ((tile_base + (int64_t)t * row_chunks) * RC) * kTileKeys;
+          ptx::bulk_store(gdst, obuf, out_bytes);
+          ptx::bulk_commit();
+        }
+      }
     }
+    if (!ALL_F32 && leader) ptx::bulk_wait_all<0>();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -220,8 +276,20 @@ bool score_umma_supported(const gvote_params* p) {
   return p->d_k % 64 == 0 && p->d_k <= 256;
 }
 
+ScoreGeometry score_geometry(const gvote_params* p) {
+  ScoreGeometry g;
+  const int R = (p->n_q_heads / p->n_kv_heads) * (p->S + 1);
+  g.row_chunks = (R + 239) / 240;
+  g.RC = (((R + g.row_chunks - 1) / g.row_chunks) + 15) & ~15;
+  if (g.RC < 16) g.RC = 16;
+  return g;
+}
+
 size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens) {
-  return (size_t)p->n_q_heads * p->S * (size_t)(((total_tokens + 7) & ~(int64_t)7) + 16 * (int64_t)batch);
+  if (!score_umma_supported(p)) return 0;
+  const ScoreGeometry g = score_geometry(p);
+  const int64_t n_tiles = (total_tokens >> 7) + batch;
+  return (size_t)p->n_kv_heads * n_tiles * g.row_chunks * g.RC * kTileKeys;
 }
 
 // Returns GVOTE_OK, or GVOTE_ERR_UNSUPPORTED_SHAPE when the tensor maps cannot describe the
@@ -230,11 +298,8 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                           bool all_f32, float* logits, uint16_t* keys16, int32_t* status, cudaStream_t st) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
-  const int R = G * S1;
-  const int row_chunks = (R + 239) / 240;
-  int RC = (R + row_chunks - 1) / row_chunks;
-  RC = (RC + 15) & ~15;
-  if (RC < 16) RC = 16;
+  const ScoreGeometry geo = score_geometry(p);
+  const int RC = geo.RC, row_chunks = geo.row_chunks;
   int acc_cols = 32;
   while (acc_cols < RC) acc_cols <<= 1;
 
@@ -252,8 +317,12 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
     if (!encode_tensor_map_bf16(&tmQ, Q, 2, dims, strides, box)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   }
   const int kchunks = d_k / 64;
-  const size_t smem = 1024 + (size_t)kchunks * RC * 128 + (size_t)kStages * kchunks * kTileKeys * 128 +
-                      (size_t)RC * sizeof(int64_t) + sizeof(ScoreSmemTail) + 64;
+  const size_t fixed = 1024 + (size_t)kchunks * RC * 128 + (size_t)kStages * kchunks * kTileKeys * 128 +
+                       sizeof(ScoreSmemTail) + 64;
+  const size_t out_bytes = (size_t)RC * kTileKeys * 2;
+  int n_out = 2;
+  size_t smem = fixed + (all_f32 ? (size_t)RC * sizeof(int64_t) : n_out * out_bytes);
+  if (!all_f32 && smem > 227 * 1024) { n_out = 1; smem = fixed + out_bytes; }
   if (smem > 227 * 1024) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   const int64_t max_tiles = ceil_div(max_N, kTileKeys);
   // one CTA per SM when the batch is uniform; a ragged batch gets four times as many, shorter
@@ -264,12 +333,13 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
   if (X < 1) X = 1;
   dim3 grid((unsigned)X, (unsigned)(Hkv * row_chunks), (unsigned)batch);
   const float scale = (float)(1.0 / sqrt((double)d_k));
+  const int64_t n_tiles_total = (total_tokens >> 7) + batch;
   auto kern = all_f32 ? score_umma_kernel<true> : score_umma_kernel<false>;
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_umma_kernel", st);
-    kern<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, S1, d_k, RC, row_chunks, acc_cols, scale, logits,
-                                           keys16, status);
+    kern<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, S1, d_k, RC, row_chunks, acc_cols, n_out, scale,
+                                           n_tiles_total, logits, keys16, status);
   }
   GVOTE_LAUNCH_CHECK("score_umma_kernel");
   return GVOTE_OK;

@@ -330,225 +330,6 @@ topk_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
   emit_row(L, N, t, ties, eq_cnt, mrow, sh);
 }
 
-// ---------------------------------------------------------------------------------- top-k on 16-bit keys
-// One CTA per synthetic row.  The row holds the upper 16 bits of the order-preserving image of each
-// logit (written by the tensor-core score kernel).  Two 8-bit histogram passes find the 16-bit
-// value T that contains the k-th largest logit; keys above T are selected outright.  Keys equal
-// to T ("candidates", a few dozen for typical rows) share 16 leading bits, so their exact order
-// is settled by recomputing their logits in fp32 from Q and K and ranking them (value
-// descending, index ascending).  Rows up to `smem_row_elems` keys are held in shared memory, so
-// the row is read from global memory once; longer rows are streamed three times.
-constexpr int kCandCap = 1024;
-
-struct Sel16Shared {
-  uint32_t hist[256];
-  float qf[512];
-  int cand_idx[kCandCap];
-  float cand_val[kCandCap];
-  uint32_t red32[kSelThreads / 32];
-  int bin;
-  uint32_t above;
-  uint32_t ncand;
-};
-
-// Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need).
-__device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    uint32_t c = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) c += sh.hist[lane * 8 + i];
-    uint32_t cs = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_down_sync(0xffffffffu, cs, o);
-      if (lane + o < 32) cs += t;
-    }
-    const uint32_t excl = cs - c;
-    if (lane == 0) { sh.bin = 0; sh.above = 0; }
-    __syncwarp();
-    if (excl < need && excl + c >= need) {
-      uint32_t a = excl;
-      int b = lane * 8 + 7;
-      for (; b > lane * 8; --b) {
-        if (a + sh.hist[b] >= need) break;
-        a += sh.hist[b];
-      }
-      sh.bin = b;
-      sh.above = a;
-    }
-  }
-  __syncthreads();
-}
-
-struct DotCtx {
-  const float* qf;
-  const __nv_bfloat16* krows;   // K + head offset + request start
-  int64_t k_tok;
-  int d_k;
-  float scale;
-  __device__ __forceinline__ float operator()(int n) const {
-    const uint4* kp = reinterpret_cast<const uint4*>(krows + (int64_t)n * k_tok);
-    float acc = 0.f;
-    for (int c = 0; c < d_k / 8; ++c) {
-      const uint4 v = __ldg(kp + c);
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 f = __bfloat1622float2(h[j]);
-        acc = fmaf(qf[c * 8 + 2 * j], f.x, acc);
-        acc = fmaf(qf[c * 8 + 2 * j + 1], f.y, acc);
-      }
-    }
-    return acc * scale;
-  }
-};
-
-__global__ void __launch_bounds__(kSelThreads)
-topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __restrict__ Q,
-                   const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
-                   const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, float scale,
-                   const int32_t* __restrict__ b_step, int64_t row_words, uint32_t* __restrict__ mask,
-                   int smem_row_elems) {
-  extern __shared__ __align__(16) uint16_t row_sm[];
-  __shared__ Sel16Shared sh;
-  const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
-  const int start = cu[r], N = cu[r + 1] - start;
-  if (N <= 0) return;
-  int k = b_step[r * Hq + g];
-  if (k <= 0) return;
-  if (k > N) k = N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int64_t pitch = (N + 7) & ~7;
-  const uint16_t* rowg = keys16 + (int64_t)Hq * S * ((((int64_t)start + 7) & ~7) + 16 * (int64_t)r) +
-                         ((int64_t)g * S + s) * pitch;
-  const bool fits = N <= smem_row_elems;
-  const uint16_t* rowp = fits ? row_sm : rowg;
-  uint32_t* mrow = mask + (int64_t)(g / G) * row_words + mask_word_offset(start, r);
-
-  // the row's query (for the exact recomputation), and pass A: load + histogram of the high byte
-  {
-    const __nv_bfloat16* qrow = Q + (((int64_t)r * Hq + g) * (S + 1) + (s + 1)) * d_k;
-    for (int i = tid; i < d_k; i += kSelThreads) sh.qf[i] = __bfloat162float(qrow[i]);
-    sh.hist[tid] = 0;
-    if (tid == 0) sh.ncand = 0;
-  }
-  __syncthreads();
-  for (int64_t v8 = tid; v8 < pitch / 8; v8 += kSelThreads) {
-    const uint4 v = *reinterpret_cast<const uint4*>(rowg + v8 * 8);
-    if (fits) *reinterpret_cast<uint4*>(row_sm + v8 * 8) = v;
-    const uint16_t* e = reinterpret_cast<const uint16_t*>(&v);
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (v8 * 8 + j < N) atomicAdd(&sh.hist[e[j] >> 8], 1u);
-  }
-  __syncthreads();
-  find_bin256(sh, (uint32_t)k);
-  const uint32_t b_hi = (uint32_t)sh.bin;
-  uint32_t above = sh.above;
-  __syncthreads();
-  sh.hist[tid] = 0;
-  __syncthreads();
-  // pass B: low byte among keys whose high byte is b_hi
-  for (int n = tid; n < N; n += kSelThreads) {
-    const uint32_t key = rowp[n];
-    if ((key >> 8) == b_hi) atomicAdd(&sh.hist[key & 255u], 1u);
-  }
-  __syncthreads();
-  find_bin256(sh, (uint32_t)k - above);
-  const uint32_t T = (b_hi << 8) | (uint32_t)sh.bin;
-  above += sh.above;
-  const uint32_t eq = sh.hist[sh.bin];
-  const uint32_t ties = (uint32_t)k - above;        // 1 <= ties <= eq
-  __syncthreads();
-
-  // pass C: select keys above T; keep or collect the candidates
-  const bool all_ties = ties >= eq;
-  for (int base = 0; base < N; base += kSelThreads) {
-    const int n = base + tid;
-    uint32_t key = 0;
-    const bool valid = n < N;
-    if (valid) key = rowp[n];
-    bool sel = valid && key > T;
-    const bool cand = valid && key == T;
-    if (all_ties) sel |= cand;
-    else if (cand) {
-      const uint32_t slot = atomicAdd(&sh.ncand, 1u);
-      if (slot < (uint32_t)kCandCap) sh.cand_idx[slot] = n;
-    }
-    const uint32_t bal = __ballot_sync(0xffffffffu, sel);
-    if (lane == 0 && bal) atomicOr(&mrow[n >> 5], bal);
-  }
-  if (all_ties) return;
-  __syncthreads();
-
-  DotCtx dot{sh.qf, K + (int64_t)(g / G) * k_head + (int64_t)start * k_tok, k_tok, d_k, scale};
-  if (eq <= (uint32_t)kCandCap) {
-    // rank the candidates by (exact logit descending, index ascending) and keep the first `ties`
-    for (int i = tid; i < (int)eq; i += kSelThreads) sh.cand_val[i] = dot(sh.cand_idx[i]);
-    __syncthreads();
-    for (int i = tid; i < (int)eq; i += kSelThreads) {
-      const float v = sh.cand_val[i];
-      const int n = sh.cand_idx[i];
-      uint32_t rank = 0;
-      for (int u = 0; u < (int)eq; ++u) {
-        const float vu = sh.cand_val[u];
-        rank += (vu > v || (vu == v && sh.cand_idx[u] < n)) ? 1u : 0u;
-      }
-      if (rank < ties) atomicOr(&mrow[n >> 5], 1u << (n & 31));
-    }
-    return;
-  }
-
-  // more candidates than the list holds (many equal logits): radix search over the recomputed
-  // 32-bit images of the candidates, four 8-bit passes, then an ordered emission
-  uint32_t prefix = 0, known = 0, acc = 0, eq2 = 0;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    sh.hist[tid] = 0;
-    __syncthreads();
-    for (int n = tid; n < N; n += kSelThreads) {
-      if (rowp[n] == T) {
-        const uint32_t key = ordered_key(dot(n));
-        if ((key & known) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
-      }
-    }
-    __syncthreads();
-    find_bin256(sh, ties - acc);
-    acc += sh.above;
-    prefix |= (uint32_t)sh.bin << shift;
-    known |= 255u << shift;
-    if (pass == 3) eq2 = sh.hist[sh.bin];
-    __syncthreads();
-  }
-  const uint32_t ties2 = ties - acc;
-  uint32_t taken = 0;
-  for (int base = 0; base < N; base += kSelThreads) {
-    const int n = base + tid;
-    const bool member = n < N && rowp[n] == T;
-    const uint32_t key = member ? ordered_key(dot(n)) : 0u;
-    bool sel = member && key > prefix;
-    const bool tie = member && key == prefix;
-    if (ties2 >= eq2) {
-      sel |= tie;
-    } else {
-      const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-      if (lane == 0) sh.red32[warp] = __popc(tb);
-      __syncthreads();
-      uint32_t before = taken, total = 0;
-      for (int w = 0; w < kSelThreads / 32; ++w) {
-        if (w < warp) before += sh.red32[w];
-        total += sh.red32[w];
-      }
-      sel |= tie && (before + __popc(tb & ((1u << lane) - 1u))) < ties2;
-      taken += total;
-      __syncthreads();
-    }
-    const uint32_t bal = __ballot_sync(0xffffffffu, sel);
-    if (lane == 0 && bal) atomicOr(&mrow[n >> 5], bal);
-  }
-}
-
 // ---------------------------------------------------------------------------------- softmax dump
 __global__ void __launch_bounds__(kSelThreads)
 softmax_dump_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int S1,
@@ -593,6 +374,9 @@ budget_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu,
 }  // namespace
 
 bool score_umma_supported(const gvote_params* p);
+int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_bfloat16* Q, const __nv_bfloat16* K,
+                      int64_t k_tok, int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens,
+                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, cudaStream_t st);
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                           bool all_f32, float* logits, uint16_t* keys16, int32_t* status, cudaStream_t st);
@@ -649,19 +433,9 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
     dim3 g2(p->S, Hq, batch);
     if (tensor_path && !all_f32) {
-      // rows up to 96K keys stay resident in shared memory (192 KB); longer rows are streamed
-      int row_elems = (int)((max_N + 7) & ~(int64_t)7);
-      if (row_elems > 96 * 1024) row_elems = 0;
-      const size_t smem = (size_t)row_elems * sizeof(uint16_t);
-      if (smem > 16 * 1024)
-        GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topk16_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)smem));
-      {
-        LaunchScope scope_("topk16_rows_kernel", st);
-        topk16_rows_kernel<<<g2, kSelThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, d_k, scale,
-                                                          b_step, m.row_words, mask, row_elems);
-      }
-      GVOTE_LAUNCH_CHECK("topk16_rows_kernel");
+      const int32_t rc = launch_topk16(p, keys16, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, b_step,
+                                       m.row_words, mask, st);
+      if (rc != GVOTE_OK) return rc;
     } else {
       {
         LaunchScope scope_("topk_rows_kernel", st);
