@@ -116,13 +116,16 @@ GVOTE_API int32_t gvote_sample(const gvote_params* p, const float* mu, const flo
 /* Algorithm 1 lines 1 (Q0), 6 and 7.  X = [h_last[r]; H_tilde[r]] is rounded to bf16, multiplied
  * by W_q (fp32 accumulation), b_q added when given ([n_q_heads*d_k] float), then rotated: row 0
  * exactly at position N_r-1, rows 1..S with the mean cos/sin of positions N_r..N_r+n_f-1.
- * Q: [batch, n_q_heads, S+1, d_k] bf16.  h_last: [batch, d_h] of p->h_dtype. */
+ * Q: [batch, n_kv_heads, G*(S+1), d_k] bf16 with G = n_q_heads / n_kv_heads; the rows of a KV head
+ * are ordered for the score contraction: first the S synthetic rows of each of its G query heads
+ * (row gl*S + s), then the G current-query rows (row G*S + gl).  h_last: [batch, d_h] of p->h_dtype. */
 GVOTE_API int32_t gvote_project(const gvote_params* p, const float* H_tilde, const void* h_last,
                       const void* W_q, int64_t wq_ld, const float* b_q_or_null,
                       const int32_t* cu_seqlens, int32_t batch,
                       void* Q, void* ws, size_t ws_bytes, void* stream);
 
-/* Algorithm 1 lines 1-3 and 8-10, given the rotated queries.  Per query head g: logits of its
+/* Algorithm 1 lines 1-3 and 8-10, given the rotated queries (layout as written by gvote_project).
+ * Per query head g: logits of its
  * S+1 rows against the N_r keys of KV head g div G, scaled by 1/sqrt(d_k); row 0 -> softmax ->
  * top-p -> b_step[r][g] = |C0|; rows 1..S -> top-k(b_step) on logits (or top-p on their softmax
  * in GVOTE_SEL_TOPP); mask[h] = OR over the rows of the head's group; budget[r][h] = popcount.

@@ -101,28 +101,42 @@ fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restric
   }
 }
 
-// Chan et al. pairwise update over the chunks of a request, in fp64; one thread per channel.
-__global__ void fit_finalize_kernel(const float2* __restrict__ partial, const int32_t* __restrict__ cu, int n_s,
-                                    int d_h, int chunks, float* __restrict__ mu, float* __restrict__ var) {
+// Chan et al. pairwise update over the chunks of a request, in fp64.  A CTA covers 32 channels;
+// eight row lanes each fold every eighth chunk, then lane 0 folds the eight partial results.
+struct Moments { double n, mean, m2; };
+__device__ __forceinline__ void chan_merge(Moments& a, double nc, double mean_c, double m2_c) {
+  if (nc <= 0.0) return;
+  const double tot = a.n + nc;
+  const double delta = mean_c - a.mean;
+  a.mean += delta * nc / tot;
+  a.m2 += m2_c + delta * delta * a.n * nc / tot;
+  a.n = tot;
+}
+
+__global__ void __launch_bounds__(256)
+fit_finalize_kernel(const float2* __restrict__ partial, const int32_t* __restrict__ cu, int n_s, int d_h, int chunks,
+                    float* __restrict__ mu, float* __restrict__ var) {
+  __shared__ Moments sm[8][32];
   const int r = blockIdx.y;
-  const int col = blockIdx.x * blockDim.x + threadIdx.x;
-  if (col >= d_h) return;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int col = blockIdx.x * 32 + tx;
   const int first = cu[r] + n_s, last = cu[r + 1];
-  double n = 0.0, mean = 0.0, m2 = 0.0;
-  for (int c = 0; c < chunks; ++c) {
-    int a, b;
-    chunk_rows(first, last, chunks, c, a, b);
-    const double nc = (double)(b - a);
-    if (nc <= 0.0) continue;
-    const float2 pc = partial[((int64_t)(r * chunks + c)) * d_h + col];
-    const double delta = (double)pc.x - mean;
-    const double tot = n + nc;
-    mean += delta * nc / tot;
-    m2 += (double)pc.y + delta * delta * n * nc / tot;
-    n = tot;
+  Moments acc{0.0, 0.0, 0.0};
+  if (col < d_h) {
+    for (int c = ty; c < chunks; c += 8) {
+      int a, b;
+      chunk_rows(first, last, chunks, c, a, b);
+      const float2 pc = partial[((int64_t)(r * chunks + c)) * d_h + col];
+      chan_merge(acc, (double)(b - a), (double)pc.x, (double)pc.y);
+    }
   }
-  mu[(int64_t)r * d_h + col] = (float)mean;
-  var[(int64_t)r * d_h + col] = (float)(m2 / (n - 1.0));   // NaN/inf when fewer than 2 rows
+  sm[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && col < d_h) {
+    for (int j = 1; j < 8; ++j) chan_merge(acc, sm[j][tx].n, sm[j][tx].mean, sm[j][tx].m2);
+    mu[(int64_t)r * d_h + col] = (float)acc.mean;
+    var[(int64_t)r * d_h + col] = (float)(acc.m2 / (acc.n - 1.0));   // NaN/inf when fewer than 2 rows
+  }
 }
 
 }  // namespace
@@ -141,10 +155,10 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
   }
   }
   GVOTE_LAUNCH_CHECK("fit_partial_kernel");
-  dim3 g2((unsigned)ceil_div(p->d_h, 128), batch);
+  dim3 g2((unsigned)ceil_div(p->d_h, 32), batch);
   {
     LaunchScope scope_("fit_finalize_kernel", st);
-  fit_finalize_kernel<<<g2, 128, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
+  fit_finalize_kernel<<<g2, 256, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
   }
   GVOTE_LAUNCH_CHECK("fit_finalize_kernel");
   return GVOTE_OK;

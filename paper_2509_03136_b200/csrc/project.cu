@@ -123,10 +123,11 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __
 }
 
 // ---------------------------------------------------------------------------------- finish
-// Sum the split-K partials, add the bias, rotate, round to bf16: Q[r][g][row][d_k].
+// Sum the split-K partials, add the bias, rotate, round to bf16.  Output rows are grouped per KV
+// head: first the S synthetic rows of each of its G query heads, then the G current-query rows.
 __global__ void project_finish_kernel(const float* __restrict__ qf, int splits, int64_t split_stride,
                                       const float* __restrict__ bias, const float* __restrict__ table, int S,
-                                      int Hq, int d_k, __nv_bfloat16* __restrict__ Q) {
+                                      int Hq, int G, int d_k, __nv_bfloat16* __restrict__ Q) {
   const int r = blockIdx.z, row = blockIdx.y;
   const int half = d_k / 2;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;   // over Hq * half
@@ -147,7 +148,9 @@ __global__ void project_finish_kernel(const float* __restrict__ qf, int splits, 
   const float c = t[j], s = t[half + j];
   const float y1 = x1 * c - x2 * s;
   const float y2 = x2 * c + x1 * s;
-  __nv_bfloat16* dst = Q + (((int64_t)r * Hq + g) * (S + 1) + row) * d_k;
+  const int kh = g / G, gl = g % G;
+  const int grow = (row == 0) ? (G * S + gl) : (gl * S + row - 1);
+  __nv_bfloat16* dst = Q + (((int64_t)r * (Hq / G) + kh) * (G * (S + 1)) + grow) * d_k;
   dst[j] = __float2bfloat16_rn(y1);
   dst[half + j] = __float2bfloat16_rn(y2);
 }
@@ -191,7 +194,8 @@ int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* 
   dim3 gf((unsigned)ceil_div((int64_t)p->n_q_heads * (p->d_k / 2), 128), S + 1, batch);
   {
     LaunchScope scope_("project_finish_kernel", st);
-  project_finish_kernel<<<gf, 128, 0, st>>>(qf, 1, (int64_t)rows_total * F, b_q, table, S, p->n_q_heads, p->d_k, Q);
+  project_finish_kernel<<<gf, 128, 0, st>>>(qf, 1, (int64_t)rows_total * F, b_q, table, S, p->n_q_heads,
+                                            p->n_q_heads / p->n_kv_heads, p->d_k, Q);
   }
   GVOTE_LAUNCH_CHECK("project_finish_kernel");
   return GVOTE_OK;

@@ -55,9 +55,47 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
-__device__ __forceinline__ uint32_t key16_of(float x) {
-  const uint32_t u = __float_as_uint(x);
-  return (u ^ (uint32_t)(((int32_t)u >> 31) | (int32_t)0x80000000)) >> 16;
+
+// Two fp32 logits -> two 16-bit keys: round to bf16 (monotone), then flip so that unsigned order
+// equals numeric order: negative values get all bits inverted, others get the sign bit set.
+__device__ __forceinline__ uint32_t key16x2_of(float lo, float hi) {
+  uint32_t p;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p) : "f"(hi), "f"(lo));
+  const uint32_t neg = (p >> 15) & 0x00010001u;          // 1 per negative half
+  return p ^ (neg * 0x7fffu + 0x80008000u);              // 0xffff for negative halves, 0x8000 otherwise
+}
+
+// Read-out of NR accumulator columns (query rows c0 .. c0+NR-1) held by this thread for key n.
+template <bool ALL_F32, int NR>
+__device__ __forceinline__ void readout_chunk(const uint32_t (&v)[NR], int c0, uint32_t real_mask,
+                                              const int64_t* row_meta, uint8_t* obuf, int m, int n, bool valid,
+                                              float scale, float* Lreq, int N, int S1, int g0, int real_row0) {
+  if (ALL_F32) {
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+      const int64_t meta = row_meta[c0 + i];
+      if (meta >= 0 && valid) Lreq[meta + n] = __uint_as_float(v[i]) * scale;
+    }
+  } else {
+    // keys need the order of the logits only, so the positive scale is not applied to them
+    uint8_t* dst = obuf + (size_t)c0 * (kTileKeys * 2) + (size_t)m * 2;
+#pragma unroll
+    for (int i = 0; i < NR; i += 2) {
+      const uint32_t kk = key16x2_of(__uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+      *reinterpret_cast<uint16_t*>(dst + i * (kTileKeys * 2)) = (uint16_t)kk;
+      *reinterpret_cast<uint16_t*>(dst + (i + 1) * (kTileKeys * 2)) = (uint16_t)(kk >> 16);
+    }
+    if (real_mask != 0 && valid) {
+      // rows of the current query (they follow the synthetic rows of the group): exact fp32 logits
+#pragma unroll
+      for (int i = 0; i < NR; ++i) {
+        if (real_mask & (1u << i)) {
+          const int g = g0 + (real_row0 + c0 + i);
+          Lreq[((int64_t)g * S1) * N + n] = __uint_as_float(v[i]) * scale;
+        }
+      }
+    }
+  }
 }
 
 template <bool ALL_F32>
@@ -92,7 +130,11 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     for (int i = threadIdx.x; i < RC; i += blockDim.x) {
       const int row = row0 + i;
       int64_t meta = -1;
-      if (row < R) meta = ((int64_t)(kh * G + row / S1) * S1 + row % S1) * N;
+      if (row < R) {
+        const int S = S1 - 1;
+        const int lrow = (row < G * S) ? (kh * G + row / S) * S1 + row % S + 1 : (kh * G + row - G * S) * S1;
+        meta = (int64_t)lrow * N;
+      }
       row_meta[i] = meta;
     }
   }
@@ -100,7 +142,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     uint32_t m = 0;
     for (int i = 0; i < 32; ++i) {
       const int row = row0 + (int)threadIdx.x * 32 + i;
-      if ((int)threadIdx.x * 32 + i < RC && row < R && row % S1 == 0) m |= 1u << i;
+      if ((int)threadIdx.x * 32 + i < RC && row < R && row >= G * (S1 - 1)) m |= 1u << i;
     }
     tail->real_mask[threadIdx.x] = m;
   }
@@ -126,7 +168,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && blockIdx.x < tiles) {
-      const int q_row = (r * Hq + kh * G) * S1 + row0;
+      const int q_row = (r * (Hq / G) + kh) * R + row0;   // the group's rows: synthetic first, then real
       ptx::mbar_arrive_expect_tx(&tail->q_full, q_bytes);
       for (int c = 0; c < kchunks; ++c) ptx::tma_load_2d(Qs + (size_t)c * RC * 128, &tmQ, &tail->q_full, c * 64, q_row);
       int it = 0;
@@ -199,44 +241,17 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (!tail->epi_go) break;
       }
       for (int c0 = half * 32; c0 < RC; c0 += 64) {
-        uint32_t v[32];
-        const bool wide = RC - c0 >= 32;
-        if (wide) {
+        const uint32_t rm = tail->real_mask[c0 >> 5];
+        if (RC - c0 >= 32) {
+          uint32_t v[32];
           ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
+          ptx::tmem_wait_ld();
+          readout_chunk<ALL_F32, 32>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1));
         } else {
-          uint32_t w[16];
-          ptx::tmem_ld_32x16(taddr + (uint32_t)c0, w);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) { v[i] = w[i]; v[16 + i] = 0; }
-        }
-        ptx::tmem_wait_ld();
-        const int nrows = wide ? 32 : 16;
-        if (ALL_F32) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if (i < nrows) {
-              const int64_t meta = row_meta[c0 + i];
-              if (meta >= 0 && valid) Lreq[meta + n] = __uint_as_float(v[i]) * scale;
-            }
-          }
-        } else {
-          uint8_t* dst = obuf + (size_t)c0 * (kTileKeys * 2) + (size_t)m * 2;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if (i < nrows)
-              *reinterpret_cast<uint16_t*>(dst + i * (kTileKeys * 2)) =
-                  (uint16_t)key16_of(__uint_as_float(v[i]) * scale);
-          }
-          const uint32_t rm = tail->real_mask[c0 >> 5];
-          if (rm != 0 && valid) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              if (rm & (1u << i)) {
-                const int row = row0 + c0 + i;     // s == 0 here
-                Lreq[((int64_t)(kh * G + row / S1) * S1) * N + n] = __uint_as_float(v[i]) * scale;
-              }
-            }
-          }
+          uint32_t v[16];
+          ptx::tmem_ld_32x16(taddr + (uint32_t)c0, v);
+          ptx::tmem_wait_ld();
+          readout_chunk<ALL_F32, 16>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1));
         }
       }
       // accumulator drained: hand it back to the MMA warp

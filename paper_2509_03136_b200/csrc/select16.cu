@@ -137,7 +137,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   if (k > N) k = N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kh = g / G;
-  const int grow_idx = (g % G) * (S + 1) + (s + 1);      // row within the head group
+  const int grow_idx = (g % G) * S + s;                  // row within the head group (synthetic rows come first)
   const int chunk = grow_idx / RC, crow = grow_idx % RC;
   RowView rv;
   rv.N = N;
@@ -149,7 +149,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   const int nv8 = (N + 7) >> 3;
 
   {
-    const __nv_bfloat16* qrow = Q + (((int64_t)r * Hq + g) * (S + 1) + (s + 1)) * d_k;
+    const __nv_bfloat16* qrow = Q + (((int64_t)r * (Hq / G) + kh) * (G * (S + 1)) + grow_idx) * d_k;
     for (int i = tid; i < d_k; i += kThreads) sh.qf[i] = __bfloat162float(qrow[i]);
     for (int i = tid; i < 256 * 32; i += kThreads) hist1[i] = 0;
     if (tid == 0) sh.ntie = 0;
@@ -157,14 +157,26 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   __syncthreads();
 
   // A. load the row, count high bytes (one counter per bin and lane)
-  for (int v8 = tid; v8 < nv8; v8 += kThreads) {
-    const uint4 v = rv.load_global(v8);
-    if (fits) *reinterpret_cast<uint4*>(row_sm + (size_t)v8 * 8) = v;
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  // (eight 16-byte loads are put in flight before any of them is consumed)
+  for (int base = 0; base < nv8; base += kThreads * 8) {
+    uint4 buf[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      atomicAdd(&hist1[((w[j] >> 8) & 255u) * 32 + lane], 1u);
-      atomicAdd(&hist1[(w[j] >> 24) * 32 + lane], 1u);
+    for (int u = 0; u < 8; ++u) {
+      const int v8 = base + u * kThreads + tid;
+      buf[u] = (v8 < nv8) ? rv.load_global(v8) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v8 = base + u * kThreads + tid;
+      if (v8 < nv8) {
+        if (fits) *reinterpret_cast<uint4*>(row_sm + (size_t)v8 * 8) = buf[u];
+        const uint32_t w[4] = {buf[u].x, buf[u].y, buf[u].z, buf[u].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          atomicAdd(&hist1[((w[j] >> 8) & 255u) * 32 + lane], 1u);
+          atomicAdd(&hist1[(w[j] >> 24) * 32 + lane], 1u);
+        }
+      }
     }
   }
   __syncthreads();

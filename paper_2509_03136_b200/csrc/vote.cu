@@ -46,7 +46,7 @@ score_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     Ks[key * kpitch + d2] = v;
   }
   const int R = G * S1;
-  const __nv_bfloat16* Qbase = Q + ((int64_t)r * Hq + (int64_t)kh * G) * S1 * d_k;   // rows of the group are contiguous
+  const __nv_bfloat16* Qbase = Q + ((int64_t)r * (Hq / G) + kh) * R * d_k;   // the group's rows: synthetic first, then real
   float* Lbase = logits + (int64_t)Hq * S1 * start + (int64_t)kh * G * S1 * N;
 
   for (int c0 = 0; c0 < R; c0 += kScoreRowChunk) {
@@ -73,8 +73,11 @@ score_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int row = c0 + rg * 8 + j;
-      if (row < R) {
+      const int grow = c0 + rg * 8 + j;
+      if (grow < R) {
+        // group row -> (query head, sample): the logits buffer keeps row 0 of a head for the real query
+        const int S = S1 - 1;
+        const int row = (grow < G * S) ? (grow / S) * S1 + grow % S + 1 : (grow - G * S) * S1;
         if (n0 + lane < N) Lbase[(int64_t)row * N + n0 + lane] = acc0[j] * scale;
         if (n0 + lane + 32 < N) Lbase[(int64_t)row * N + n0 + lane + 32] = acc1[j] * scale;
       }
@@ -86,9 +89,9 @@ score_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
 struct SelShared {
   uint32_t cnt[2048];
   unsigned long long mass[2048];
-  unsigned long long red64[kSelThreads / 32];
-  uint32_t red32[kSelThreads / 32];
-  float redf[kSelThreads / 32];
+  unsigned long long red64[32];
+  uint32_t red32[32];
+  float redf[32];
   // results of a digit search
   int bin;
   uint32_t cnt_above;
@@ -101,8 +104,7 @@ __device__ __forceinline__ float block_max(float v, float* red) {
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   float m = red[0];
-#pragma unroll
-  for (int i = 1; i < kSelThreads / 32; ++i) m = fmaxf(m, red[i]);
+  for (int i = 1; i < (int)blockDim.x / 32; ++i) m = fmaxf(m, red[i]);
   __syncthreads();
   return m;
 }
@@ -111,8 +113,7 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   unsigned long long s = 0;
-#pragma unroll
-  for (int i = 0; i < kSelThreads / 32; ++i) s += red[i];
+  for (int i = 0; i < (int)blockDim.x / 32; ++i) s += red[i];
   __syncthreads();
   return s;
 }
@@ -121,8 +122,7 @@ __device__ __forceinline__ uint32_t block_sum_u32(uint32_t v, uint32_t* red) {
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   uint32_t s = 0;
-#pragma unroll
-  for (int i = 0; i < kSelThreads / 32; ++i) s += red[i];
+  for (int i = 0; i < (int)blockDim.x / 32; ++i) s += red[i];
   __syncthreads();
   return s;
 }
@@ -138,7 +138,7 @@ __device__ __forceinline__ unsigned long long mass_fix(float l, float mx) {
 template <bool MASS>
 __device__ void find_bin(SelShared& sh, int nbins, unsigned long long need) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int per = nbins / kSelThreads;
+  const int per = nbins / (int)blockDim.x;
   unsigned long long w = 0;
   uint32_t c = 0;
   for (int i = 0; i < per; ++i) {
@@ -160,7 +160,7 @@ __device__ void find_bin(SelShared& sh, int nbins, unsigned long long need) {
   __syncthreads();
   unsigned long long hi_w = 0;
   uint32_t hi_c = 0;
-  for (int i = warp + 1; i < kSelThreads / 32; ++i) { hi_w += sh.red64[i]; hi_c += sh.red32[i]; }
+  for (int i = warp + 1; i < (int)blockDim.x / 32; ++i) { hi_w += sh.red64[i]; hi_c += sh.red32[i]; }
   const unsigned long long excl_w = ws - w + hi_w;   // weight in bins of higher threads
   const uint32_t excl_c = cs - c + hi_c;
   if (excl_w < need && excl_w + w >= need) {
@@ -198,9 +198,9 @@ __device__ void radix_threshold(const float* __restrict__ row, int N, float mx, 
   uint32_t known_mask = 0;
   for (int pass = 0; pass < 3; ++pass) {
     const int nb = 1 << bits[pass];
-    for (int b = tid; b < nb; b += kSelThreads) { sh.cnt[b] = 0; if (MASS) sh.mass[b] = 0; }
+    for (int b = tid; b < nb; b += blockDim.x) { sh.cnt[b] = 0; if (MASS) sh.mass[b] = 0; }
     __syncthreads();
-    for (int n = tid; n < N; n += kSelThreads) {
+    for (int n = tid; n < N; n += blockDim.x) {
       const float l = row[n];
       const uint32_t key = ordered_key(l);
       if ((key & known_mask) == prefix) {
@@ -231,7 +231,7 @@ __device__ void emit_row(const float* __restrict__ row, int N, uint32_t t, uint3
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool all_ties = ties >= eq_cnt;
   uint32_t taken = 0;   // ties taken so far (ordered path only)
-  for (int base = 0; base < N; base += kSelThreads) {
+  for (int base = 0; base < N; base += blockDim.x) {
     const int n = base + tid;
     uint32_t key = 0;
     bool valid = n < N;
@@ -248,7 +248,7 @@ __device__ void emit_row(const float* __restrict__ row, int N, uint32_t t, uint3
       uint32_t before = taken;
       for (int w = 0; w < warp; ++w) before += sh.red32[w];
       uint32_t total = 0;
-      for (int w = 0; w < kSelThreads / 32; ++w) total += sh.red32[w];
+      for (int w = 0; w < (int)blockDim.x / 32; ++w) total += sh.red32[w];
       const uint32_t rank = before + __popc(tb & ((1u << lane) - 1u));
       sel |= tie && rank < ties;
       taken += total;
@@ -262,22 +262,41 @@ __device__ void emit_row(const float* __restrict__ row, int N, uint32_t t, uint3
 // ---------------------------------------------------------------------------------- top-p rows
 // One CTA per row.  rows_per_head = 1: only the current query's row of every head (row 0);
 // rows_per_head = S+1: every row (top-p mode).  Row 0 always publishes b_step = |C0|.
-__global__ void __launch_bounds__(kSelThreads)
+constexpr int kToppThreads = 1024;
+__global__ void __launch_bounds__(kToppThreads)
 topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
                  int rows_per_head, float p_nuc, int include_c0, int64_t row_words, uint32_t* __restrict__ mask,
-                 int32_t* __restrict__ b_step) {
+                 int32_t* __restrict__ b_step, int row_elems) {
+  extern __shared__ __align__(16) float row_sm[];
   __shared__ SelShared sh;
   const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x;   // row < rows_per_head
   const int start = cu[r], N = cu[r + 1] - start;
   if (N <= 0) { if (row == 0 && threadIdx.x == 0) b_step[r * Hq + g] = 0; return; }
-  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
-  const int tid = threadIdx.x;
+  const float* Lg = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  const int tid = threadIdx.x, nthr = blockDim.x;
 
+  // the row is staged in shared memory when it fits (eight loads in flight per thread), so the
+  // passes below do not wait on global memory; the running maximum is taken on the way in
+  const bool fits = N <= row_elems;
+  const float* L = fits ? row_sm : Lg;
   float mx = -INFINITY;
-  for (int n = tid; n < N; n += kSelThreads) mx = fmaxf(mx, L[n]);
-  mx = block_max(mx, sh.redf);
+  for (int base = 0; base < N; base += nthr * 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int n = base + u * nthr + tid;
+      v[u] = (n < N) ? Lg[n] : -INFINITY;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int n = base + u * nthr + tid;
+      if (fits && n < N) row_sm[n] = v[u];
+      mx = fmaxf(mx, v[u]);
+    }
+  }
+  mx = block_max(mx, sh.redf);      // (its barriers also publish the staged row)
   unsigned long long z = 0;
-  for (int n = tid; n < N; n += kSelThreads) z += mass_fix(L[n], mx);
+  for (int n = tid; n < N; n += nthr) z += mass_fix(L[n], mx);
   z = block_sum_u64(z, sh.red64);
   // smallest integer mass that is >= p * Z
   unsigned long long need = (unsigned long long)ceil((double)p_nuc * (double)z);
@@ -423,12 +442,18 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
     }
     GVOTE_LAUNCH_CHECK("softmax_dump_kernel");
   }
+  // top-p rows up to 48K keys are staged in shared memory (192 KB)
+  int topp_row_elems = (int)max_N;
+  if (topp_row_elems > 48 * 1024) topp_row_elems = 0;
+  const size_t topp_smem = (size_t)topp_row_elems * sizeof(float);
+  if (topp_smem > 16 * 1024)
+    GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topp_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem));
   if (p->sel_mode == GVOTE_SEL_TOPK_C0) {
     dim3 g1(1, Hq, batch);
     {
       LaunchScope scope_("topp_rows_kernel", st);
-      topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0, m.row_words,
-                                                   mask, b_step);
+      topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0,
+                                                            m.row_words, mask, b_step, topp_row_elems);
     }
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
     dim3 g2(p->S, Hq, batch);
@@ -447,8 +472,8 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
     dim3 g1(S1, Hq, batch);
     {
       LaunchScope scope_("topp_rows_kernel", st);
-      topp_rows_kernel<<<g1, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0, m.row_words,
-                                                   mask, b_step);
+      topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0,
+                                                            m.row_words, mask, b_step, topp_row_elems);
     }
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
   }

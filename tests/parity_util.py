@@ -74,3 +74,29 @@ def upload_layer(li, gv, torch, device="cuda"):
         cu=torch.from_numpy(li.cu_seqlens).to(device),
     )
     return d
+
+
+def to_group_major(Q: np.ndarray, G: int) -> np.ndarray:
+    """Oracle query rows [H_q, S+1, d_k] (row 0 = current query) -> the library's layout
+    [H_kv, G*S + G, d_k]: per KV head the S synthetic rows of each of its G heads, then the G
+    current-query rows."""
+    H_q, S1, d_k = Q.shape
+    S, H_kv = S1 - 1, H_q // G
+    out = np.empty((H_kv, G * S1, d_k), dtype=Q.dtype)
+    for g in range(H_q):
+        kh, gl = divmod(g, G)
+        out[kh, gl * S:(gl + 1) * S] = Q[g, 1:]
+        out[kh, G * S + gl] = Q[g, 0]
+    return out
+
+
+def from_group_major(Qg: np.ndarray, G: int) -> np.ndarray:
+    H_kv, R, d_k = Qg.shape
+    S1 = R // G
+    S = S1 - 1
+    out = np.empty((H_kv * G, S1, d_k), dtype=Qg.dtype)
+    for g in range(H_kv * G):
+        kh, gl = divmod(g, G)
+        out[g, 1:] = Qg[kh, gl * S:(gl + 1) * S]
+        out[g, 0] = Qg[kh, G * S + gl]
+    return out

@@ -107,7 +107,7 @@ def test_project_matches_oracle(gv, idx, bias):
     hl = rng.normal(size=(cfg.batch, cfg.d_h)).astype(np.float32)
     d = pu.upload_layer(li, gv, torch)
     ws = gv.alloc_workspace(p, *_geom(cfg))
-    Q = torch.empty(cfg.batch, cfg.n_q_heads, cfg.S + 1, cfg.d_k, dtype=torch.bfloat16, device="cuda")
+    Q = torch.empty(cfg.batch, cfg.n_kv_heads, cfg.G * (cfg.S + 1), cfg.d_k, dtype=torch.bfloat16, device="cuda")
     gv.gvote_project(p, torch.from_numpy(Ht).cuda(), torch.from_numpy(hl).cuda(), d["W_q"], d["b_q"], d["cu"],
                      cfg.batch, Q, ws)
     Qg = Q.float().cpu().numpy().astype(np.float64)
@@ -115,7 +115,7 @@ def test_project_matches_oracle(gv, idx, bias):
     for r in range(cfg.batch):
         Qo = o.queries_for_request(Ht[r].astype(np.float64), hl[r].astype(np.float64), W, li.b_q, cfg.seq_lens[r],
                                    n_q_heads=cfg.n_q_heads, d_k=cfg.d_k, theta=cfg.rope_theta, n_f=cfg.n_f)
-        diff = np.abs(Qg[r] - Qo)
+        diff = np.abs(pu.from_group_major(Qg[r], cfg.G) - Qo)
         assert np.all(diff <= 2.0 ** -7 * np.abs(Qo) + 1e-6)            # at most one bf16 step
         assert (diff == 0).mean() > 0.98
 
@@ -128,7 +128,8 @@ def _run_vote(gv, cfg, li, Q_or, sel_mode, include_c0, want_probs):
     ws = gv.alloc_workspace(p, *geom)
     K = gv.bf16_from_bits(li.K)
     cu = torch.from_numpy(li.cu_seqlens).cuda()
-    Qd = torch.from_numpy(np.ascontiguousarray(np.stack(Q_or))).to(torch.bfloat16).contiguous().cuda()      # values are on the bf16 grid already
+    Qgm = np.ascontiguousarray(np.stack([pu.to_group_major(q, cfg.G) for q in Q_or]))
+    Qd = torch.from_numpy(Qgm).to(torch.bfloat16).contiguous().cuda()   # values are on the bf16 grid already
     mask = torch.full((cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch)), -1, dtype=torch.int32,
                       device="cuda")
     budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
