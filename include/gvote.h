@@ -105,6 +105,27 @@ GVOTE_API int32_t gvote_fit(const gvote_params* p, const void* h, int64_t h_row_
                   const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
                   float* mu, float* var, void* ws, size_t ws_bytes, void* stream);
 
+/* Fit without any allocation (the paper has no counterpart: this entry point exists for the
+ * integration, not for the method).  Same result as gvote_fit, but the per-chunk partial moments
+ * live in a fixed 1 MiB array inside the library's device image (GVOTE_FIT_STATIC_MAX_ENTRIES
+ * pairs of floats, present on every GPU that loads the library until the process exits), so the
+ * caller passes inputs and outputs only and the call obtains no memory, from CUDA or from
+ * anyone else.  Use it where asking for device memory is not possible: inside an allocator or
+ * memory-pool callback, in a serving loop whose pool is frozen after warm-up, on a thread that
+ * may not wait on the allocator's lock.
+ *  - Limit: batch * d_h <= GVOTE_FIT_STATIC_MAX_ENTRIES, else GVOTE_ERR_UNSUPPORTED_SHAPE and
+ *    nothing is enqueued.  Long inputs are fine: fewer, longer row chunks are used instead.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current).  Make that first call before starting any stream capture.
+ *  - All calls on a device share the one array.  It needs no clearing (every entry a call reads
+ *    it has written itself), but two calls whose kernels may overlap on the GPU (different
+ *    streams, no dependency) race on it: serialise them.
+ * Arguments as in gvote_fit, minus the workspace and total_tokens. */
+#define GVOTE_FIT_STATIC_MAX_ENTRIES 131072
+GVOTE_API int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_t h_row_stride,
+                         const int32_t* cu_seqlens, int32_t batch, int64_t max_N,
+                         float* mu, float* var, void* stream);
+
 /* Step 3 / Algorithm 1 line 5.  H_tilde[r][s][c] = mu[r][c] + sqrt(var[r][c]) * z, z a standard
  * normal drawn by Box-Muller from Philox4x32-10 with key = (seed low, seed high) and counter
  * = (c div 4, s, layer_id, r); word pairs (0,1) and (2,3) of a block give channels 4b..4b+3;

@@ -6,6 +6,8 @@
 // rows, every thread keeps shifted first and second moments of four channels in registers, and
 // one (mean, M2) pair per channel and chunk goes to scratch.  A second, tiny kernel merges the
 // chunks with Chan's parallel-variance update in fp64.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace gvote {
@@ -165,3 +167,70 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
 }
 
 }  // namespace gvote
+
+// ---------------------------------------------------------------------------------- no-allocation variant
+// gvote_fit_static: the same two kernels as gvote_fit, with the per-chunk (mean, M2) partials kept
+// in a fixed array that is part of the loaded library image instead of a caller workspace.  It is
+// meant for callers that cannot obtain device memory at the point where they need the fit: code
+// running inside a memory-pool callback, a serving loop whose allocator is frozen after warm-up,
+// or a host thread that must not take the allocator's lock.
+
+namespace gvote {
+namespace {
+
+constexpr size_t kStaticFitEntries = GVOTE_FIT_STATIC_MAX_ENTRIES;   // float2 entries, 1 MiB in all
+static __device__ __align__(256) float2 g_fit_static_scratch[kStaticFitEntries];
+
+// In host code the array's name only stands for the symbol; the address a kernel can use has to
+// be asked for, once per device, while that device is current.
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+float2* g_static_ptr[kMaxDevices] = {};
+
+int32_t static_scratch_for_current_device(float2** out) {
+  int dev = -1;
+  GVOTE_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    GVOTE_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_fit_static_scratch));
+    if (!ptr) return GVOTE_ERR_CUDA;
+    g_static_ptr[dev] = static_cast<float2*>(ptr);
+  }
+  *out = g_static_ptr[dev];
+  return GVOTE_OK;
+}
+
+}  // namespace
+}  // namespace gvote
+
+extern "C" int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_t h_row_stride,
+                                    const int32_t* cu_seqlens, int32_t batch, int64_t max_N, float* mu, float* var,
+                                    void* stream) {
+  using namespace gvote;
+  const int32_t pv = validate_params(p);
+  if (pv != GVOTE_OK) return pv;
+  if (batch < 1 || max_N < 0) return GVOTE_ERR_INVALID_ARG;
+  if (!h || !cu_seqlens || !mu || !var) return GVOTE_ERR_INVALID_ARG;
+  if (!aligned16(h) || !aligned16(cu_seqlens) || !aligned16(mu) || !aligned16(var)) return GVOTE_ERR_UNALIGNED;
+  if (h_row_stride < p->d_h || h_row_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  if (max_N - p->n_s < 2) return GVOTE_ERR_INVALID_ARG;
+  // one chunk per request is the least the kernels can run with
+  const int64_t per_chunk = (int64_t)batch * p->d_h;
+  if (per_chunk > (int64_t)kStaticFitEntries) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  // as many row chunks as fill the GPU, as few as the fixed array holds, at least 32 rows each
+  const int64_t strips = ceil_div(p->d_h, kFitStripCols);
+  int64_t chunks = 1184 / (strips * batch);
+  const int64_t fit_in_array = (int64_t)kStaticFitEntries / per_chunk;
+  const int64_t by_rows = ceil_div(max_N > 0 ? max_N : 1, 32);
+  if (chunks > fit_in_array) chunks = fit_in_array;
+  if (chunks > by_rows) chunks = by_rows;
+  if (chunks < 1) chunks = 1;
+  float2* scratch = nullptr;
+  const int32_t sv = static_scratch_for_current_device(&scratch);
+  if (sv != GVOTE_OK) return sv;
+  // every entry the merge kernel reads is written by the partial kernel of the same call, so the
+  // array needs no clearing between calls
+  return launch_fit(p, h, h_row_stride, cu_seqlens, batch, (int)chunks, scratch, mu, var, (cudaStream_t)stream);
+}

@@ -22,7 +22,7 @@ SEL_TOPK_C0, SEL_TOPP = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
-    "gvote_workspace_bytes", "gvote_fit", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
+    "gvote_workspace_bytes", "gvote_fit", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
     "gvote_compact", "gvote_compress", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
@@ -62,6 +62,8 @@ def load():
     lib.gvote_workspace_bytes.argtypes = [P, i32, i64, i64]
     lib.gvote_fit.restype = i32
     lib.gvote_fit.argtypes = [P, vp, i64, vp, i32, i64, i64, vp, vp, vp, sz, vp]
+    lib.gvote_fit_static.restype = i32
+    lib.gvote_fit_static.argtypes = [P, vp, i64, vp, i32, i64, vp, vp, vp]
     lib.gvote_sample.restype = i32
     lib.gvote_sample.argtypes = [P, vp, vp, i32, vp, vp, vp]
     lib.gvote_project.restype = i32
@@ -167,6 +169,20 @@ def gvote_fit(p, h, cu_seqlens, geom, mu, var, ws) -> None:
     _dev(cu_seqlens, torch.int32, "cu_seqlens"); _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
     _check(load().gvote_fit(ctypes.byref(p), _ptr(h), h.stride(0), _ptr(cu_seqlens), batch, total, max_N,
                             _ptr(mu), _ptr(var), _ptr(ws), ws.numel(), _stream()), "gvote_fit")
+
+
+FIT_STATIC_MAX_ENTRIES = 131072
+
+
+def gvote_fit_static(p, h, cu_seqlens, batch: int, max_N: int, mu, var) -> None:
+    """`gvote_fit` for callers that cannot ask for device memory where they stand (an allocator
+    callback, a serving loop with a frozen pool): no workspace argument, the partial sums go to
+    a fixed array inside the library.  Needs batch * d_h <= FIT_STATIC_MAX_ENTRIES; calls that
+    could overlap on the GPU must be serialised by the caller, they share that array."""
+    _dev(h, torch.float32 if p.h_dtype == DTYPE_F32 else torch.bfloat16, "h", dense=False)
+    _dev(cu_seqlens, torch.int32, "cu_seqlens"); _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
+    _check(load().gvote_fit_static(ctypes.byref(p), _ptr(h), h.stride(0), _ptr(cu_seqlens), batch, max_N,
+                                   _ptr(mu), _ptr(var), _stream()), "gvote_fit_static")
 
 
 def gvote_sample(p, mu, var, batch, H_tilde, raw=None) -> None:
