@@ -182,6 +182,7 @@ def workload_config(cfg, args):
             "n_f": cfg.n_f, "n_s": cfg.n_s, "sel_mode": "topk_c0", "h_dtype": "f32", "kv_dtype": "bf16",
             "l2": "inputs larger than L2 (every layer has its own tensors; K/V restored from pristine copies "
                   "between steps, outside the timed intervals)",
+            "streams": max(1, args.streams),
             "timing": "sum of per-step CUDA-event intervals on the launch stream"}
 
 
@@ -194,6 +195,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
+    ap.add_argument("--streams", type=int, default=1,
+                    help="CUDA streams the layers of a step are spread over (each with its own workspace)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -239,7 +242,10 @@ def main():
 
     dev = torch.device("cuda", local)
     p_layer = [gv.params_from_config(cfg, layer_id=l) for l in range(L)]
-    ws = gv.alloc_workspace(p_layer[0], *geom)
+    n_streams = max(1, min(args.streams, L))
+    ws_s = [gv.alloc_workspace(p_layer[0], *geom) for _ in range(n_streams)]
+    ws = ws_s[0]
+    side = [torch.cuda.Stream(device=dev) for _ in range(n_streams - 1)]
     cu = torch.from_numpy(layers[0].cu_seqlens).to(dev)
     d_h = [torch.from_numpy(li.h).to(dev) for li in layers]
     d_W = [gv.bf16_from_bits(li.W_q, dev) for li in layers]
@@ -257,9 +263,23 @@ def main():
             d_K[l].copy_(d_K0[l]); d_V[l].copy_(d_V0[l])
 
     def one_pass():
+        # layers are independent (Section 3.2): layer l goes to stream l mod n_streams, so the short,
+        # latency-bound kernels of one layer run under the streaming kernels of another
+        main = torch.cuda.current_stream()
+        if side:
+            fork = torch.cuda.Event()
+            fork.record(main)
+            for st in side:
+                st.wait_event(fork)
         for l in range(L):
-            gv.gvote_compress(p_layer[l], d_h[l], d_W[l], None, d_K[l], d_V[l], cu, geom, d_mask[l], d_budget[l],
-                              d_bstep[l], ws)
+            k = l % n_streams
+            with torch.cuda.stream(main if k == 0 else side[k - 1]):
+                gv.gvote_compress(p_layer[l], d_h[l], d_W[l], None, d_K[l], d_V[l], cu, geom, d_mask[l], d_budget[l],
+                                  d_bstep[l], ws_s[k])
+        for st in side:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
 
     def barrier():
         torch.cuda.synchronize()
@@ -291,7 +311,8 @@ def main():
     total_ms = timed_steps(args.steps)
     tc1 = time.perf_counter()
     launches = gv.gvote_launch_count() - n0
-    assert gv.gvote_poll_status(ws) == 0, "a device-side wait timed out"
+    for w in ws_s:
+        assert gv.gvote_poll_status(w) == 0, "a device-side wait timed out"
     if dist is not None:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)

@@ -83,7 +83,7 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   if (chunks > max_chunks) chunks = max_chunks;
   if (chunks < 1) chunks = 1;
   m.fit_chunks = (int)chunks;
-  m.proj_splits = 1;
+  m.proj_splits = project_umma_splits(p, batch * (p->S + 1));
   m.n_tiles = (total_tokens >> 7) + batch;
   m.row_words = gvote_mask_row_words(total_tokens, batch);
   size_t off = 0;
@@ -99,6 +99,8 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   m.rope = take((size_t)batch * 4 * (p->d_k / 2) * sizeof(float));
   m.logits = take((size_t)p->n_q_heads * S1 * (size_t)total_tokens * sizeof(float));
   m.keys16 = take(keys16_elems(p, batch, total_tokens) * sizeof(uint16_t));
+  m.real_scratch_bytes = real_topp_scratch_bytes(p, batch);
+  m.real_scratch = take(m.real_scratch_bytes);
   m.prefix = take((size_t)p->n_kv_heads * m.row_words * sizeof(int32_t));
   m.flags = take(((size_t)2 * p->n_kv_heads * m.n_tiles + 4) * sizeof(int32_t));
   m.total = off;
@@ -227,17 +229,18 @@ int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_strid
   cudaStream_t st = (cudaStream_t)stream;
   float* mu = reinterpret_cast<float*>(w + m.mu);
   float* var = reinterpret_cast<float*>(w + m.var);
-  float* Ht = reinterpret_cast<float*>(w + m.h_tilde);
   __nv_bfloat16* Q = reinterpret_cast<__nv_bfloat16*>(w + m.q_bf16);
-  PROPAGATE(launch_fit(p, h, h_row_stride, cu_seqlens, batch, m.fit_chunks,
-                       reinterpret_cast<float2*>(w + m.fit_partial), mu, var, st));
-  PROPAGATE(launch_sample(p, mu, var, batch, Ht, nullptr, st));
+  PROPAGATE(launch_fit_partial(p, h, h_row_stride, cu_seqlens, batch, m.fit_chunks,
+                               reinterpret_cast<float2*>(w + m.fit_partial), st));
+  __nv_bfloat16* X = reinterpret_cast<__nv_bfloat16*>(w + m.x_bf16);
+  float* rope = reinterpret_cast<float*>(w + m.rope);
   if (h_last_or_null)
-    PROPAGATE(launch_project(p, Ht, h_last_or_null, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w,
-                             Q, st));
+    PROPAGATE(launch_prep(p, reinterpret_cast<const float2*>(w + m.fit_partial), m.fit_chunks, h_last_or_null, p->d_h,
+                          nullptr, cu_seqlens, batch, mu, var, X, rope, st));
   else
-    PROPAGATE(launch_project(p, Ht, h, h_row_stride, cu_seqlens, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q,
-                             st));
+    PROPAGATE(launch_prep(p, reinterpret_cast<const float2*>(w + m.fit_partial), m.fit_chunks, h, h_row_stride,
+                          cu_seqlens, cu_seqlens, batch, mu, var, X, rope, st));
+  PROPAGATE(launch_project_staged(p, X, rope, W_q, wq_ld, b_q_or_null, batch, m, w, Q, st));
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
                         max_N, mask, nullptr, b_step, nullptr, m, w, st));   // budgets come from the scan below
   return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,

@@ -66,6 +66,8 @@ struct WorkspaceMap {
   size_t rope;          // float [batch][4][d_k/2]  (cos0, sin0, cbar, sbar)
   size_t logits;        // float [Hq*(S+1) * total_tokens], request-major
   size_t keys16;        // uint16 [Hq*S * (padded tokens)]: 16-bit logit keys of the synthetic rows
+  size_t real_scratch;  // row maxima and mass histograms of the current-query rows (topp_real.cu)
+  size_t real_scratch_bytes;
   size_t prefix;        // int32 [Hkv][row_words]  exclusive popcount prefix per mask word
   size_t flags;         // int32 [2*Hkv*n_tiles + 4]  compaction "tile loaded" flags + ticket
   size_t total;
@@ -80,14 +82,27 @@ struct WorkspaceMap {
 struct ScoreGeometry { int RC; int row_chunks; };
 ScoreGeometry score_geometry(const gvote_params* p);
 size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens);
+size_t real_topp_scratch_bytes(const gvote_params* p, int32_t batch);
 WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
 // ---------------------------------------------------------------------------------- stage launchers
 // (each enqueues kernels on `st`; pointers are device pointers; see gvote.h for the layouts)
 int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
                    int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st);
+int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                           int fit_chunks, float2* partial, cudaStream_t st);
 int32_t launch_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch,
                       float* H_tilde, uint32_t* raw, cudaStream_t st);
+// Fused middle of the whole pass: merges the fit partials (mu, var), draws the S samples and writes
+// the bf16 projection input X = [h_last; H~] and the RoPE tables, in one launch.
+int32_t launch_prep(const gvote_params* p, const float2* partial, int fit_chunks, const void* h_last,
+                    int64_t h_last_ld, const int32_t* h_last_rows_from_cu, const int32_t* cu, int32_t batch,
+                    float* mu, float* var, __nv_bfloat16* X, float* rope_table, cudaStream_t st);
+// Projection of a staged X (bf16 [batch*(S+1), d_h]) with ready RoPE tables: GEMM + finish.
+int32_t launch_project_staged(const gvote_params* p, const __nv_bfloat16* X, const float* rope_table, const void* W_q,
+                              int64_t wq_ld, const float* b_q, int32_t batch, const WorkspaceMap& m, char* ws,
+                              __nv_bfloat16* Q, cudaStream_t st);
+int project_umma_splits(const gvote_params* p, int rows_total);
 int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* h_last, int64_t h_last_ld,
                        const int32_t* h_last_rows_from_cu,  // when non-null: row index = cu[r+1]-1 of h_last
                        const void* W_q, int64_t wq_ld, const float* b_q, const int32_t* cu, int32_t batch,
@@ -129,6 +144,43 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 // tile offset in the compaction tile list (both over-allocate by one unit per request).
 __device__ __forceinline__ int64_t mask_word_offset(int cu_r, int r) { return (int64_t)(cu_r >> 5) + r; }
 __device__ __forceinline__ int64_t tile_offset(int cu_r, int r) { return (int64_t)(cu_r >> 7) + r; }
+
+
+// Rows of chunk `c` of a request whose fitted rows are [first, last): [a, b).
+__device__ __forceinline__ void fit_chunk_rows(int first, int last, int chunks, int c, int& a, int& b) {
+  const int n = max(last - first, 0);
+  const int per = (n + chunks - 1) / chunks;
+  a = min(first + c * per, last);
+  b = min(a + per, last);
+}
+
+// Merging the per-chunk (mean, M2) pairs of one channel (the pairwise update of Chan, Golub and
+// LeVeque, written against a common reference value so that one pass and no division per chunk
+// suffice): with ref = mean of chunk 0, A = sum n_c (mean_c - ref), B = sum n_c (mean_c - ref)^2,
+// C = sum M2_c, the merged mean is ref + A/n and the merged M2 is C + B - A^2/n.  `lane` of
+// `lanes` takes every lanes-th chunk; the caller adds the lanes' (n, A, B + C) and finishes.
+struct FitMoments { double n, a, bc; };
+__device__ __forceinline__ FitMoments fit_merge_lane(const float2* __restrict__ partial, int r, int chunks, int d_h,
+                                                     int col, int first, int last, int lane, int lanes, double ref) {
+  FitMoments m{0.0, 0.0, 0.0};
+  for (int c = lane; c < chunks; c += lanes) {
+    int a, b;
+    fit_chunk_rows(first, last, chunks, c, a, b);
+    if (b <= a) continue;
+    const float2 pc = partial[((int64_t)(r * chunks + c)) * d_h + col];
+    const double nc = (double)(b - a), d = (double)pc.x - ref;
+    m.n += nc;
+    m.a = fma(nc, d, m.a);
+    m.bc += fma(nc * d, d, (double)pc.y);
+  }
+  return m;
+}
+__device__ __forceinline__ void fit_merge_finish(const FitMoments& m, double ref, float& mu, float& var) {
+  const double mean = ref + m.a / m.n;
+  const double m2 = m.bc - m.a * m.a / m.n;
+  mu = (float)mean;
+  var = (float)(fmax(m2, 0.0) / (m.n - 1.0));      // NaN/inf when fewer than 2 rows
+}
 
 #endif  // __CUDACC__
 

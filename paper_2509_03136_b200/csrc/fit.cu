@@ -40,14 +40,6 @@ __device__ __forceinline__ void acc4(float4& s1, float4& s2, const float4& v, co
   s2.z = fmaf(dz, dz, s2.z); s2.w = fmaf(dw, dw, s2.w);
 }
 
-// Rows of chunk `c` of a request whose fitted rows are [first, last): [a, b).
-__device__ __forceinline__ void chunk_rows(int first, int last, int chunks, int c, int& a, int& b) {
-  int n = max(last - first, 0);
-  int per = (n + chunks - 1) / chunks;
-  a = min(first + c * per, last);
-  b = min(a + per, last);
-}
-
 template <typename T>
 __global__ void __launch_bounds__(kFitTx* kFitTy)
 fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restrict__ cu, int n_s, int d_h,
@@ -57,7 +49,7 @@ fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restric
   const int col = (blockIdx.x * kFitTx + tx) * 4;
   const bool active = col < d_h;
   int a, b;
-  chunk_rows(cu[r] + n_s, cu[r + 1], chunks, c, a, b);
+  fit_chunk_rows(cu[r] + n_s, cu[r + 1], chunks, c, a, b);
 
   float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1, sh = s1;
   if (active && a < b) {
@@ -103,64 +95,57 @@ fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restric
   }
 }
 
-// Chan et al. pairwise update over the chunks of a request, in fp64.  A CTA covers 32 channels;
-// eight row lanes each fold every eighth chunk, then lane 0 folds the eight partial results.
-struct Moments { double n, mean, m2; };
-__device__ __forceinline__ void chan_merge(Moments& a, double nc, double mean_c, double m2_c) {
-  if (nc <= 0.0) return;
-  const double tot = a.n + nc;
-  const double delta = mean_c - a.mean;
-  a.mean += delta * nc / tot;
-  a.m2 += m2_c + delta * delta * a.n * nc / tot;
-  a.n = tot;
-}
-
+// Merge of the chunks of a request (see fit_merge_lane).  A CTA covers 32 channels; eight row lanes
+// each fold every eighth chunk, then lane 0 adds the eight partial results.
 __global__ void __launch_bounds__(256)
 fit_finalize_kernel(const float2* __restrict__ partial, const int32_t* __restrict__ cu, int n_s, int d_h, int chunks,
                     float* __restrict__ mu, float* __restrict__ var) {
-  __shared__ Moments sm[8][32];
+  __shared__ FitMoments sm[8][32];
   const int r = blockIdx.y;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int col = blockIdx.x * 32 + tx;
   const int first = cu[r] + n_s, last = cu[r + 1];
-  Moments acc{0.0, 0.0, 0.0};
+  FitMoments acc{0.0, 0.0, 0.0};
+  double ref = 0.0;
   if (col < d_h) {
-    for (int c = ty; c < chunks; c += 8) {
-      int a, b;
-      chunk_rows(first, last, chunks, c, a, b);
-      const float2 pc = partial[((int64_t)(r * chunks + c)) * d_h + col];
-      chan_merge(acc, (double)(b - a), (double)pc.x, (double)pc.y);
-    }
+    ref = (double)partial[((int64_t)r * chunks) * d_h + col].x;
+    acc = fit_merge_lane(partial, r, chunks, d_h, col, first, last, ty, 8, ref);
   }
   sm[ty][tx] = acc;
   __syncthreads();
   if (ty == 0 && col < d_h) {
-    for (int j = 1; j < 8; ++j) chan_merge(acc, sm[j][tx].n, sm[j][tx].mean, sm[j][tx].m2);
-    mu[(int64_t)r * d_h + col] = (float)acc.mean;
-    var[(int64_t)r * d_h + col] = (float)(acc.m2 / (acc.n - 1.0));   // NaN/inf when fewer than 2 rows
+    for (int j = 1; j < 8; ++j) { acc.n += sm[j][tx].n; acc.a += sm[j][tx].a; acc.bc += sm[j][tx].bc; }
+    fit_merge_finish(acc, ref, mu[(int64_t)r * d_h + col], var[(int64_t)r * d_h + col]);
   }
 }
 
 }  // namespace
 
-int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                   int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st) {
+int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                           int fit_chunks, float2* partial, cudaStream_t st) {
   const int strips = (int)ceil_div(p->d_h, kFitStripCols);
   dim3 grid(strips, fit_chunks, batch), block(kFitTx, kFitTy);
   {
     LaunchScope scope_("fit_partial_kernel", st);
-  if (p->h_dtype == GVOTE_DTYPE_F32) {
-    fit_partial_kernel<float><<<grid, block, 0, st>>>((const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks, partial);
-  } else {
-    fit_partial_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)h, ld, cu, p->n_s, p->d_h,
-                                                              fit_chunks, partial);
-  }
+    if (p->h_dtype == GVOTE_DTYPE_F32) {
+      fit_partial_kernel<float><<<grid, block, 0, st>>>((const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks, partial);
+    } else {
+      fit_partial_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)h, ld, cu, p->n_s, p->d_h,
+                                                                fit_chunks, partial);
+    }
   }
   GVOTE_LAUNCH_CHECK("fit_partial_kernel");
+  return GVOTE_OK;
+}
+
+int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                   int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st) {
+  const int32_t rc = launch_fit_partial(p, h, ld, cu, batch, fit_chunks, partial, st);
+  if (rc != GVOTE_OK) return rc;
   dim3 g2((unsigned)ceil_div(p->d_h, 32), batch);
   {
     LaunchScope scope_("fit_finalize_kernel", st);
-  fit_finalize_kernel<<<g2, 256, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
+    fit_finalize_kernel<<<g2, 256, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
   }
   GVOTE_LAUNCH_CHECK("fit_finalize_kernel");
   return GVOTE_OK;

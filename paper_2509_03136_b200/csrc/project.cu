@@ -59,7 +59,8 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ cu, int d_k, doubl
 }
 
 // ---------------------------------------------------------------------------------- GEMM (SIMT)
-// out[row][f] = sum_c X[row][c] * W[f][c].  One warp per output feature, kProjRows rows per CTA;
+// The tensor-core kernel lives in project_umma.cu; this one takes over when a tensor map cannot be
+// built for W_q or X.  out[row][f] = sum_c X[row][c] * W[f][c].  One warp per output feature, kProjRows rows per CTA;
 // the X chunk is staged in shared memory and shared by the CTA's warps.
 constexpr int kProjWarps = 8;
 constexpr int kProjRows = 40;
@@ -157,48 +158,66 @@ __global__ void project_finish_kernel(const float* __restrict__ qf, int splits, 
 
 }  // namespace
 
+int32_t launch_project_umma(const gvote_params* p, const __nv_bfloat16* X, const __nv_bfloat16* W, int64_t wq_ld,
+                            int rows_total, int splits, float* part, int32_t* status, cudaStream_t st);
+
+int32_t launch_project_staged(const gvote_params* p, const __nv_bfloat16* X, const float* rope_table, const void* W_q,
+                              int64_t wq_ld, const float* b_q, int32_t batch, const WorkspaceMap& m, char* ws,
+                              __nv_bfloat16* Q, cudaStream_t st) {
+  const int d_h = p->d_h, S = p->S, F = p->n_q_heads * p->d_k;
+  const int rows_total = batch * (S + 1);
+  float* qf = reinterpret_cast<float*>(ws + m.q_f32);
+  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
+
+  // tensor-core path; the SIMT kernel serves operands a TMA tensor map cannot describe
+  int splits = m.proj_splits;
+  const int32_t rc = launch_project_umma(p, X, (const __nv_bfloat16*)W_q, wq_ld, rows_total, splits, qf, status, st);
+  if (rc == GVOTE_ERR_UNSUPPORTED_SHAPE) {
+    splits = 1;
+    dim3 gp((unsigned)ceil_div(F, kProjWarps), (unsigned)ceil_div(rows_total, kProjRows));
+    {
+      LaunchScope scope_("project_simt_kernel", st);
+      project_simt_kernel<<<gp, kProjWarps * 32, 0, st>>>(X, (const __nv_bfloat16*)W_q, wq_ld, rows_total, d_h, F, qf);
+    }
+    GVOTE_LAUNCH_CHECK("project_simt_kernel");
+  } else if (rc != GVOTE_OK) {
+    return rc;
+  }
+
+  dim3 gf((unsigned)ceil_div((int64_t)p->n_q_heads * (p->d_k / 2), 128), S + 1, batch);
+  {
+    LaunchScope scope_("project_finish_kernel", st);
+    project_finish_kernel<<<gf, 128, 0, st>>>(qf, splits, (int64_t)rows_total * F, b_q, rope_table, S, p->n_q_heads,
+                                              p->n_q_heads / p->n_kv_heads, p->d_k, Q);
+  }
+  GVOTE_LAUNCH_CHECK("project_finish_kernel");
+  return GVOTE_OK;
+}
+
 int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* h_last, int64_t h_last_ld,
                        const int32_t* h_last_rows_from_cu, const void* W_q, int64_t wq_ld, const float* b_q,
                        const int32_t* cu, int32_t batch, const WorkspaceMap& m, char* ws, __nv_bfloat16* Q,
                        cudaStream_t st) {
-  const int d_h = p->d_h, S = p->S, F = p->n_q_heads * p->d_k;
-  const int rows_total = batch * (S + 1);
+  const int d_h = p->d_h, S = p->S;
   __nv_bfloat16* X = reinterpret_cast<__nv_bfloat16*>(ws + m.x_bf16);
-  float* qf = reinterpret_cast<float*>(ws + m.q_f32);
   float* table = reinterpret_cast<float*>(ws + m.rope);
 
   dim3 gx((unsigned)ceil_div(d_h, 256), S + 1, batch);
   {
     LaunchScope scope_("xstage_kernel", st);
-  if (p->h_dtype == GVOTE_DTYPE_F32)
-    xstage_kernel<float><<<gx, 256, 0, st>>>(H_tilde, (const float*)h_last, h_last_ld, h_last_rows_from_cu, d_h, S, X);
-  else
-    xstage_kernel<__nv_bfloat16><<<gx, 256, 0, st>>>(H_tilde, (const __nv_bfloat16*)h_last, h_last_ld,
-                                                     h_last_rows_from_cu, d_h, S, X);
+    if (p->h_dtype == GVOTE_DTYPE_F32)
+      xstage_kernel<float><<<gx, 256, 0, st>>>(H_tilde, (const float*)h_last, h_last_ld, h_last_rows_from_cu, d_h, S, X);
+    else
+      xstage_kernel<__nv_bfloat16><<<gx, 256, 0, st>>>(H_tilde, (const __nv_bfloat16*)h_last, h_last_ld,
+                                                       h_last_rows_from_cu, d_h, S, X);
   }
   GVOTE_LAUNCH_CHECK("xstage_kernel");
-
   {
     LaunchScope scope_("rope_table_kernel", st);
-  rope_table_kernel<<<batch, 64, 0, st>>>(cu, p->d_k, p->rope_theta, p->n_f, table);
+    rope_table_kernel<<<batch, 64, 0, st>>>(cu, p->d_k, p->rope_theta, p->n_f, table);
   }
   GVOTE_LAUNCH_CHECK("rope_table_kernel");
-
-  dim3 gp((unsigned)ceil_div(F, kProjWarps), (unsigned)ceil_div(rows_total, kProjRows));
-  {
-    LaunchScope scope_("project_simt_kernel", st);
-  project_simt_kernel<<<gp, kProjWarps * 32, 0, st>>>(X, (const __nv_bfloat16*)W_q, wq_ld, rows_total, d_h, F, qf);
-  }
-  GVOTE_LAUNCH_CHECK("project_simt_kernel");
-
-  dim3 gf((unsigned)ceil_div((int64_t)p->n_q_heads * (p->d_k / 2), 128), S + 1, batch);
-  {
-    LaunchScope scope_("project_finish_kernel", st);
-  project_finish_kernel<<<gf, 128, 0, st>>>(qf, 1, (int64_t)rows_total * F, b_q, table, S, p->n_q_heads,
-                                            p->n_q_heads / p->n_kv_heads, p->d_k, Q);
-  }
-  GVOTE_LAUNCH_CHECK("project_finish_kernel");
-  return GVOTE_OK;
+  return launch_project_staged(p, X, table, W_q, wq_ld, b_q, batch, m, ws, Q, st);
 }
 
 }  // namespace gvote

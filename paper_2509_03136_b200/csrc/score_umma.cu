@@ -12,8 +12,8 @@
 //   warps 2-9: read-out - tcgen05.ld 32 rows at a time; thread = one key; two warps per lane quadrant
 //
 // Read-out, default mode.  The S x N logits never reach HBM as fp32.  Every logit is scaled and
-// turned into the upper 16 bits of an order-preserving image of its fp32 pattern (all the top-k
-// search needs to bracket its threshold), staged in shared memory as a [row][128 keys] tile and
+// turned into a 16-bit key (its half-precision rounding: all the top-k search needs to bracket its
+// threshold), staged in shared memory as a [row][128 keys] tile and
 // written with one bulk copy per tile into a tile-blocked buffer keys16[head][tile][chunk][row][128].
 // Only the rows of the current query (one per query head) are also written as fp32, because the
 // softmax mass of line 2 needs them exactly.  In the all-fp32 mode (per-sample top-p, softmax dump)
@@ -33,6 +33,7 @@ constexpr int kStages = 3;
 constexpr int kEpiWarps = 8;
 constexpr int kUmmaThreads = 64 + 32 * kEpiWarps;
 constexpr int kMaxChunks32 = 8;   // RC <= 256
+constexpr int kMaxGroup = 64;     // query heads per KV head
 
 struct ScoreSmemTail {
   uint64_t full[kStages];
@@ -44,6 +45,7 @@ struct ScoreSmemTail {
   volatile int abort_flag;
   volatile int epi_go;                // read-out warps continue (decided by their leader, read after a barrier)
   uint32_t real_mask[kMaxChunks32];   // per 32-row chunk: rows that belong to the current query
+  uint32_t rowmax[kMaxGroup];         // running maximum (order-preserving image) of each current-query row
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -56,20 +58,20 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
 }
 
 
-// Two fp32 logits -> two 16-bit keys: round to bf16 (monotone), then flip so that unsigned order
-// equals numeric order: negative values get all bits inverted, others get the sign bit set.
+// Two fp32 logits -> two 16-bit keys: their half-precision roundings (monotone; 11 significant bits,
+// values beyond the half range saturate to the largest finite half).
 __device__ __forceinline__ uint32_t key16x2_of(float lo, float hi) {
   uint32_t p;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p) : "f"(hi), "f"(lo));
-  const uint32_t neg = (p >> 15) & 0x00010001u;          // 1 per negative half
-  return p ^ (neg * 0x7fffu + 0x80008000u);              // 0xffff for negative halves, 0x8000 otherwise
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(p) : "f"(hi), "f"(lo));
+  return p;
 }
 
 // Read-out of NR accumulator columns (query rows c0 .. c0+NR-1) held by this thread for key n.
 template <bool ALL_F32, int NR>
 __device__ __forceinline__ void readout_chunk(const uint32_t (&v)[NR], int c0, uint32_t real_mask,
                                               const int64_t* row_meta, uint8_t* obuf, int m, int n, bool valid,
-                                              float scale, float* Lreq, int N, int S1, int g0, int real_row0) {
+                                              float scale, float* Lreq, int N, int S1, int g0, int real_row0,
+                                              uint32_t* rowmax_s) {
   if (ALL_F32) {
 #pragma unroll
     for (int i = 0; i < NR; ++i) {
@@ -77,21 +79,25 @@ __device__ __forceinline__ void readout_chunk(const uint32_t (&v)[NR], int c0, u
       if (meta >= 0 && valid) Lreq[meta + n] = __uint_as_float(v[i]) * scale;
     }
   } else {
-    // keys need the order of the logits only, so the positive scale is not applied to them
+    // the scaled logit is what gets rounded: 1/sqrt(d_k) keeps it well inside the half range
     uint8_t* dst = obuf + (size_t)c0 * (kTileKeys * 2) + (size_t)m * 2;
 #pragma unroll
     for (int i = 0; i < NR; i += 2) {
-      const uint32_t kk = key16x2_of(__uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+      const uint32_t kk = key16x2_of(__uint_as_float(v[i]) * scale, __uint_as_float(v[i + 1]) * scale);
       *reinterpret_cast<uint16_t*>(dst + i * (kTileKeys * 2)) = (uint16_t)kk;
       *reinterpret_cast<uint16_t*>(dst + (i + 1) * (kTileKeys * 2)) = (uint16_t)(kk >> 16);
     }
-    if (real_mask != 0 && valid) {
-      // rows of the current query (they follow the synthetic rows of the group): exact fp32 logits
+    if (real_mask != 0) {
+      // rows of the current query (they follow the synthetic rows of the group): exact fp32 logits,
+      // and their running maximum for the softmax of Algorithm 1 line 1 (real_mask is warp-uniform)
 #pragma unroll
       for (int i = 0; i < NR; ++i) {
         if (real_mask & (1u << i)) {
-          const int g = g0 + (real_row0 + c0 + i);
-          Lreq[((int64_t)g * S1) * N + n] = __uint_as_float(v[i]) * scale;
+          const int gl = real_row0 + c0 + i;
+          const float l = __uint_as_float(v[i]) * scale;
+          if (valid) Lreq[((int64_t)(g0 + gl) * S1) * N + n] = l;
+          const uint32_t wmax = __reduce_max_sync(0xffffffffu, valid ? ordered_key(l) : 0u);
+          if ((threadIdx.x & 31) == 0) atomicMax(&rowmax_s[gl], wmax);
         }
       }
     }
@@ -103,7 +109,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                   const int32_t* __restrict__ cu, int Hq, int G, int S1, int d_k, int RC, int row_chunks,
                   int acc_cols, int n_out, float scale, int64_t n_tiles_total, float* __restrict__ logits,
-                  uint16_t* __restrict__ keys16, int32_t* __restrict__ status) {
+                  uint16_t* __restrict__ keys16, uint32_t* __restrict__ rowmax, int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int r = blockIdx.z;
   const int kh = blockIdx.y / row_chunks, chunk = blockIdx.y % row_chunks;
@@ -151,6 +157,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     ptx::mbar_init(&tail->q_full, 1);
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(&tail->tmem_full[a], 1); ptx::mbar_init(&tail->tmem_empty[a], kEpiWarps); }
     tail->abort_flag = 0;
+    for (int i = 0; i < kMaxGroup; ++i) tail->rowmax[i] = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmK);
     ptx::prefetch_tensormap(&tmQ);
@@ -246,12 +253,12 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
           uint32_t v[32];
           ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
           ptx::tmem_wait_ld();
-          readout_chunk<ALL_F32, 32>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1));
+          readout_chunk<ALL_F32, 32>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1), tail->rowmax);
         } else {
           uint32_t v[16];
           ptx::tmem_ld_32x16(taddr + (uint32_t)c0, v);
           ptx::tmem_wait_ld();
-          readout_chunk<ALL_F32, 16>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1));
+          readout_chunk<ALL_F32, 16>(v, c0, rm, row_meta, obuf, m, n, valid, scale, Lreq, N, S1, kh * G, row0 - G * (S1 - 1), tail->rowmax);
         }
       }
       // accumulator drained: hand it back to the MMA warp
@@ -278,6 +285,8 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
     atomicExch(&status[1], 2);
   }
+  if (!ALL_F32 && rowmax != nullptr && (int)threadIdx.x < G && tail->rowmax[threadIdx.x] != 0)
+    atomicMax(&rowmax[r * Hq + kh * G + (int)threadIdx.x], tail->rowmax[threadIdx.x]);
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, 2 * acc_cols);
@@ -288,7 +297,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
 // ------------------------------------------------------------------------------------ host side
 bool score_umma_supported(const gvote_params* p) {
-  return p->d_k % 64 == 0 && p->d_k <= 256;
+  return p->d_k % 64 == 0 && p->d_k <= 256 && p->n_q_heads / p->n_kv_heads <= kMaxGroup;
 }
 
 ScoreGeometry score_geometry(const gvote_params* p) {
@@ -311,7 +320,8 @@ size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens) 
 // operands (the caller then takes the SIMT path).
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                          bool all_f32, float* logits, uint16_t* keys16, int32_t* status, cudaStream_t st) {
+                          bool all_f32, float* logits, uint16_t* keys16, uint32_t* rowmax, int32_t* status,
+                          cudaStream_t st) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
   const ScoreGeometry geo = score_geometry(p);
   const int RC = geo.RC, row_chunks = geo.row_chunks;
@@ -354,7 +364,7 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
   {
     LaunchScope scope_("score_umma_kernel", st);
     kern<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, S1, d_k, RC, row_chunks, acc_cols, n_out, scale,
-                                           n_tiles_total, logits, keys16, status);
+                                           n_tiles_total, logits, keys16, rowmax, status);
   }
   GVOTE_LAUNCH_CHECK("score_umma_kernel");
   return GVOTE_OK;

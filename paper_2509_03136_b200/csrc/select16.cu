@@ -1,38 +1,78 @@
 // Algorithm 1 line 9 for the synthetic queries: the k = |C0| largest logits of a row, found on the
-// 16-bit keys the tensor-core score kernel leaves behind (the upper half of an order-preserving
-// image of each fp32 logit), and OR-ed into the head's keep mask (line 10).
+// 16-bit keys the tensor-core score kernel leaves behind (each logit rounded to half precision), and
+// OR-ed into the head's keep mask (line 10).
 //
-// One CTA per synthetic row.
-//   A. The row is read once from the tile-blocked key buffer into shared memory; while it streams
-//      in, its high bytes are counted in a histogram that keeps one counter per (bin, lane), so no
-//      two lanes of a warp ever hit the same address.
-//   B. The 256 bins are reduced; the bin holding the k-th largest key is found by a suffix scan.
-//   C. The low bytes of the keys in that bin are counted (plain 256-bin histogram: few keys, well
-//      spread), which fixes the 16-bit threshold T: keys above T are selected outright.
-//   D. One pass over the row emits the mask words (8 keys per thread, 4 threads per word) and
-//      collects the keys equal to T.  Those candidates share 16 leading bits, so their order is
-//      settled exactly: their logits are recomputed in fp32 from Q and K and ranked by (value
-//      descending, index ascending); the first k - #above of them are selected.
-// Rows longer than the shared-memory budget are streamed from global memory in each pass instead.
+// One small CTA per synthetic row, many resident per SM.  Keys are compared as half-precision numbers,
+// two per instruction; for counting they are mapped to an order-preserving 16-bit code.
+//   1. A fixed, evenly spaced sample of 2048 keys brackets the k-th largest key between two of the
+//      sample's order statistics, a few standard deviations of the sampling error either side of the
+//      expected rank.  (Rows of at most 2048 keys are sampled completely, which settles the threshold
+//      at once.)
+//   2. Window pass: one sweep over the row counts the keys above a window of codes bracketed by two
+//      order statistics of the sample and builds a 2048-bin histogram of the keys inside it.  A window
+//      of at most 2048 codes gives the 16-bit threshold T exactly; a wider one is narrowed to the bin
+//      that holds T and swept once more.  If the bracket misses (rare) the sweep is repeated on the
+//      codes above or below it.
+//   3. Emission: one more sweep sets the mask bits of the keys above T (eight keys per thread, four
+//      threads per mask word) and collects the keys equal to T.  Those round to the same half-
+//      precision value, so their order is settled exactly: their logits are recomputed in fp32 from Q
+//      and K and ranked by (value descending, index ascending); the first k - #above are selected.
+// Sweeps skip 8-key vectors that hold nothing at or above the level of interest with a handful of
+// instructions, so a sparse selection costs about one instruction per key and sweep.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace gvote {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kTieCap = 1024;
+constexpr int kThreads = 128;
+constexpr int kWin = 2048;              // codes per histogram window
+constexpr int kTieCap = 512;
+constexpr int kSampleVecs = 256;        // sample = 256 vectors of 8 consecutive keys
 constexpr int kTileKeys = 128;
+constexpr int kLoads = 4;               // 16-byte loads in flight per thread
+constexpr uint32_t kPadKey = 0xfc00u;   // -inf: what positions past the end of a row read as
+constexpr uint32_t kMinCode = 0x0400u;  // code of the most negative finite half: no key lies below it
+
+// Half bits -> code whose unsigned order is the numeric order (-0 and +0 share a code), and back.
+__device__ __forceinline__ uint32_t code_of(uint32_t h) {
+  if (h == 0x8000u) h = 0u;
+  return (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+}
+__device__ __forceinline__ uint32_t raw_of(uint32_t c) { return (c & 0x8000u) ? (c & 0x7fffu) : (~c & 0xffffu); }
+__device__ __forceinline__ __half2 pair_of(uint32_t raw) {
+  const uint32_t p = raw | (raw << 16);
+  return *reinterpret_cast<const __half2*>(&p);
+}
+__device__ __forceinline__ __half2 as_h2(uint32_t w) { return *reinterpret_cast<const __half2*>(&w); }
+// No key has code 0x7fff (it is -0's slot), and as a bound it would turn into -0, which compares
+// equal to +0: bounds step over it.
+__device__ __forceinline__ uint32_t fix_lo(uint32_t c) { return c == 0x7fffu ? 0x8000u : c; }
+__device__ __forceinline__ uint32_t fix_hi(uint32_t c) { return c == 0x7fffu ? 0x7ffeu : c; }
 
 struct Sel16Shared {
-  uint32_t hist[256];
+  uint32_t hist[kWin];
   float qf[512];
   int tie_idx[kTieCap];
   float tie_val[kTieCap];
-  uint32_t red32[kThreads / 32];
+  uint32_t red[kThreads / 32];
   int bin;
   uint32_t above;
+  uint32_t inside;
   uint32_t ntie;
 };
+
+__device__ __forceinline__ uint32_t block_sum(Sel16Shared& sh, uint32_t v) {
+  v = (uint32_t)warp_sum_i((int)v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  uint32_t s = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) s += sh.red[w];
+  return s;
+}
 
 // Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need).
 __device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
@@ -64,6 +104,49 @@ __device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
   __syncthreads();
 }
 
+// The rank-th largest code (rank >= 1, at most the number of sampled keys) among the sampled vectors
+// (two per thread, `have` of them real), by a two-level 256-bin histogram.  Also returns how many
+// sampled codes lie above it and how many equal it.  Every thread of the CTA calls it.
+__device__ uint32_t sample_kth(Sel16Shared& sh, const uint4 (&sv)[2], int have, uint32_t rank, uint32_t& above,
+                               uint32_t& equal) {
+  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    if (i >= have) break;
+    const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      atomicAdd(&sh.hist[code_of(w[j] & 0xffffu) >> 8], 1u);
+      atomicAdd(&sh.hist[code_of(w[j] >> 16) >> 8], 1u);
+    }
+  }
+  __syncthreads();
+  find_bin256(sh, rank);
+  const uint32_t b_hi = (uint32_t)sh.bin, above_hi = sh.above;
+  __syncthreads();
+  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    if (i >= have) break;
+    const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t c0 = code_of(w[j] & 0xffffu), c1 = code_of(w[j] >> 16);
+      if ((c0 >> 8) == b_hi) atomicAdd(&sh.hist[c0 & 255u], 1u);
+      if ((c1 >> 8) == b_hi) atomicAdd(&sh.hist[c1 & 255u], 1u);
+    }
+  }
+  __syncthreads();
+  find_bin256(sh, rank - above_hi);
+  const uint32_t t = (b_hi << 8) | (uint32_t)sh.bin;
+  above = above_hi + sh.above;
+  equal = sh.hist[sh.bin];
+  __syncthreads();
+  return t;
+}
+
 // Exact fp32 logit of key n for this row's query (fixed summation order).
 struct DotCtx {
   const float* qf;
@@ -89,161 +172,265 @@ struct DotCtx {
 };
 
 // Where a row's keys live: eight consecutive keys form one 16-byte vector; vector v8 of the row
-// sits in tile v8 / 16 at offset (v8 % 16) * 8.  Keys at positions >= N are read as 0 (below any
-// real key, whose image is never 0).
+// sits in tile v8 / 16 at offset (v8 % 16) * 8.  Positions >= N read as -inf.
 struct RowView {
-  const uint16_t* smem_row;     // non-null when the row is resident in shared memory
   const uint16_t* grow;         // first tile of the row in global memory
   int64_t tile_stride;          // elements between consecutive tiles of the same row
-  int N;
-  __device__ __forceinline__ uint4 mask_tail(uint4 v, int v8) const {
+  int N, nv8;
+  __device__ __forceinline__ uint4 load(int v8) const {
+    if (v8 >= nv8) return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u);
+    uint4 v = *reinterpret_cast<const uint4*>(grow + (int64_t)(v8 >> 4) * tile_stride + (v8 & 15) * 8);
     if (v8 * 8 + 8 > N) {
       uint16_t* e = reinterpret_cast<uint16_t*>(&v);
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (v8 * 8 + j >= N) e[j] = 0;
+        if (v8 * 8 + j >= N) e[j] = (uint16_t)kPadKey;
     }
     return v;
   }
-  __device__ __forceinline__ uint4 load_global(int v8) const {
-    const uint4 v = *reinterpret_cast<const uint4*>(grow + (int64_t)(v8 >> 4) * tile_stride + (v8 & 15) * 8);
-    return mask_tail(v, v8);
-  }
-  __device__ __forceinline__ uint4 load(int v8) const {
-    if (smem_row) return *reinterpret_cast<const uint4*>(smem_row + (size_t)v8 * 8);
-    return load_global(v8);
-  }
   __device__ __forceinline__ uint32_t key_at(int n) const {
-    if (smem_row) return smem_row[n];
     return grow[(int64_t)(n >> 7) * tile_stride + (n & 127)];
   }
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+// One sweep: A = number of keys with code > hi; hist[(c - lo) >> shift] = number of keys with code c
+// in [lo, hi] ((hi - lo) >> shift < kWin).  Neither bound is 0x7fff.
+__device__ uint32_t window_pass(const RowView& rv, uint32_t lo, uint32_t hi, int shift, Sel16Shared& sh) {
+  for (int b = threadIdx.x; b < kWin; b += kThreads) sh.hist[b] = 0;
+  __syncthreads();
+  const __half2 tlo = pair_of(raw_of(lo)), thi = pair_of(raw_of(hi));
+  uint32_t a16 = 0;   // 16 per key above the window
+  for (int base = 0; base < rv.nv8; base += kThreads * kLoads) {
+    uint4 buf[kLoads];
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) buf[u] = rv.load(base + u * kThreads + (int)threadIdx.x);
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const uint32_t w[4] = {buf[u].x, buf[u].y, buf[u].z, buf[u].w};
+      uint32_t ge[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ge[j] = __hge2_mask(as_h2(w[j]), tlo);
+      if ((ge[0] | ge[1] | ge[2] | ge[3]) == 0u) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t gt = __hgt2_mask(as_h2(w[j]), thi);
+        a16 += __popc(gt);
+        const uint32_t in = ge[j] & ~gt;
+        if (in & 0xffffu) {
+          const uint32_t b = (code_of(w[j] & 0xffffu) - lo) >> shift;
+          if (b < (uint32_t)kWin) atomicAdd(&sh.hist[b], 1u);
+        }
+        if (in >> 16) {
+          const uint32_t b = (code_of(w[j] >> 16) - lo) >> shift;
+          if (b < (uint32_t)kWin) atomicAdd(&sh.hist[b], 1u);
+        }
+      }
+    }
+  }
+  return block_sum(sh, a16 >> 4);    // (its barriers also publish the histogram)
+}
+
+// Largest window bin whose suffix count reaches `need`; publishes sh.bin, sh.above (count in the
+// bins above it) and sh.inside (count in the whole window).  If the window holds fewer than `need`
+// keys, sh.bin = -1.  Thread t owns the 16 bins below kWin - 16 t.
+__device__ void window_find(Sel16Shared& sh, uint32_t need) {
+  constexpr int kPer = kWin / kThreads;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int top = kWin - 1 - tid * kPer;
+  uint32_t own = 0;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) own += sh.hist[top - i];
+  uint32_t inc = own;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) sh.red[warp] = inc;
+  if (tid == 0) { sh.bin = -1; sh.above = 0; }
+  __syncthreads();
+  uint32_t before = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    if (w < warp) before += sh.red[w];
+    total += sh.red[w];
+  }
+  const uint32_t excl = before + inc - own;
+  if (excl < need && excl + own >= need) {
+    uint32_t a = excl;
+    int b = top;
+    for (; b > top - kPer + 1; --b) {
+      if (a + sh.hist[b] >= need) break;
+      a += sh.hist[b];
+    }
+    sh.bin = b;
+    sh.above = a;
+  }
+  if (tid == 0) sh.inside = total;
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads, 8)
 topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __restrict__ Q,
                    const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int RC, int row_chunks,
                    int64_t n_tiles_total, float scale, const int32_t* __restrict__ b_step, int64_t row_words,
-                   uint32_t* __restrict__ mask, int row_elems) {
-  extern __shared__ __align__(16) uint8_t dyn_smem[];
+                   uint32_t* __restrict__ mask) {
   __shared__ Sel16Shared sh;
-  uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn_smem);                     // [256][32]
-  uint16_t* row_sm = reinterpret_cast<uint16_t*>(dyn_smem + 256 * 32 * 4);     // [row_elems]
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int start = cu[r], N = cu[r + 1] - start;
   if (N <= 0) return;
-  int k = b_step[r * Hq + g];
+  const int k = b_step[r * Hq + g];
   if (k <= 0) return;
-  if (k > N) k = N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int kh = g / G;
   const int grow_idx = (g % G) * S + s;                  // row within the head group (synthetic rows come first)
   const int chunk = grow_idx / RC, crow = grow_idx % RC;
   RowView rv;
   rv.N = N;
+  rv.nv8 = (N + 7) >> 3;
   rv.tile_stride = (int64_t)row_chunks * RC * kTileKeys;
   rv.grow = keys16 + ((((int64_t)kh * n_tiles_total + tile_offset(start, r)) * row_chunks + chunk) * RC + crow) * kTileKeys;
-  const bool fits = N <= row_elems;
-  rv.smem_row = fits ? row_sm : nullptr;
   uint32_t* mrow = mask + (int64_t)kh * row_words + mask_word_offset(start, r);
-  const int nv8 = (N + 7) >> 3;
+  const int words = (N + 31) >> 5;
 
+  if (k >= N) {                                          // every key is selected
+    for (int w = tid; w < words; w += kThreads) {
+      const uint32_t v = (w == words - 1 && (N & 31)) ? ((1u << (N & 31)) - 1u) : 0xffffffffu;
+      atomicOr(&mrow[w], v);
+    }
+    return;
+  }
   {
     const __nv_bfloat16* qrow = Q + (((int64_t)r * (Hq / G) + kh) * (G * (S + 1)) + grow_idx) * d_k;
     for (int i = tid; i < d_k; i += kThreads) sh.qf[i] = __bfloat162float(qrow[i]);
-    for (int i = tid; i < 256 * 32; i += kThreads) hist1[i] = 0;
     if (tid == 0) sh.ntie = 0;
   }
-  __syncthreads();
 
-  // A. load the row, count high bytes (one counter per bin and lane)
-  // (eight 16-byte loads are put in flight before any of them is consumed)
-  for (int base = 0; base < nv8; base += kThreads * 8) {
-    uint4 buf[8];
+  // ---------------------------------------------------------------- 1. sample
+  uint32_t T = 0, above = 0, eq = 0;
+  bool found = false;
+  uint32_t lo, hi = 0xffffu;
+  {
+    uint4 sv[2];
+    int have = 0;
+    const bool whole = rv.nv8 <= kSampleVecs;
+    const int stride8 = whole ? 1 : rv.nv8 / kSampleVecs;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int v8 = base + u * kThreads + tid;
-      buf[u] = (v8 < nv8) ? rv.load_global(v8) : make_uint4(0u, 0u, 0u, 0u);
+    for (int i = 0; i < 2; ++i) {
+      const int j = tid + i * kThreads;
+      const int v8 = whole ? j : j * stride8 + (stride8 >> 1);
+      sv[i] = rv.load(v8);                                // vectors past the row read as -inf
+      if (v8 < rv.nv8) have = i + 1;
     }
+    if (whole) {
+      // the whole row is in the sample: its k-th largest code is the threshold
+      T = sample_kth(sh, sv, have, (uint32_t)k, above, eq);
+      found = true;
+      lo = T;
+    } else {
+      // bracket the k-th largest key between two order statistics of the sample, a few standard
+      // deviations of the sampling error either side of the expected rank
+      const float m_s = (float)(kSampleVecs * 8);
+      const float rk = (float)k * m_s / (float)N;
+      const float dlt = 4.5f * sqrtf(rk) + 6.0f;
+      int r_lo = (int)ceilf(rk + dlt);
+      if (r_lo > kSampleVecs * 8) r_lo = kSampleVecs * 8;
+      const int r_hi = (int)floorf(rk - dlt);
+      uint32_t a_s, e_s;
+      lo = sample_kth(sh, sv, 2, (uint32_t)r_lo, a_s, e_s);
+      hi = r_hi >= 1 ? sample_kth(sh, sv, 2, (uint32_t)r_hi, a_s, e_s) : 0xffffu;
+    }
+  }
+
+  // ---------------------------------------------------------------- 2. window passes
+  // A window is [lo, hi] in code space, histogrammed in 2048 bins of 2^shift codes.  A window wider
+  // than 2048 codes is narrowed to the bin that holds the threshold and swept again; a bracket that
+  // turns out wrong (rare) is replaced by everything above or below it.
+  if (!found) {
+    if (lo < kMinCode) lo = kMinCode;
+    if (hi < lo) hi = lo;
+    lo = fix_lo(lo);
+    hi = fix_hi(hi);
+    for (int iter = 0; iter < 12; ++iter) {
+      int shift = 0;
+      while (((hi - lo) >> shift) >= (uint32_t)kWin) ++shift;
+      const uint32_t A = window_pass(rv, lo, hi, shift, sh);
+      if (A >= (uint32_t)k) {                             // the threshold lies above the window
+        lo = fix_lo(hi + 1u);
+        hi = 0xffffu;
+        continue;
+      }
+      window_find(sh, (uint32_t)k - A);
+      const int bin = sh.bin;
+      if (bin < 0) {                                      // the threshold lies below the window
+        if (lo <= kMinCode) break;                        // cannot happen: k < N keys lie at or above kMinCode
+        hi = fix_hi(lo - 1u);
+        lo = kMinCode;
+        __syncthreads();
+        continue;
+      }
+      if (shift == 0) {
+        T = lo + (uint32_t)bin;
+        above = A + sh.above;
+        eq = sh.hist[bin];
+        found = true;
+        break;
+      }
+      const uint32_t nlo = lo + ((uint32_t)bin << shift);
+      const uint32_t nhi = min(nlo + (1u << shift) - 1u, hi);
+      lo = fix_lo(nlo);
+      hi = fix_hi(nhi);
+      __syncthreads();
+    }
+    __syncthreads();
+    if (!found) return;
+  }
+  const uint32_t ties = (uint32_t)k - above;              // 1 <= ties <= eq
+  const bool all_ties = ties >= eq;
+
+  // ---------------------------------------------------------------- 3. emission
+  {
+    const __half2 tt = pair_of(raw_of(T));
+    for (int base = 0; base < rv.nv8; base += kThreads * kLoads) {
+      uint4 buf[kLoads];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int v8 = base + u * kThreads + tid;
-      if (v8 < nv8) {
-        if (fits) *reinterpret_cast<uint4*>(row_sm + (size_t)v8 * 8) = buf[u];
+      for (int u = 0; u < kLoads; ++u) buf[u] = rv.load(base + u * kThreads + tid);
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int v8 = base + u * kThreads + tid;
         const uint32_t w[4] = {buf[u].x, buf[u].y, buf[u].z, buf[u].w};
+        uint32_t ge[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ge[j] = __hge2_mask(as_h2(w[j]), tt);
+        if (!__any_sync(0xffffffffu, (ge[0] | ge[1] | ge[2] | ge[3]) != 0u)) continue;   // warp-uniform skip
+        // bit 2j of the low half and bit 2j+1 of the high half of word j mark its two keys
+        uint32_t gacc = 0, eacc = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          atomicAdd(&hist1[((w[j] >> 8) & 255u) * 32 + lane], 1u);
-          atomicAdd(&hist1[(w[j] >> 24) * 32 + lane], 1u);
+          const uint32_t pick = (1u << (2 * j)) | (1u << (17 + 2 * j));
+          const uint32_t gt = __hgt2_mask(as_h2(w[j]), tt);
+          gacc |= gt & pick;
+          eacc |= (ge[j] & ~gt) & pick;
         }
+        uint32_t bits = (gacc | (gacc >> 16)) & 0xffu;
+        uint32_t eqbits = (eacc | (eacc >> 16)) & 0xffu;
+        if (all_ties) bits |= eqbits;
+        else {
+          while (eqbits) {
+            const int j = __ffs(eqbits) - 1;
+            eqbits &= eqbits - 1;
+            const uint32_t slot = atomicAdd(&sh.ntie, 1u);
+            if (slot < (uint32_t)kTieCap) sh.tie_idx[slot] = v8 * 8 + j;
+          }
+        }
+        uint32_t word = bits << (8 * (lane & 3));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        if ((lane & 3) == 0 && word) atomicOr(&mrow[v8 >> 2], word);
       }
     }
-  }
-  __syncthreads();
-  // B. reduce over lanes (rotated read: conflict free); the padding keys (0) sit in bin 0
-  {
-    uint32_t c = 0;
-#pragma unroll 8
-    for (int j = 0; j < 32; ++j) c += hist1[tid * 32 + ((j + tid) & 31)];
-    if (tid == 0) c -= (uint32_t)(nv8 * 8 - N);
-    sh.hist[tid] = c;
-  }
-  __syncthreads();
-  find_bin256(sh, (uint32_t)k);
-  const uint32_t b_hi = (uint32_t)sh.bin;
-  uint32_t above = sh.above;
-  __syncthreads();
-  sh.hist[tid] = 0;
-  __syncthreads();
-  // C. low bytes of the keys whose high byte is b_hi
-  for (int v8 = tid; v8 < nv8; v8 += kThreads) {
-    const uint4 v = rv.load(v8);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (((w[j] >> 8) & 255u) == b_hi && (v8 * 8 + 2 * j) < N) atomicAdd(&sh.hist[w[j] & 255u], 1u);
-      if ((w[j] >> 24) == b_hi && (v8 * 8 + 2 * j + 1) < N) atomicAdd(&sh.hist[(w[j] >> 16) & 255u], 1u);
-    }
-  }
-  __syncthreads();
-  find_bin256(sh, (uint32_t)k - above);
-  const uint32_t T = (b_hi << 8) | (uint32_t)sh.bin;
-  above += sh.above;
-  const uint32_t eq = sh.hist[sh.bin];
-  const uint32_t ties = (uint32_t)k - above;        // 1 <= ties <= eq
-  __syncthreads();
-
-  // D. emit: 8 keys per thread, 4 threads per mask word; collect the keys equal to T
-  const bool all_ties = ties >= eq;
-  for (int base = 0; base < nv8; base += kThreads) {
-    const int v8 = base + tid;
-    uint32_t bits = 0, eqbits = 0;
-    if (v8 < nv8) {
-      const uint4 v = rv.load(v8);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
-        bits |= (lo > T ? 1u : 0u) << (2 * j);
-        bits |= (hi > T ? 1u : 0u) << (2 * j + 1);
-        eqbits |= (lo == T ? 1u : 0u) << (2 * j);
-        eqbits |= (hi == T ? 1u : 0u) << (2 * j + 1);
-      }
-      if (T == 0) eqbits &= (v8 * 8 + 8 > N) ? ((1u << (N - v8 * 8)) - 1u) : 0xffu;   // padding is not a key
-    }
-    if (all_ties) bits |= eqbits;
-    else {
-      while (eqbits) {
-        const int j = __ffs(eqbits) - 1;
-        eqbits &= eqbits - 1;
-        const uint32_t slot = atomicAdd(&sh.ntie, 1u);
-        if (slot < (uint32_t)kTieCap) sh.tie_idx[slot] = v8 * 8 + j;
-      }
-    }
-    uint32_t word = bits << (8 * (lane & 3));
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    if ((lane & 3) == 0 && word) atomicOr(&mrow[v8 >> 2], word);
   }
   if (all_ties) return;
   __syncthreads();
@@ -271,10 +458,10 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   uint32_t prefix = 0, known = 0, acc = 0, eq2 = 0;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    sh.hist[tid] = 0;
+    for (int b = tid; b < 256; b += kThreads) sh.hist[b] = 0;
     __syncthreads();
     for (int n = tid; n < N; n += kThreads) {
-      if (rv.key_at(n) == T) {
+      if (code_of(rv.key_at(n)) == T) {
         const uint32_t key = ordered_key(dot(n));
         if ((key & known) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
       }
@@ -289,9 +476,10 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   }
   const uint32_t ties2 = ties - acc;
   uint32_t taken = 0;
+  const int warp = tid >> 5;
   for (int base = 0; base < N; base += kThreads) {
     const int n = base + tid;
-    const bool member = n < N && rv.key_at(n) == T;
+    const bool member = n < N && code_of(rv.key_at(n)) == T;
     const uint32_t key = member ? ordered_key(dot(n)) : 0u;
     bool sel = member && key > prefix;
     const bool tie = member && key == prefix;
@@ -299,16 +487,16 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
       sel |= tie;
     } else {
       const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-      if (lane == 0) sh.red32[warp] = __popc(tb);
+      __syncthreads();
+      if (lane == 0) sh.red[warp] = __popc(tb);
       __syncthreads();
       uint32_t before = taken, total = 0;
       for (int w = 0; w < kThreads / 32; ++w) {
-        if (w < warp) before += sh.red32[w];
-        total += sh.red32[w];
+        if (w < warp) before += sh.red[w];
+        total += sh.red[w];
       }
       sel |= tie && (before + __popc(tb & ((1u << lane) - 1u))) < ties2;
       taken += total;
-      __syncthreads();
     }
     const uint32_t bal = __ballot_sync(0xffffffffu, sel);
     if (lane == 0 && bal) atomicOr(&mrow[n >> 5], bal);
@@ -322,19 +510,13 @@ int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_
                       int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   const ScoreGeometry geo = score_geometry(p);
-  // rows up to 80K keys stay resident in shared memory next to the 32 KB histogram; longer rows
-  // are streamed from global memory in each pass
-  int row_elems = (int)((max_N + 127) & ~(int64_t)127);
-  if (row_elems > 80 * 1024) row_elems = 0;
-  const size_t smem = 256 * 32 * 4 + (size_t)row_elems * sizeof(uint16_t);
-  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topk16_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(p->S, Hq, batch);
   const float scale = (float)(1.0 / sqrt((double)p->d_k));
   {
     LaunchScope scope_("topk16_rows_kernel", st);
-    topk16_rows_kernel<<<grid, kThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
-                                                     geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
-                                                     row_words, mask, row_elems);
+    topk16_rows_kernel<<<grid, kThreads, 0, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
+                                                  geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
+                                                  row_words, mask);
   }
   GVOTE_LAUNCH_CHECK("topk16_rows_kernel");
   return GVOTE_OK;
