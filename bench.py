@@ -141,6 +141,7 @@ def flops(cfg):
 
 STAGE_OF = {
     "fit_partial_kernel": "fit", "fit_finalize_kernel": "fit", "sample_kernel": "sample",
+    "prep_kernel": "sample", "real_hist_kernel": "vote", "real_resolve_kernel": "vote", "topk16_rows_kernel": "vote",
     "xstage_kernel": "project", "rope_table_kernel": "project", "project_simt_kernel": "project",
     "project_umma_kernel": "project", "project_finish_kernel": "project",
     "score_simt_kernel": "vote", "score_umma_kernel": "vote", "topp_rows_kernel": "vote",
@@ -195,7 +196,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
-    ap.add_argument("--streams", type=int, default=1,
+    ap.add_argument("--streams", type=int, default=4,
                     help="CUDA streams the layers of a step are spread over (each with its own workspace)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
@@ -232,7 +233,8 @@ def main():
         args.warmup = 3
 
     # weak scaling: every rank compresses its own requests (same shapes, its own seed)
-    cfg = synth.make_config(args.workload, seed=base_cfg.seed + 1000 * rank, **over)
+    from paper_2509_03136_b200 import shard
+    cfg = shard.rank_workload(base_cfg, rank)
     L = cfg.n_layers
     geom = (cfg.batch, cfg.total_tokens, max(cfg.seq_lens))
     workers = max(1, min(len(os.sched_getaffinity(0)) // max(world, 1), 16))
@@ -262,21 +264,23 @@ def main():
         for l in range(L):
             d_K[l].copy_(d_K0[l]); d_V[l].copy_(d_V0[l])
 
-    def one_pass():
+    def one_pass(spread=True):
         # layers are independent (Section 3.2): layer l goes to stream l mod n_streams, so the short,
         # latency-bound kernels of one layer run under the streaming kernels of another
         main = torch.cuda.current_stream()
-        if side:
+        side_now = side if spread else []
+        ns = len(side_now) + 1
+        if side_now:
             fork = torch.cuda.Event()
             fork.record(main)
-            for st in side:
+            for st in side_now:
                 st.wait_event(fork)
         for l in range(L):
-            k = l % n_streams
-            with torch.cuda.stream(main if k == 0 else side[k - 1]):
+            k = l % ns
+            with torch.cuda.stream(main if k == 0 else side_now[k - 1]):
                 gv.gvote_compress(p_layer[l], d_h[l], d_W[l], None, d_K[l], d_V[l], cu, geom, d_mask[l], d_budget[l],
                                   d_bstep[l], ws_s[k])
-        for st in side:
+        for st in side_now:
             join = torch.cuda.Event()
             join.record(st)
             main.wait_event(join)
@@ -289,13 +293,13 @@ def main():
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def timed_steps(n):
+    def timed_steps(n, spread=True):
         total_ms = 0.0
         for _ in range(n):
             restore()
             barrier()
             ev0.record()
-            one_pass()
+            one_pass(spread)
             ev1.record()
             torch.cuda.synchronize()
             total_ms += ev0.elapsed_time(ev1)
@@ -313,16 +317,14 @@ def main():
     launches = gv.gvote_launch_count() - n0
     for w in ws_s:
         assert gv.gvote_poll_status(w) == 0, "a device-side wait timed out"
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = shard.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * cfg.total_tokens / (ms_per_step * 1e-3)
+    value = shard.job_throughput(cfg.total_tokens, world, ms_per_step * 1e-3)
 
     # ---- per-kernel timing: the same steps again with an event pair around every launch
+    # (on one stream, so that every event pair brackets one kernel running alone)
     gv.gvote_profile_enable(True)
-    timed_steps(args.steps)
+    serial_ms = timed_steps(args.steps, spread=False) / args.steps
     prof = gv.gvote_profile_report()
     gv.gvote_profile_enable(False)
     # clock samples cover the warm-up, the timed steps and their event-instrumented repeat (same work)
@@ -364,6 +366,7 @@ def main():
     sel_s = (stage_us.get("project", 0) + stage_us.get("vote", 0) + stage_us.get("compact", 0)) * 1e-6
     pass_roofline = {
         "kept_fraction": kept_frac, "per_layer_us": layer_s * 1e6, "stage_us_per_layer": stage_us,
+        "per_layer_us_one_stream_instrumented": serial_ms * 1e3 / L,
         "full_bytes_roofline_us": full_t * 1e6, "full_bytes_frac": full_t / layer_s,
         "literal_roofline_us": lit_t * 1e6, "literal_frac_whole_pass": lit_t / layer_s,
         "literal_frac_select_compact_only": (lit_t / sel_s) if sel_s > 0 else None,
@@ -395,10 +398,7 @@ def main():
             dt = time.perf_counter() - t0
             if s >= 1:
                 e2e_total += dt
-        if dist is not None:
-            t = torch.tensor([e2e_total], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_total = float(t.item())
+        e2e_total = shard.max_over_ranks(e2e_total, dist, dev)
         gv.gvote_host_arena_release()
         h2d = sum(a.numel() * a.element_size() for l in range(L) for a in (hh[l], hW[l], hK[l], hV[l])) + L * hcu.numel() * 4
         d2h = sum(a.numel() * a.element_size() for l in range(L) for a in (hK[l], hV[l], hmask[l], hbud[l], hbs[l]))
