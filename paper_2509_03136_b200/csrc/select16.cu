@@ -4,21 +4,22 @@
 //
 // One small CTA per synthetic row, many resident per SM.  Keys are compared as half-precision numbers,
 // two per instruction; for counting they are mapped to an order-preserving 16-bit code.
-//   1. A fixed, evenly spaced sample of 2048 keys brackets the k-th largest key between two of the
-//      sample's order statistics, a few standard deviations of the sampling error either side of the
-//      expected rank.  (Rows of at most 2048 keys are sampled completely, which settles the threshold
-//      at once.)
-//   2. Window pass: one sweep over the row counts the keys above a window of codes bracketed by two
-//      order statistics of the sample and builds a 2048-bin histogram of the keys inside it.  A window
-//      of at most 2048 codes gives the 16-bit threshold T exactly; a wider one is narrowed to the bin
-//      that holds T and swept once more.  If the bracket misses (rare) the sweep is repeated on the
-//      codes above or below it.
-//   3. Emission: one more sweep sets the mask bits of the keys above T (eight keys per thread, four
-//      threads per mask word) and collects the keys equal to T.  Those round to the same half-
-//      precision value, so their order is settled exactly: their logits are recomputed in fp32 from Q
-//      and K and ranked by (value descending, index ascending); the first k - #above are selected.
-// Sweeps skip 8-key vectors that hold nothing at or above the level of interest with a handful of
-// instructions, so a sparse selection costs about one instruction per key and sweep.
+//   1. A fixed, evenly spaced sample of 4096 keys brackets the k-th largest key between two of
+//      the sample's order statistics, a few standard deviations of the sampling error either side of
+//      the expected rank.  (Rows of at most 4096 keys are sampled completely, which settles the
+//      threshold at once.)
+//   2. One sweep over the row marks, in a shared-memory bit row, every key above the bracket, counts
+//      them, and lists the keys inside the bracket (every thread in a list of its own).  If the bracket holds (#above <= k <= #above +
+//      #listed, and the list fits), the k - #above largest listed keys are found inside the list with
+//      a two-level histogram and marked too; the bit row is then OR-ed into the mask.
+//   3. Keys that share the 16-bit threshold value T round to the same half-precision number, so their
+//      order is settled exactly: their logits are recomputed in fp32 from Q and K and ranked by (value
+//      descending, index ascending); the first k - #above-T of them are selected.
+//   4. If the bracket misses or the list overflows (rare), nothing has been written yet and the row
+//      takes the slower exact route: window sweeps that count the keys above a window of codes and
+//      histogram the keys inside it in 2048 bins (a window wider than 2048 codes is narrowed to the
+//      bin that holds T and swept again), then an emission sweep.
+// Sweeps test eight keys with four compare instructions and skip vectors with nothing of interest.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -28,8 +29,9 @@ namespace {
 
 constexpr int kThreads = 128;
 constexpr int kWin = 2048;              // codes per histogram window
-constexpr int kTieCap = 512;
-constexpr int kSampleVecs = 256;        // sample = 256 vectors of 8 consecutive keys
+constexpr int kTieCap = 256;
+constexpr int kOvfCap = 384;            // bracket keys that did not fit their thread's list
+constexpr int kSampleRound = kThreads * 4;   // sample vectors per round (four per thread): at least one round
 constexpr int kTileKeys = 128;
 constexpr int kLoads = 4;               // 16-byte loads in flight per thread
 constexpr uint32_t kPadKey = 0xfc00u;   // -inf: what positions past the end of a row read as
@@ -53,7 +55,7 @@ __device__ __forceinline__ uint32_t fix_hi(uint32_t c) { return c == 0x7fffu ? 0
 
 struct Sel16Shared {
   uint32_t hist[kWin];
-  float qf[512];
+  __nv_bfloat16 qf[512];
   int tie_idx[kTieCap];
   float tie_val[kTieCap];
   uint32_t red[kThreads / 32];
@@ -61,6 +63,9 @@ struct Sel16Shared {
   uint32_t above;
   uint32_t inside;
   uint32_t ntie;
+  uint32_t novf;
+  uint32_t ovf_n[kOvfCap];
+  uint16_t ovf_key[kOvfCap];
 };
 
 __device__ __forceinline__ uint32_t block_sum(Sel16Shared& sh, uint32_t v) {
@@ -104,52 +109,16 @@ __device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
   __syncthreads();
 }
 
-// The rank-th largest code (rank >= 1, at most the number of sampled keys) among the sampled vectors
-// (two per thread, `have` of them real), by a two-level 256-bin histogram.  Also returns how many
-// sampled codes lie above it and how many equal it.  Every thread of the CTA calls it.
-__device__ uint32_t sample_kth(Sel16Shared& sh, const uint4 (&sv)[2], int have, uint32_t rank, uint32_t& above,
-                               uint32_t& equal) {
-  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    if (i >= have) break;
-    const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      atomicAdd(&sh.hist[code_of(w[j] & 0xffffu) >> 8], 1u);
-      atomicAdd(&sh.hist[code_of(w[j] >> 16) >> 8], 1u);
-    }
-  }
-  __syncthreads();
-  find_bin256(sh, rank);
-  const uint32_t b_hi = (uint32_t)sh.bin, above_hi = sh.above;
-  __syncthreads();
-  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    if (i >= have) break;
-    const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t c0 = code_of(w[j] & 0xffffu), c1 = code_of(w[j] >> 16);
-      if ((c0 >> 8) == b_hi) atomicAdd(&sh.hist[c0 & 255u], 1u);
-      if ((c1 >> 8) == b_hi) atomicAdd(&sh.hist[c1 & 255u], 1u);
-    }
-  }
-  __syncthreads();
-  find_bin256(sh, rank - above_hi);
-  const uint32_t t = (b_hi << 8) | (uint32_t)sh.bin;
-  above = above_hi + sh.above;
-  equal = sh.hist[sh.bin];
-  __syncthreads();
-  return t;
-}
+// The sample: vector i of `n_vecs` (at most four per thread) is vector i * stride + stride / 2 of the
+// row (stride 1 samples the whole row).
+struct Sample {
+  int n_vecs, stride;
+  __device__ __forceinline__ int vec(int i) const { return i * stride + (stride >> 1); }
+};
 
 // Exact fp32 logit of key n for this row's query (fixed summation order).
 struct DotCtx {
-  const float* qf;
+  const __nv_bfloat16* qf;
   const __nv_bfloat16* krows;   // K + head offset + request start
   int64_t k_tok;
   int d_k;
@@ -163,8 +132,9 @@ struct DotCtx {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float2 f = __bfloat1622float2(h[j]);
-        acc = fmaf(qf[c * 8 + 2 * j], f.x, acc);
-        acc = fmaf(qf[c * 8 + 2 * j + 1], f.y, acc);
+        const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qf + c * 8 + 2 * j));
+        acc = fmaf(q.x, f.x, acc);
+        acc = fmaf(q.y, f.y, acc);
       }
     }
     return acc * scale;
@@ -192,6 +162,90 @@ struct RowView {
     return grow[(int64_t)(n >> 7) * tile_stride + (n & 127)];
   }
 };
+
+// 256-bin histogram (left in sh.hist[0..256)) of the sampled codes' high bytes (level 1), or of the low
+// bytes of the sampled codes whose high byte is `only` (level 2).
+// Level 1 sees every sampled key and a few bins take most of them, so plain shared-memory atomics
+// would serialise on those addresses.  It counts into one 8-bit counter per (bin, lane) instead, four
+// bins to a word, word index (bin / 4) * 32 + lane: the lanes of a warp never meet, and a counter
+// takes at most (warps) * (sample keys per thread) = 4 * 32 increments, well below 256.
+template <bool LEVEL2>
+__device__ void sample_hist(const RowView& rv, const Sample& sm, uint32_t only, Sel16Shared& sh) {
+  const int lane = threadIdx.x & 31;
+  for (int b = threadIdx.x; b < (LEVEL2 ? 256 : kWin); b += kThreads) sh.hist[b] = 0;
+  __syncthreads();
+  {
+    uint4 sv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = u * kThreads + (int)threadIdx.x;
+      sv[u] = i < sm.n_vecs ? rv.load(sm.vec(i)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (u * kThreads + (int)threadIdx.x >= sm.n_vecs) continue;
+      const uint32_t w[4] = {sv[u].x, sv[u].y, sv[u].z, sv[u].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t c0 = code_of(w[j] & 0xffffu), c1 = code_of(w[j] >> 16);
+        if (!LEVEL2) {
+          atomicAdd(&sh.hist[(c0 >> 10) * 32 + lane], 1u << ((c0 >> 5) & 24u));
+          atomicAdd(&sh.hist[(c1 >> 10) * 32 + lane], 1u << ((c1 >> 5) & 24u));
+        } else {
+          if ((c0 >> 8) == only) atomicAdd(&sh.hist[c0 & 255u], 1u);
+          if ((c1 >> 8) == only) atomicAdd(&sh.hist[c1 & 255u], 1u);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (!LEVEL2) {
+    // fold the lanes: thread t sums bins 2t and 2t+1
+    uint32_t tot[2] = {0u, 0u};
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int bin = 2 * (int)threadIdx.x + q;
+      const uint32_t* wrow = &sh.hist[(bin >> 2) * 32];
+      const int sh8 = (bin & 3) * 8;
+      for (int l = 0; l < 32; ++l) tot[q] += (wrow[(l + lane) & 31] >> sh8) & 255u;   // rotated: conflict free
+    }
+    __syncthreads();
+    sh.hist[2 * threadIdx.x] = tot[0];
+    sh.hist[2 * threadIdx.x + 1] = tot[1];
+    __syncthreads();
+  }
+}
+
+// The sample's rank_a-th and rank_b-th largest codes (1 <= rank_a <= rank_b <= sampled keys; rank_a = 0
+// asks for the second one only).  For the second one also the number of sampled codes above it and
+// equal to it.  Every thread of the CTA calls it.
+__device__ void sample_ranks(const RowView& rv, const Sample& sm, uint32_t rank_a, uint32_t rank_b, Sel16Shared& sh,
+                             uint32_t& code_a, uint32_t& code_b, uint32_t& above_b, uint32_t& equal_b) {
+  sample_hist<false>(rv, sm, 0u, sh);
+  uint32_t bin_a = 0, up_a = 0;
+  if (rank_a) {
+    find_bin256(sh, rank_a);
+    bin_a = (uint32_t)sh.bin;
+    up_a = sh.above;
+    __syncthreads();
+  }
+  find_bin256(sh, rank_b);
+  const uint32_t bin_b = (uint32_t)sh.bin, up_b = sh.above;
+  __syncthreads();
+  sample_hist<true>(rv, sm, bin_b, sh);
+  find_bin256(sh, rank_b - up_b);
+  code_b = (bin_b << 8) | (uint32_t)sh.bin;
+  above_b = up_b + sh.above;
+  equal_b = sh.hist[sh.bin];
+  __syncthreads();
+  code_a = 0xffffu;
+  if (rank_a) {
+    if (bin_a != bin_b) sample_hist<true>(rv, sm, bin_a, sh);
+    find_bin256(sh, rank_a - up_a);
+    code_a = (bin_a << 8) | (uint32_t)sh.bin;
+    __syncthreads();
+  }
+}
 
 // One sweep: A = number of keys with code > hi; hist[(c - lo) >> shift] = number of keys with code c
 // in [lo, hi] ((hi - lo) >> shift < kWin).  Neither bound is 0x7fff.
@@ -276,7 +330,8 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
                    const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int RC, int row_chunks,
                    int64_t n_tiles_total, float scale, const int32_t* __restrict__ b_step, int64_t row_words,
-                   uint32_t* __restrict__ mask) {
+                   uint32_t* __restrict__ mask, int bitrow_bytes, int cand_per_thread) {
+  extern __shared__ __align__(16) uint8_t dyn_smem[];   // [bit row | candidate lists]
   __shared__ Sel16Shared sh;
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int start = cu[r], N = cu[r + 1] - start;
@@ -304,55 +359,181 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   }
   {
     const __nv_bfloat16* qrow = Q + (((int64_t)r * (Hq / G) + kh) * (G * (S + 1)) + grow_idx) * d_k;
-    for (int i = tid; i < d_k; i += kThreads) sh.qf[i] = __bfloat162float(qrow[i]);
-    if (tid == 0) sh.ntie = 0;
+    for (int i = tid; i < d_k; i += kThreads) sh.qf[i] = qrow[i];
+    if (tid == 0) { sh.ntie = 0; sh.novf = 0; }
   }
 
   // ---------------------------------------------------------------- 1. sample
   uint32_t T = 0, above = 0, eq = 0;
   bool found = false;
   uint32_t lo, hi = 0xffffu;
-  {
-    uint4 sv[2];
-    int have = 0;
-    const bool whole = rv.nv8 <= kSampleVecs;
-    const int stride8 = whole ? 1 : rv.nv8 / kSampleVecs;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int j = tid + i * kThreads;
-      const int v8 = whole ? j : j * stride8 + (stride8 >> 1);
-      sv[i] = rv.load(v8);                                // vectors past the row read as -inf
-      if (v8 < rv.nv8) have = i + 1;
-    }
-    if (whole) {
-      // the whole row is in the sample: its k-th largest code is the threshold
-      T = sample_kth(sh, sv, have, (uint32_t)k, above, eq);
-      found = true;
-      lo = T;
-    } else {
-      // bracket the k-th largest key between two order statistics of the sample, a few standard
-      // deviations of the sampling error either side of the expected rank
-      const float m_s = (float)(kSampleVecs * 8);
-      const float rk = (float)k * m_s / (float)N;
-      const float dlt = 4.5f * sqrtf(rk) + 6.0f;
-      int r_lo = (int)ceilf(rk + dlt);
-      if (r_lo > kSampleVecs * 8) r_lo = kSampleVecs * 8;
-      const int r_hi = (int)floorf(rk - dlt);
-      uint32_t a_s, e_s;
-      lo = sample_kth(sh, sv, 2, (uint32_t)r_lo, a_s, e_s);
-      hi = r_hi >= 1 ? sample_kth(sh, sv, 2, (uint32_t)r_hi, a_s, e_s) : 0xffffu;
-    }
-  }
-
-  // ---------------------------------------------------------------- 2. window passes
-  // A window is [lo, hi] in code space, histogrammed in 2048 bins of 2^shift codes.  A window wider
-  // than 2048 codes is narrowed to the bin that holds the threshold and swept again; a bracket that
-  // turns out wrong (rare) is replaced by everything above or below it.
-  if (!found) {
+  if (rv.nv8 <= kSampleRound) {
+    // the whole row is the sample: its k-th largest code is the threshold
+    const Sample sm{rv.nv8, 1};
+    uint32_t unused;
+    sample_ranks(rv, sm, 0u, (uint32_t)k, sh, unused, T, above, eq);
+    found = true;
+    lo = T;
+  } else {
+    // 512 evenly spaced vectors (4096 keys); bracket the k-th largest key between two order statistics
+    // of the sample, 4.5 standard deviations of the (hypergeometric) sampling error either side
+    Sample sm;
+    sm.n_vecs = kSampleRound;
+    sm.stride = rv.nv8 / sm.n_vecs;
+    const float m_s = (float)(sm.n_vecs * 8);
+    const float frac = (float)k / (float)N;
+    const float rk = frac * m_s;
+    const float dlt = 4.5f * sqrtf(rk * (1.0f - frac)) + 6.0f;
+    int r_lo = (int)ceilf(rk + dlt);
+    if (r_lo > sm.n_vecs * 8) r_lo = sm.n_vecs * 8;
+    const int r_hi = (int)floorf(rk - dlt);
+    uint32_t a_s, e_s;
+    sample_ranks(rv, sm, r_hi >= 1 ? (uint32_t)r_hi : 0u, (uint32_t)r_lo, sh, hi, lo, a_s, e_s);
     if (lo < kMinCode) lo = kMinCode;
     if (hi < lo) hi = lo;
     lo = fix_lo(lo);
     hi = fix_hi(hi);
+  }
+
+  // ---------------------------------------------------------------- 2. one sweep with a bit row and lists
+  // Every thread lists the bracket keys it meets in a slice of its own, entry = key << 16 | vector
+  // number within the thread << 3 | position in the vector, stored slot-major (conflict free, no
+  // atomics, no warp scans).
+  if (!found && words * 4 <= bitrow_bytes) {
+    uint32_t* bitrow = reinterpret_cast<uint32_t*>(dyn_smem);
+    uint32_t* cand = reinterpret_cast<uint32_t*>(dyn_smem + bitrow_bytes);      // [cand_per_thread][kThreads]
+    const __half2 tlo = pair_of(raw_of(lo)), thi = pair_of(raw_of(hi));
+    uint32_t a16 = 0;   // 16 per key above the bracket
+    int cnt = 0;        // bracket keys this thread has met
+    for (int base = 0; base < rv.nv8; base += kThreads * kLoads) {
+      uint4 buf[kLoads];
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) buf[u] = rv.load(base + u * kThreads + tid);
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int v8 = base + u * kThreads + tid;
+        const uint32_t w[4] = {buf[u].x, buf[u].y, buf[u].z, buf[u].w};
+        uint32_t ge[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ge[j] = __hge2_mask(as_h2(w[j]), tlo);
+        uint32_t bits = 0;
+        if ((ge[0] | ge[1] | ge[2] | ge[3]) != 0u) {
+          // bit 2j of the low half and bit 2j+1 of the high half of word j mark its two keys
+          uint32_t gacc = 0, cacc = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t pick = (1u << (2 * j)) | (1u << (17 + 2 * j));
+            const uint32_t gt = __hgt2_mask(as_h2(w[j]), thi);
+            a16 += __popc(gt);
+            gacc |= gt & pick;
+            cacc |= (ge[j] & ~gt) & pick;
+          }
+          bits = (gacc | (gacc >> 16)) & 0xffu;
+          uint32_t cbits = (cacc | (cacc >> 16)) & 0xffu;
+          const uint32_t tag = (uint32_t)(v8 / kThreads) << 3;
+          while (cbits) {
+            const int j = __ffs(cbits) - 1;
+            cbits &= cbits - 1;
+            const uint32_t ww = (j < 4) ? ((j < 2) ? w[0] : w[1]) : ((j < 6) ? w[2] : w[3]);
+            const uint32_t key = (j & 1) ? (ww >> 16) : (ww & 0xffffu);
+            if (cnt < cand_per_thread) {
+              cand[cnt * kThreads + tid] = (key << 16) | tag | (uint32_t)j;
+              ++cnt;
+            } else {                                     // the rare key beyond the slice: shared spill list
+              const uint32_t slot = atomicAdd(&sh.novf, 1u);
+              if (slot < (uint32_t)kOvfCap) { sh.ovf_n[slot] = (uint32_t)(v8 * 8 + j); sh.ovf_key[slot] = (uint16_t)key; }
+            }
+          }
+        }
+        uint32_t word = bits << (8 * (lane & 3));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        if ((lane & 3) == 0 && (v8 >> 2) < words) bitrow[v8 >> 2] = word;
+      }
+    }
+    const uint32_t A = block_sum(sh, a16 >> 4);
+    const uint32_t novf = sh.novf;
+    const uint32_t C = block_sum(sh, (uint32_t)cnt) + novf;
+    bool settled = novf <= (uint32_t)kOvfCap && A <= (uint32_t)k && A + C >= (uint32_t)k;
+    if (settled && A < (uint32_t)k) {
+      // the k - A largest of the listed keys: two-level histogram over the lists
+      const uint32_t need = (uint32_t)k - A;
+      for (int b = tid; b < 256; b += kThreads) sh.hist[b] = 0;
+      __syncthreads();
+      for (int i = 0; i < cnt; ++i) atomicAdd(&sh.hist[code_of(cand[i * kThreads + tid] >> 16) >> 8], 1u);
+      for (int i = tid; i < (int)novf; i += kThreads) atomicAdd(&sh.hist[code_of(sh.ovf_key[i]) >> 8], 1u);
+      __syncthreads();
+      find_bin256(sh, need);
+      const uint32_t b_top = (uint32_t)sh.bin;
+      uint32_t up = sh.above;
+      __syncthreads();
+      for (int b = tid; b < 256; b += kThreads) sh.hist[b] = 0;
+      __syncthreads();
+      for (int i = 0; i < cnt; ++i) {
+        const uint32_t c = code_of(cand[i * kThreads + tid] >> 16);
+        if ((c >> 8) == b_top) atomicAdd(&sh.hist[c & 255u], 1u);
+      }
+      for (int i = tid; i < (int)novf; i += kThreads) {
+        const uint32_t c = code_of(sh.ovf_key[i]);
+        if ((c >> 8) == b_top) atomicAdd(&sh.hist[c & 255u], 1u);
+      }
+      __syncthreads();
+      find_bin256(sh, need - up);
+      T = (b_top << 8) | (uint32_t)sh.bin;
+      up += sh.above;
+      eq = sh.hist[sh.bin];
+      const uint32_t ties = need - up;              // 1 <= ties <= eq
+      __syncthreads();
+      if (ties < eq && eq > (uint32_t)kTieCap) {
+        settled = false;                            // too many equal 16-bit keys for the list: exact route
+      } else {
+        for (int i = 0; i < cnt; ++i) {
+          const uint32_t e = cand[i * kThreads + tid];
+          const uint32_t c = code_of(e >> 16);
+          const uint32_t n = ((((e >> 3) & 0x1fffu) * kThreads + (uint32_t)tid) << 3) | (e & 7u);
+          if (c > T || (c == T && ties >= eq)) atomicOr(&bitrow[n >> 5], 1u << (n & 31));
+          else if (c == T) sh.tie_idx[atomicAdd(&sh.ntie, 1u)] = (int)n;
+        }
+        for (int i = tid; i < (int)novf; i += kThreads) {
+          const uint32_t c = code_of(sh.ovf_key[i]), n = sh.ovf_n[i];
+          if (c > T || (c == T && ties >= eq)) atomicOr(&bitrow[n >> 5], 1u << (n & 31));
+          else if (c == T) sh.tie_idx[atomicAdd(&sh.ntie, 1u)] = (int)n;
+        }
+        __syncthreads();
+        if (ties < eq) {
+          DotCtx dot{sh.qf, K + (int64_t)kh * k_head + (int64_t)start * k_tok, k_tok, d_k, scale};
+          for (int i = tid; i < (int)eq; i += kThreads) sh.tie_val[i] = dot(sh.tie_idx[i]);
+          __syncthreads();
+          for (int i = tid; i < (int)eq; i += kThreads) {
+            const float v = sh.tie_val[i];
+            const int n = sh.tie_idx[i];
+            uint32_t rank = 0;
+            for (int u = 0; u < (int)eq; ++u) {
+              const float vu = sh.tie_val[u];
+              rank += (vu > v || (vu == v && sh.tie_idx[u] < n)) ? 1u : 0u;
+            }
+            if (rank < ties) atomicOr(&bitrow[n >> 5], 1u << (n & 31));
+          }
+        }
+      }
+    }
+    __syncthreads();
+    if (settled) {
+      for (int w = tid; w < words; w += kThreads) {
+        const uint32_t v = bitrow[w];
+        if (v) atomicOr(&mrow[w], v);
+      }
+      return;
+    }
+    if (tid == 0) sh.ntie = 0;
+    __syncthreads();
+  }
+
+  // ---------------------------------------------------------------- 4. exact route: window sweeps
+  // A window is [lo, hi] in code space, histogrammed in 2048 bins of 2^shift codes.  A window wider
+  // than 2048 codes is narrowed to the bin that holds the threshold and swept again; a bracket that
+  // turns out wrong (rare) is replaced by everything above or below it.
+  if (!found) {
     for (int iter = 0; iter < 12; ++iter) {
       int shift = 0;
       while (((hi - lo) >> shift) >= (uint32_t)kWin) ++shift;
@@ -390,7 +571,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   const uint32_t ties = (uint32_t)k - above;              // 1 <= ties <= eq
   const bool all_ties = ties >= eq;
 
-  // ---------------------------------------------------------------- 3. emission
+  // ---------------------------------------------------------------- emission sweep
   {
     const __half2 tt = pair_of(raw_of(T));
     for (int base = 0; base < rv.nv8; base += kThreads * kLoads) {
@@ -512,11 +693,24 @@ int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_
   const ScoreGeometry geo = score_geometry(p);
   dim3 grid(p->S, Hq, batch);
   const float scale = (float)(1.0 / sqrt((double)p->d_k));
+  // The one-sweep route needs a bit row of max_N bits and a list slice per thread sized for the widest
+  // bracket (k = N/2: 4.5 standard deviations of the 4096-key sample's rank, 32, plus 6, either side,
+  // times the keys per sampled key), spread over the threads, plus 1.7 standard deviations of that
+  // share; what a thread meets beyond its slice goes to a small shared spill list.  Rows too long for 32 KB of bits go
+  // straight to the exact route.
+  int bitrow_bytes = 0, cand_per_thread = 0;
+  if (max_N > (int64_t)kSampleRound * 8 && max_N <= 256 * 1024) {
+    bitrow_bytes = (int)align_up((size_t)ceil_div(max_N, 32) * 4, 16);
+    const double share = 2.0 * (4.5 * 32.0 + 6.0) * ((double)max_N / (kSampleRound * 8)) / kThreads;
+    cand_per_thread = (int)ceil(share + 1.7 * sqrt(share));
+  }
+  const size_t smem = (size_t)bitrow_bytes + (size_t)cand_per_thread * kThreads * sizeof(uint32_t);
+  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topk16_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("topk16_rows_kernel", st);
-    topk16_rows_kernel<<<grid, kThreads, 0, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
-                                                  geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
-                                                  row_words, mask);
+    topk16_rows_kernel<<<grid, kThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
+                                                     geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
+                                                     row_words, mask, bitrow_bytes, cand_per_thread);
   }
   GVOTE_LAUNCH_CHECK("topk16_rows_kernel");
   return GVOTE_OK;

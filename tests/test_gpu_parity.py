@@ -228,6 +228,37 @@ def test_vote_single_dominant_key(gv):
     assert np.array_equal(gv.unpack_mask(mask[0], 0, 77), om[0])
 
 
+@pytest.mark.parametrize("shift_sampled,shift_sign", [(0.0, 0.0), (-6.0, 0.0), (+6.0, 0.0), (0.0, 1.0)])
+def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
+    """Rows long enough for the sampled one-sweep top-k.  The kernel samples fixed positions (every
+    fourth 8-key vector here); shifting the logits at exactly those positions makes the sample's
+    bracket miss the true threshold, so the exact route has to take over.  shift_sign = 1 centres
+    the logits on zero with tiny magnitudes (half-precision codes are densest there)."""
+    N, d_k, S = 16384, 64, 6
+    cfg = synth.make_small(11, seq_lens=(N,), S=S, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=d_k, p_nuc=0.9)
+    li = synth.make_layer(cfg, 0)
+    rng = np.random.default_rng(3)
+    e = rng.normal(size=d_k)
+    e /= np.linalg.norm(e)
+    v = rng.normal(size=N) * (1e-3 if shift_sign else 1.0)
+    sampled = np.zeros(N, dtype=bool)
+    nv8, n_vecs = N // 8, 512
+    stride = nv8 // n_vecs
+    for i in range(n_vecs):
+        sampled[(i * stride + stride // 2) * 8:(i * stride + stride // 2) * 8 + 8] = True
+    v[sampled] += shift_sampled
+    Kf = (v[:, None] * e[None, :] * math.sqrt(d_k)).astype(np.float32)[None]          # logit of key n = v_n q.e
+    li.K = synth.f32_to_bf16_bits(Kf)
+    q = o.round_to_bf16(np.stack([e * (1.0 + 0.05 * r) for r in range(S + 1)]))     # rows differ a little
+    Q_or = [np.stack([q, q[::-1].copy()])]
+    mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    Kr = o.bf16_bits_to_f64(li.K)
+    gm = np.stack([gv.unpack_mask(mask[0], 0, N)])
+    pu.check_vote_against_oracle(Q_or[0], Kr, float(np.float32(cfg.p_nuc)), "topk", False, gm, b_step[0])
+    om, ob, _, _, _ = o.vote(Q_or[0], Kr, p_nuc=float(np.float32(cfg.p_nuc)))
+    assert abs(int(budget[0, 0]) - int(ob[0])) <= 0.005 * N
+
+
 # ----------------------------------------------------------------------------- compact
 @pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
                                                   ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
