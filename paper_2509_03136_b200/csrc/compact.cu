@@ -81,8 +81,8 @@ constexpr int kSpinLimit = 1 << 22;
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, int64_t tok, int64_t head,
                const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
-               const int32_t* __restrict__ cu, int batch, int Hkv, int d_k, int64_t row_words, int64_t n_tiles,
-               int32_t* flags, int32_t* ticket, int32_t* status) {
+               const int32_t* __restrict__ cu, const int32_t* __restrict__ budget, int batch, int Hkv, int d_k,
+               int64_t row_words, int64_t n_tiles, int32_t* flags, int32_t* ticket, int32_t* status) {
   extern __shared__ __align__(16) uint4 rows_sm[];   // [kept rows][d_k*2/16]
   __shared__ int s_ticket;
   __shared__ int s_src[kCompactTile];                // source token (within request) of each kept row
@@ -102,6 +102,8 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   const int t = (int)(gt - tile_offset(start, r));
   const int tiles = (N + kCompactTile - 1) / kCompactTile;
   if (t >= tiles) return;   // padding slot of the tile list
+  // a head that keeps every key moves nothing, and none of its tiles waits for another
+  if (budget[r * Hkv + h] == N) return;
   __nv_bfloat16* base = ((slab & 1) ? Vp : Kp) + (int64_t)h * head + (int64_t)start * tok;
   int32_t* my_flags = flags + (int64_t)slab * n_tiles + tile_offset(start, r);
 
@@ -186,8 +188,8 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
   const int64_t ctas = m.n_tiles * 2 * Hkv;
   {
     LaunchScope scope_("compact_kernel", st);
-  compact_kernel<<<(unsigned)ctas, kCompactThreads, smem, st>>>(K, V, tok, head, mask, prefix, cu, batch, Hkv, p->d_k,
-                                                                m.row_words, m.n_tiles, flags, ticket, status);
+  compact_kernel<<<(unsigned)ctas, kCompactThreads, smem, st>>>(K, V, tok, head, mask, prefix, cu, budget, batch, Hkv,
+                                                                p->d_k, m.row_words, m.n_tiles, flags, ticket, status);
   }
   GVOTE_LAUNCH_CHECK("compact_kernel");
   return GVOTE_OK;

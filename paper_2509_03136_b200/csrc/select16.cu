@@ -163,65 +163,102 @@ struct RowView {
   }
 };
 
-// 256-bin histogram (left in sh.hist[0..256)) of the sampled codes' high bytes (level 1), or of the low
-// bytes of the sampled codes whose high byte is `only` (level 2).
-// Level 1 sees every sampled key and a few bins take most of them, so plain shared-memory atomics
-// would serialise on those addresses.  It counts into one 8-bit counter per (bin, lane) instead, four
-// bins to a word, word index (bin / 4) * 32 + lane: the lanes of a warp never meet, and a counter
-// takes at most (warps) * (sample keys per thread) = 4 * 32 increments, well below 256.
-template <bool LEVEL2>
-__device__ void sample_hist(const RowView& rv, const Sample& sm, uint32_t only, Sel16Shared& sh) {
+// The sampled vectors of this thread (those past the sample read as -inf and are not counted).
+struct SampleRegs {
+  uint4 v[4];
+  int have;
+};
+__device__ __forceinline__ SampleRegs sample_load(const RowView& rv, const Sample& sm) {
+  SampleRegs sr;
+  sr.have = 0;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int i = u * kThreads + (int)threadIdx.x;
+    sr.v[u] = rv.load(i < sm.n_vecs ? sm.vec(i) : rv.nv8);
+    if (i < sm.n_vecs) sr.have = u + 1;
+  }
+  return sr;
+}
+
+// High byte of a key's code from the high byte hb of its half bits, and back.
+__device__ __forceinline__ uint32_t ord_hi(uint32_t hb) { return hb >= 0x80u ? 0xffu - hb : 0x80u + hb; }
+
+// Level 1: 256-bin histogram (left in sh.hist[0..256), indexed by the code's high byte) of the sampled
+// keys.  Every sampled key takes part and a few bins take most of them, so plain shared-memory
+// atomics would serialise on those addresses.  Counting goes into one 8-bit counter per (bin, lane)
+// instead, four bins to a word, word index (bin / 4) * 32 + lane: the lanes of a warp never meet, and
+// a counter takes at most (warps) * (sample keys per thread) = 4 * 32 increments, well below 256.
+// Bins are those of the raw half bits here (no per-key recoding); the fold puts them in code order.
+__device__ void sample_hist_hi(const SampleRegs& sr, Sel16Shared& sh) {
   const int lane = threadIdx.x & 31;
-  for (int b = threadIdx.x; b < (LEVEL2 ? 256 : kWin); b += kThreads) sh.hist[b] = 0;
+  for (int b = threadIdx.x; b < kWin; b += kThreads) sh.hist[b] = 0;
   __syncthreads();
-  {
-    uint4 sv[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = u * kThreads + (int)threadIdx.x;
-      sv[u] = i < sm.n_vecs ? rv.load(sm.vec(i)) : make_uint4(0u, 0u, 0u, 0u);
-    }
+  for (int u = 0; u < 4; ++u) {
+    if (u >= sr.have) break;
+    const uint32_t w[4] = {sr.v[u].x, sr.v[u].y, sr.v[u].z, sr.v[u].w};
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (u * kThreads + (int)threadIdx.x >= sm.n_vecs) continue;
-      const uint32_t w[4] = {sv[u].x, sv[u].y, sv[u].z, sv[u].w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t c0 = code_of(w[j] & 0xffffu), c1 = code_of(w[j] >> 16);
-        if (!LEVEL2) {
-          atomicAdd(&sh.hist[(c0 >> 10) * 32 + lane], 1u << ((c0 >> 5) & 24u));
-          atomicAdd(&sh.hist[(c1 >> 10) * 32 + lane], 1u << ((c1 >> 5) & 24u));
-        } else {
-          if ((c0 >> 8) == only) atomicAdd(&sh.hist[c0 & 255u], 1u);
-          if ((c1 >> 8) == only) atomicAdd(&sh.hist[c1 & 255u], 1u);
-        }
-      }
+    for (int j = 0; j < 4; ++j) {
+      uint32_t h0 = w[j] & 0xffffu, h1 = w[j] >> 16;
+      if (h0 == 0x8000u) h0 = 0u;                        // -0 counts as +0
+      if (h1 == 0x8000u) h1 = 0u;
+      atomicAdd(&sh.hist[(h0 >> 10) * 32 + lane], 1u << ((h0 >> 5) & 24u));
+      atomicAdd(&sh.hist[(h1 >> 10) * 32 + lane], 1u << ((h1 >> 5) & 24u));
     }
   }
   __syncthreads();
-  if (!LEVEL2) {
-    // fold the lanes: thread t sums bins 2t and 2t+1
-    uint32_t tot[2] = {0u, 0u};
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const int bin = 2 * (int)threadIdx.x + q;
-      const uint32_t* wrow = &sh.hist[(bin >> 2) * 32];
-      const int sh8 = (bin & 3) * 8;
-      for (int l = 0; l < 32; ++l) tot[q] += (wrow[(l + lane) & 31] >> sh8) & 255u;   // rotated: conflict free
+  // fold the lanes: thread t < 64 sums word row t (raw bins 4t .. 4t+3), two bins per accumulator
+  uint32_t even = 0, odd = 0;
+  if (threadIdx.x < 64) {
+    const uint32_t* wrow = &sh.hist[threadIdx.x * 32];
+#pragma unroll 8
+    for (int l = 0; l < 32; ++l) {
+      const uint32_t w = wrow[(l + lane) & 31];           // rotated: conflict free
+      even += w & 0x00ff00ffu;
+      odd += (w >> 8) & 0x00ff00ffu;
     }
-    __syncthreads();
-    sh.hist[2 * threadIdx.x] = tot[0];
-    sh.hist[2 * threadIdx.x + 1] = tot[1];
-    __syncthreads();
   }
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    const uint32_t hb = 4u * threadIdx.x;
+    sh.hist[ord_hi(hb)] = even & 0xffffu;
+    sh.hist[ord_hi(hb + 1)] = odd & 0xffffu;
+    sh.hist[ord_hi(hb + 2)] = even >> 16;
+    sh.hist[ord_hi(hb + 3)] = odd >> 16;
+  }
+  __syncthreads();
+}
+
+// Level 2: 256-bin histogram (sh.hist[0..256), indexed by the code's low byte) of the sampled keys
+// whose code has high byte `only`.
+__device__ void sample_hist_lo(const SampleRegs& sr, uint32_t only, Sel16Shared& sh) {
+  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
+  __syncthreads();
+  const bool neg = only < 0x80u;                          // codes below 0x8000 are negative numbers
+  const uint32_t raw_hb = neg ? 0xffu - only : only - 0x80u;
+  const uint32_t flip = neg ? 0xffu : 0u;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (u >= sr.have) break;
+    const uint32_t w[4] = {sr.v[u].x, sr.v[u].y, sr.v[u].z, sr.v[u].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t h0 = w[j] & 0xffffu, h1 = w[j] >> 16;
+      if (h0 == 0x8000u) h0 = 0u;
+      if (h1 == 0x8000u) h1 = 0u;
+      if ((h0 >> 8) == raw_hb) atomicAdd(&sh.hist[(h0 & 255u) ^ flip], 1u);
+      if ((h1 >> 8) == raw_hb) atomicAdd(&sh.hist[(h1 & 255u) ^ flip], 1u);
+    }
+  }
+  __syncthreads();
 }
 
 // The sample's rank_a-th and rank_b-th largest codes (1 <= rank_a <= rank_b <= sampled keys; rank_a = 0
 // asks for the second one only).  For the second one also the number of sampled codes above it and
 // equal to it.  Every thread of the CTA calls it.
-__device__ void sample_ranks(const RowView& rv, const Sample& sm, uint32_t rank_a, uint32_t rank_b, Sel16Shared& sh,
+__device__ void sample_ranks(const SampleRegs& sr, uint32_t rank_a, uint32_t rank_b, Sel16Shared& sh,
                              uint32_t& code_a, uint32_t& code_b, uint32_t& above_b, uint32_t& equal_b) {
-  sample_hist<false>(rv, sm, 0u, sh);
+  sample_hist_hi(sr, sh);
   uint32_t bin_a = 0, up_a = 0;
   if (rank_a) {
     find_bin256(sh, rank_a);
@@ -232,7 +269,7 @@ __device__ void sample_ranks(const RowView& rv, const Sample& sm, uint32_t rank_
   find_bin256(sh, rank_b);
   const uint32_t bin_b = (uint32_t)sh.bin, up_b = sh.above;
   __syncthreads();
-  sample_hist<true>(rv, sm, bin_b, sh);
+  sample_hist_lo(sr, bin_b, sh);
   find_bin256(sh, rank_b - up_b);
   code_b = (bin_b << 8) | (uint32_t)sh.bin;
   above_b = up_b + sh.above;
@@ -240,7 +277,7 @@ __device__ void sample_ranks(const RowView& rv, const Sample& sm, uint32_t rank_
   __syncthreads();
   code_a = 0xffffu;
   if (rank_a) {
-    if (bin_a != bin_b) sample_hist<true>(rv, sm, bin_a, sh);
+    if (bin_a != bin_b) sample_hist_lo(sr, bin_a, sh);
     find_bin256(sh, rank_a - up_a);
     code_a = (bin_a << 8) | (uint32_t)sh.bin;
     __syncthreads();
@@ -370,8 +407,9 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   if (rv.nv8 <= kSampleRound) {
     // the whole row is the sample: its k-th largest code is the threshold
     const Sample sm{rv.nv8, 1};
+    const SampleRegs sr = sample_load(rv, sm);
     uint32_t unused;
-    sample_ranks(rv, sm, 0u, (uint32_t)k, sh, unused, T, above, eq);
+    sample_ranks(sr, 0u, (uint32_t)k, sh, unused, T, above, eq);
     found = true;
     lo = T;
   } else {
@@ -388,7 +426,8 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
     if (r_lo > sm.n_vecs * 8) r_lo = sm.n_vecs * 8;
     const int r_hi = (int)floorf(rk - dlt);
     uint32_t a_s, e_s;
-    sample_ranks(rv, sm, r_hi >= 1 ? (uint32_t)r_hi : 0u, (uint32_t)r_lo, sh, hi, lo, a_s, e_s);
+    const SampleRegs sr = sample_load(rv, sm);
+    sample_ranks(sr, r_hi >= 1 ? (uint32_t)r_hi : 0u, (uint32_t)r_lo, sh, hi, lo, a_s, e_s);
     if (lo < kMinCode) lo = kMinCode;
     if (hi < lo) hi = lo;
     lo = fix_lo(lo);
