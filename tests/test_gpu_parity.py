@@ -386,6 +386,13 @@ def test_compress_full_size_c2_layer(gv):
     _check_compress(gv, cfg, synth.make_layer(cfg, 3), layer_id=3)
 
 
+def test_compress_full_size_c4_layer(gv):
+    """One layer of the 128K-context Qwen2.5-7B-shaped workload (N = 131072, G = 7, S = 64, p = 0.98):
+    two row chunks per KV head in the score contraction, 2 MB of mask bits, 1.9 GB of hidden states."""
+    cfg = synth.make_config("c4")
+    _check_compress(gv, cfg, synth.make_layer(cfg, 1), layer_id=1)
+
+
 def test_compress_host_variant_matches_device_variant(gv):
     cfg = synth.make_config("c0")
     li = synth.make_layer(cfg, 0)
