@@ -77,8 +77,8 @@ struct WorkspaceMap {
   int64_t row_words;    // mask words per head
 };
 
-// Row tiling of the tensor-core score kernel: the (S+1)*G rows of a head group are split into
-// `row_chunks` chunks of RC rows (RC a multiple of 16, at most 240).
+// Row tiling of the tensor-core score kernel: the G*S synthetic rows of a head group are split into
+// `row_chunks` chunks of RC = 128 rows (the current-query rows travel with chunk 0).
 struct ScoreGeometry { int RC; int row_chunks; };
 ScoreGeometry score_geometry(const gvote_params* p);
 size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens);

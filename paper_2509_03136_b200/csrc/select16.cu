@@ -141,15 +141,17 @@ struct DotCtx {
   }
 };
 
-// Where a row's keys live: eight consecutive keys form one 16-byte vector; vector v8 of the row
-// sits in tile v8 / 16 at offset (v8 % 16) * 8.  Positions >= N read as -inf.
+// Where a row's keys live: eight consecutive keys form one 16-byte vector; vector v8 of the row sits in
+// tile v8 / 16, at chunk position (v8 % 16) ^ swz of the row's 16 chunks there (the score kernel stores
+// its tiles XOR-swizzled by the row number, swz = row % 16).  Positions >= N read as -inf.
 struct RowView {
   const uint16_t* grow;         // first tile of the row in global memory
   int64_t tile_stride;          // elements between consecutive tiles of the same row
   int N, nv8;
+  uint32_t swz;
   __device__ __forceinline__ uint4 load(int v8) const {
     if (v8 >= nv8) return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u);
-    uint4 v = *reinterpret_cast<const uint4*>(grow + (int64_t)(v8 >> 4) * tile_stride + (v8 & 15) * 8);
+    uint4 v = *reinterpret_cast<const uint4*>(grow + (int64_t)(v8 >> 4) * tile_stride + (((uint32_t)v8 & 15u) ^ swz) * 8);
     if (v8 * 8 + 8 > N) {
       uint16_t* e = reinterpret_cast<uint16_t*>(&v);
 #pragma unroll
@@ -159,7 +161,7 @@ struct RowView {
     return v;
   }
   __device__ __forceinline__ uint32_t key_at(int n) const {
-    return grow[(int64_t)(n >> 7) * tile_stride + (n & 127)];
+    return grow[(int64_t)(n >> 7) * tile_stride + (((((uint32_t)n & 127u) >> 3) ^ swz) << 3) + (n & 7)];
   }
 };
 
@@ -383,6 +385,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   rv.N = N;
   rv.nv8 = (N + 7) >> 3;
   rv.tile_stride = (int64_t)row_chunks * RC * kTileKeys;
+  rv.swz = (uint32_t)crow & 15u;
   rv.grow = keys16 + ((((int64_t)kh * n_tiles_total + tile_offset(start, r)) * row_chunks + chunk) * RC + crow) * kTileKeys;
   uint32_t* mrow = mask + (int64_t)kh * row_words + mask_word_offset(start, r);
   const int words = (N + 31) >> 5;
