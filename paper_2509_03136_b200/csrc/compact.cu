@@ -97,44 +97,54 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   const int slab = (int)(tk % slabs);
   const int h = slab >> 1;
   if (gt >= n_tiles) return;
-  const int r = find_request(cu, batch, gt);
+  const int r = batch == 1 ? 0 : find_request(cu, batch, gt);
   const int start = cu[r], N = cu[r + 1] - start;
   const int t = (int)(gt - tile_offset(start, r));
   const int tiles = (N + kCompactTile - 1) / kCompactTile;
   if (t >= tiles) return;   // padding slot of the tile list
-  // a head that keeps every key moves nothing, and none of its tiles waits for another
-  if (budget[r * Hkv + h] == N) return;
   __nv_bfloat16* base = ((slab & 1) ? Vp : Kp) + (int64_t)h * head + (int64_t)start * tok;
   int32_t* my_flags = flags + (int64_t)slab * n_tiles + tile_offset(start, r);
 
-  // the tile's four mask words and its destination offset
+  // the tile's four mask words and its destination offset: every load below is issued before the
+  // first of them is needed
   const int64_t woff = (int64_t)h * row_words + mask_word_offset(start, r) + (int64_t)t * (kCompactTile / 32);
   const int words = min(kCompactTile / 32, ((N + 31) >> 5) - t * (kCompactTile / 32));
+  const int w_mine = min(tid >> 5, words - 1), lastw = words - 1;
+  const int kept_all = budget[r * Hkv + h];
   const int dst0 = prefix[woff];
-  if (tid < kCompactTile) {
-    const int w = tid >> 5, b = tid & 31;
-    if (w < words) {
-      const uint32_t mw = mask[woff + w];
-      if ((mw >> b) & 1u) {
-        const int rank = (prefix[woff + w] - dst0) + __popc(mw & ((1u << b) - 1u));
-        s_src[rank] = t * kCompactTile + tid;
-      }
-    }
+  const uint32_t mw = mask[woff + w_mine];
+  const int pw = prefix[woff + w_mine];
+  const int p_last = prefix[woff + lastw];
+  const uint32_t m_last = mask[woff + lastw];
+  // a head that keeps every key moves nothing, and none of its tiles waits for another
+  if (kept_all == N) return;
+  if (tid < kCompactTile && (tid >> 5) < words) {
+    const int b = tid & 31;
+    if ((mw >> b) & 1u) s_src[(pw - dst0) + __popc(mw & ((1u << b) - 1u))] = t * kCompactTile + tid;
   }
-  int cnt = 0;
-  {
-    const int lastw = words - 1;
-    cnt = prefix[woff + lastw] - dst0 + __popc(mask[woff + lastw]);
-  }
+  const int cnt = p_last - dst0 + __popc(m_last);
   __syncthreads();
   const int pieces = d_k / 8;                       // 16-byte pieces per row
   // rows whose destination equals their source need no move; they form a prefix of the tile
   // exactly when nothing was dropped before them: dst0 + i == src_i.
-  for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
-    const int i = idx / pieces, pc = idx % pieces;
-    const int src = s_src[i];
-    if (src != dst0 + i)
-      rows_sm[idx] = *reinterpret_cast<const uint4*>(base + (int64_t)src * tok + pc * 8);
+  // All of a thread's pieces are requested before any is waited for (asynchronous copies straight
+  // into shared memory); (row, piece) advance without divisions.
+  const int step_i = kCompactThreads / pieces, step_pc = kCompactThreads % pieces;
+  {
+    int i = tid / pieces, pc = tid % pieces;
+    for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
+      const int src = s_src[i];
+      if (src != dst0 + i) {
+        const uint32_t dst_s = static_cast<uint32_t>(__cvta_generic_to_shared(&rows_sm[idx]));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_s), "l"(base + (int64_t)src * tok + pc * 8)
+                     : "memory");
+      }
+      i += step_i;
+      pc += step_pc;
+      if (pc >= pieces) { pc -= pieces; ++i; }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
   __syncthreads();
   if (tid == 0) {
@@ -159,10 +169,15 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   }
   __syncthreads();
   if (!s_ok) return;
-  for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
-    const int i = idx / pieces, pc = idx % pieces;
-    if (s_src[i] != dst0 + i)
-      *reinterpret_cast<uint4*>(base + (int64_t)(dst0 + i) * tok + pc * 8) = rows_sm[idx];
+  {
+    int i = tid / pieces, pc = tid % pieces;
+    for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
+      if (s_src[i] != dst0 + i)
+        *reinterpret_cast<uint4*>(base + (int64_t)(dst0 + i) * tok + pc * 8) = rows_sm[idx];
+      i += step_i;
+      pc += step_pc;
+      if (pc >= pieces) { pc -= pieces; ++i; }
+    }
   }
 }
 
