@@ -196,7 +196,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
-    ap.add_argument("--streams", type=int, default=4,
+    ap.add_argument("--streams", type=int, default=6,
                     help="CUDA streams the layers of a step are spread over (each with its own workspace)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

@@ -4,7 +4,7 @@
 //
 // One small CTA per synthetic row, many resident per SM.  Keys are compared as half-precision numbers,
 // two per instruction; for counting they are mapped to an order-preserving 16-bit code.
-//   1. A fixed, evenly spaced sample of 4096 keys brackets the k-th largest key between two of
+//   1. A fixed sample of 4096 keys (128 evenly spaced runs of 32) brackets the k-th largest key between two of
 //      the sample's order statistics, a few standard deviations of the sampling error either side of
 //      the expected rank.  (Rows of at most 4096 keys are sampled completely, which settles the
 //      threshold at once.)
@@ -109,11 +109,17 @@ __device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
   __syncthreads();
 }
 
-// The sample: vector i of `n_vecs` (at most four per thread) is vector i * stride + stride / 2 of the
-// row (stride 1 samples the whole row).
+// The sample: vector i of `n_vecs` (at most four per thread).  A row of at most n_vecs vectors is
+// sampled completely (stride 0).  Otherwise thread t takes four consecutive vectors (64 bytes, one
+// DRAM access) from the middle of the t-th of kThreads equal stretches of the row: scattering single
+// 16-byte vectors instead costs four times the DRAM accesses for the same number of keys.
 struct Sample {
   int n_vecs, stride;
-  __device__ __forceinline__ int vec(int i) const { return i * stride + (stride >> 1); }
+  __device__ __forceinline__ int vec(int i) const {
+    if (stride == 0) return i;
+    const int t = i % kThreads, u = i / kThreads;
+    return t * stride + ((stride >> 1) & ~3) + u;
+  }
 };
 
 // Exact fp32 logit of key n for this row's query (fixed summation order).
@@ -409,18 +415,18 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
   uint32_t lo, hi = 0xffffu;
   if (rv.nv8 <= kSampleRound) {
     // the whole row is the sample: its k-th largest code is the threshold
-    const Sample sm{rv.nv8, 1};
+    const Sample sm{rv.nv8, 0};
     const SampleRegs sr = sample_load(rv, sm);
     uint32_t unused;
     sample_ranks(sr, 0u, (uint32_t)k, sh, unused, T, above, eq);
     found = true;
     lo = T;
   } else {
-    // 512 evenly spaced vectors (4096 keys); bracket the k-th largest key between two order statistics
+    // 128 evenly spaced runs of 32 keys (4096 keys); bracket the k-th largest key between two order statistics
     // of the sample, 4.5 standard deviations of the (hypergeometric) sampling error either side
     Sample sm;
     sm.n_vecs = kSampleRound;
-    sm.stride = rv.nv8 / sm.n_vecs;
+    sm.stride = rv.nv8 / kThreads;                      // >= 4 here
     const float m_s = (float)(sm.n_vecs * 8);
     const float frac = (float)k / (float)N;
     const float rk = frac * m_s;

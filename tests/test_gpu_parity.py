@@ -230,8 +230,8 @@ def test_vote_single_dominant_key(gv):
 
 @pytest.mark.parametrize("shift_sampled,shift_sign", [(0.0, 0.0), (-6.0, 0.0), (+6.0, 0.0), (0.0, 1.0)])
 def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
-    """Rows long enough for the sampled one-sweep top-k.  The kernel samples fixed positions (every
-    fourth 8-key vector here); shifting the logits at exactly those positions makes the sample's
+    """Rows long enough for the sampled one-sweep top-k.  The kernel samples fixed positions (128
+    evenly spaced runs of 32 keys); shifting the logits at exactly those positions makes the sample's
     bracket miss the true threshold, so the exact route has to take over.  shift_sign = 1 centres
     the logits on zero with tiny magnitudes (half-precision codes are densest there)."""
     N, d_k, S = 16384, 64, 6
@@ -242,10 +242,11 @@ def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
     e /= np.linalg.norm(e)
     v = rng.normal(size=N) * (1e-3 if shift_sign else 1.0)
     sampled = np.zeros(N, dtype=bool)
-    nv8, n_vecs = N // 8, 512
-    stride = nv8 // n_vecs
-    for i in range(n_vecs):
-        sampled[(i * stride + stride // 2) * 8:(i * stride + stride // 2) * 8 + 8] = True
+    nv8 = N // 8
+    stride = nv8 // 128                                  # 128 runs of four 8-key vectors
+    for t in range(128):
+        first = t * stride + ((stride // 2) & ~3)
+        sampled[first * 8:(first + 4) * 8] = True
     v[sampled] += shift_sampled
     Kf = (v[:, None] * e[None, :] * math.sqrt(d_k)).astype(np.float32)[None]          # logit of key n = v_n q.e
     li.K = synth.f32_to_bf16_bits(Kf)
