@@ -129,20 +129,26 @@ struct DotCtx {
   int64_t k_tok;
   int d_k;
   float scale;
+  __device__ __forceinline__ void add8(float& acc, const uint4& v, int c) const {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h[j]);
+      const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qf + c * 8 + 2 * j));
+      acc = fmaf(q.x, f.x, acc);
+      acc = fmaf(q.y, f.y, acc);
+    }
+  }
   __device__ __forceinline__ float operator()(int n) const {
     const uint4* kp = reinterpret_cast<const uint4*>(krows + (int64_t)n * k_tok);
     float acc = 0.f;
-    for (int c = 0; c < d_k / 8; ++c) {
-      const uint4 v = __ldg(kp + c);
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 f = __bfloat1622float2(h[j]);
-        const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qf + c * 8 + 2 * j));
-        acc = fmaf(q.x, f.x, acc);
-        acc = fmaf(q.y, f.y, acc);
-      }
+    const int nc = d_k / 8;
+    int c = 0;
+    for (; c + 4 <= nc; c += 4) {                     // four loads in flight, summed in index order
+      const uint4 v0 = __ldg(kp + c), v1 = __ldg(kp + c + 1), v2 = __ldg(kp + c + 2), v3 = __ldg(kp + c + 3);
+      add8(acc, v0, c); add8(acc, v1, c + 1); add8(acc, v2, c + 2); add8(acc, v3, c + 3);
     }
+    for (; c < nc; ++c) add8(acc, __ldg(kp + c), c);
     return acc * scale;
   }
 };
