@@ -102,7 +102,7 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   m.real_scratch_bytes = real_topp_scratch_bytes(p, batch);
   m.real_scratch = take(m.real_scratch_bytes);
   m.prefix = take((size_t)p->n_kv_heads * m.row_words * sizeof(int32_t));
-  m.flags = take(((size_t)2 * p->n_kv_heads * m.n_tiles + 4) * sizeof(int32_t));
+  m.flags = take(((size_t)2 * p->n_kv_heads * m.n_tiles + (size_t)2 * p->n_kv_heads * 32) * sizeof(int32_t));
   m.total = off;
   return m;
 }

@@ -69,7 +69,7 @@ struct WorkspaceMap {
   size_t real_scratch;  // row maxima and mass histograms of the current-query rows (topp_real.cu)
   size_t real_scratch_bytes;
   size_t prefix;        // int32 [Hkv][row_words]  exclusive popcount prefix per mask word
-  size_t flags;         // int32 [2*Hkv*n_tiles + 4]  compaction "tile loaded" flags + ticket
+  size_t flags;         // int32 [2*Hkv*n_tiles] compaction "tile loaded" flags + [2*Hkv][32] ticket counters
   size_t total;
   int fit_chunks;       // row chunks per request in the fit
   int proj_splits;      // split-K factor of the projection

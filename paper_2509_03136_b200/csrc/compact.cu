@@ -2,24 +2,27 @@
 //
 // Two kernels.  mask_scan_kernel turns each (request, KV head) bit row into an exclusive popcount
 // prefix per 32-key word and the head's budget.  compact_kernel then moves the kept rows of one
-// 128-token tile per CTA to their destination rows, 16 bytes per thread per step.
+// 128-token tile per CTA to their destination rows: thread = token, one bulk copy per row into
+// shared memory and one out of it.
 //
 // In-place safety.  Row i moves to row prefix(i) <= i, so a tile's destination may still hold
 // rows that an EARLIER tile of the same slab has not read yet.  Each CTA therefore (1) takes a
-// ticket, which orders tiles so that a lower tile of a slab is always taken by a CTA that is
-// already running, (2) loads its kept rows into shared memory, (3) publishes a "loaded" flag,
+// ticket of its slab, which orders tiles so that a lower tile of a slab is always taken by a CTA
+// that is already running, (2) loads its kept rows into shared memory, (3) publishes a "loaded" flag,
 // (4) waits until the (at most two) earlier tiles whose rows its destination range overlaps have
 // published theirs, (5) stores.  The wait is bounded: when it runs out the CTA records
 // GVOTE_ERR_TIMEOUT in the workspace status word, skips its stores and returns.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace gvote {
 namespace {
 
 constexpr int kScanThreads = 256;
+constexpr int kTicketPitch = 32;     // ints between two slabs' ticket counters (128 bytes)
 
 // One CTA per (request, head): prefix[h][word] = kept keys of the request before this word.
-// Also clears the compaction flags of the request's tiles (and the ticket, once).
+// Also clears the compaction flags of the request's tiles (and the head's two ticket counters).
 __global__ void __launch_bounds__(kScanThreads)
 mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu, int Hkv, int64_t row_words,
                  int32_t* __restrict__ prefix, int32_t* __restrict__ budget, int32_t* __restrict__ flags,
@@ -34,7 +37,7 @@ mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ 
   int32_t* pf = prefix + (int64_t)h * row_words + woff;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) carry = 0;
-  if (r == 0 && h == 0 && tid == 0) { ticket[0] = 0; }
+  if (r == 0 && tid < 2) ticket[(2 * h + tid) * kTicketPitch] = 0;   // this head's K and V slabs
   if (flags) {
     const int tiles = (N + kCompactTile - 1) / kCompactTile;
     const int64_t toff = tile_offset(start, r);
@@ -75,7 +78,7 @@ __device__ __forceinline__ int find_request(const int32_t* __restrict__ cu, int 
   return lo;
 }
 
-constexpr int kCompactThreads = 256;
+constexpr int kCompactThreads = kCompactTile;    // one thread per token of the tile
 constexpr int kSpinLimit = 1 << 22;
 
 __global__ void __launch_bounds__(kCompactThreads)
@@ -83,19 +86,24 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
                const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
                const int32_t* __restrict__ cu, const int32_t* __restrict__ budget, int batch, int Hkv, int d_k,
                int64_t row_words, int64_t n_tiles, int32_t* flags, int32_t* ticket, int32_t* status) {
-  extern __shared__ __align__(16) uint4 rows_sm[];   // [kept rows][d_k*2/16]
+  extern __shared__ __align__(128) uint8_t rows_sm[];   // [kept rows][d_k * 2 bytes]
+  __shared__ __align__(8) uint64_t s_bar;
   __shared__ int s_ticket;
-  __shared__ int s_src[kCompactTile];                // source token (within request) of each kept row
   __shared__ int s_ok;
   const int tid = threadIdx.x;
-  if (tid == 0) s_ticket = atomicAdd(ticket, 1);
-  __syncthreads();
-  const int64_t tk = s_ticket;
-  // ticket order: tile-major, then (head, K|V): lower tiles of a slab always come first
+  // A CTA belongs to one slab (a head's K or V) by its block index and takes that slab's next tile:
+  // within a slab, a lower tile is always taken by a CTA that is already running.  One counter per
+  // slab (on a line of its own) instead of one for all keeps the atomics from queueing on one address.
   const int slabs = 2 * Hkv;
-  const int64_t gt = tk / slabs;
-  const int slab = (int)(tk % slabs);
+  const int slab = (int)(blockIdx.x % slabs);
   const int h = slab >> 1;
+  if (tid == 0) {
+    s_ticket = atomicAdd(&ticket[slab * kTicketPitch], 1);
+    ptx::mbar_init(&s_bar, kCompactThreads);
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  const int64_t gt = s_ticket;
   if (gt >= n_tiles) return;
   const int r = batch == 1 ? 0 : find_request(cu, batch, gt);
   const int start = cu[r], N = cu[r + 1] - start;
@@ -118,34 +126,26 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   const uint32_t m_last = mask[woff + lastw];
   // a head that keeps every key moves nothing, and none of its tiles waits for another
   if (kept_all == N) return;
-  if (tid < kCompactTile && (tid >> 5) < words) {
-    const int b = tid & 31;
-    if ((mw >> b) & 1u) s_src[(pw - dst0) + __popc(mw & ((1u << b) - 1u))] = t * kCompactTile + tid;
-  }
   const int cnt = p_last - dst0 + __popc(m_last);
-  __syncthreads();
-  const int pieces = d_k / 8;                       // 16-byte pieces per row
-  // rows whose destination equals their source need no move; they form a prefix of the tile
-  // exactly when nothing was dropped before them: dst0 + i == src_i.
-  // All of a thread's pieces are requested before any is waited for (asynchronous copies straight
-  // into shared memory); (row, piece) advance without divisions.
-  const int step_i = kCompactThreads / pieces, step_pc = kCompactThreads % pieces;
-  {
-    int i = tid / pieces, pc = tid % pieces;
-    for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
-      const int src = s_src[i];
-      if (src != dst0 + i) {
-        const uint32_t dst_s = static_cast<uint32_t>(__cvta_generic_to_shared(&rows_sm[idx]));
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_s), "l"(base + (int64_t)src * tok + pc * 8)
-                     : "memory");
-      }
-      i += step_i;
-      pc += step_pc;
-      if (pc >= pieces) { pc -= pieces; ++i; }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+
+  // Thread = token.  A kept token whose destination differs from its source (the rows that stay
+  // put form a prefix of the slab) is fetched with one bulk copy of the whole row into the slot of
+  // its rank; every thread arrives on the mbarrier, the fetching ones with their byte count.
+  const uint32_t row_bytes = (uint32_t)d_k * 2u;
+  const int b = tid & 31;
+  const bool kept = (tid >> 5) < words && ((mw >> b) & 1u);
+  const int rank = (pw - dst0) + __popc(mw & ((1u << b) - 1u));
+  const int src = t * kCompactTile + tid;
+  const bool moves = kept && src != dst0 + rank;
+  uint8_t* slot = rows_sm + (size_t)rank * row_bytes;
+  if (moves) {
+    ptx::mbar_arrive_expect_tx(&s_bar, row_bytes);
+    ptx::bulk_load(slot, base + (int64_t)src * tok, row_bytes, &s_bar);
+  } else {
+    ptx::mbar_arrive(&s_bar);
   }
+  bool landed = ptx::mbar_wait(&s_bar, 0);
+  if (!landed) landed = ptx::mbar_wait(&s_bar, 0);          // the copies are in flight: do not leave under them
   __syncthreads();
   if (tid == 0) {
     __threadfence();
@@ -167,17 +167,13 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
     }
     s_ok = ok;
   }
+  if (!landed) { atomicExch(&status[0], GVOTE_ERR_TIMEOUT); atomicExch(&status[1], 4); }
   __syncthreads();
-  if (!s_ok) return;
-  {
-    int i = tid / pieces, pc = tid % pieces;
-    for (int idx = tid; idx < cnt * pieces; idx += kCompactThreads) {
-      if (s_src[i] != dst0 + i)
-        *reinterpret_cast<uint4*>(base + (int64_t)(dst0 + i) * tok + pc * 8) = rows_sm[idx];
-      i += step_i;
-      pc += step_pc;
-      if (pc >= pieces) { pc -= pieces; ++i; }
-    }
+  if (!s_ok || !landed) return;
+  if (moves) {
+    ptx::bulk_store(base + (int64_t)(dst0 + rank) * tok, slot, row_bytes);
+    ptx::bulk_commit();
+    ptx::bulk_wait_read<0>();                       // shared memory must outlive the copy's reads
   }
 }
 
