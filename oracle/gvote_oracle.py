@@ -288,6 +288,29 @@ def compact(K: np.ndarray, V: np.ndarray, mask: np.ndarray):
     return Kc, Vc
 
 
+def pack_varlen(K: np.ndarray, V: np.ndarray, cu_seqlens: np.ndarray, masks: Sequence[np.ndarray]):
+    """Section 3.4 of the paper hands the per-head, non-uniform caches to a variable-length
+    attention kernel: every (request, KV head) pair becomes one "sequence" of its kept rows.
+
+    K, V [H_kv, T, d_k] (any dtype; moved, not computed on), requests packed along T by
+    cu_seqlens; masks[r] [H_kv, N_r] bool.  Returns (K_packed, V_packed, cu_seqlens_k):
+    K_packed [total_kept, d_k] holds sequence s = r * H_kv + h at rows
+    cu_seqlens_k[s] .. cu_seqlens_k[s+1]-1, kept rows in ascending index order."""
+    H_kv, d_k = K.shape[0], K.shape[2]
+    parts_k, parts_v, lens = [], [], []
+    for r in range(len(cu_seqlens) - 1):
+        a, b = int(cu_seqlens[r]), int(cu_seqlens[r + 1])
+        for kh in range(H_kv):
+            idx = np.nonzero(masks[r][kh])[0]
+            parts_k.append(K[kh, a:b][idx])
+            parts_v.append(V[kh, a:b][idx])
+            lens.append(idx.shape[0])
+    cu_k = np.zeros(len(lens) + 1, dtype=np.int64)
+    cu_k[1:] = np.cumsum(lens)
+    empty = np.zeros((0, d_k), dtype=K.dtype)
+    return (np.concatenate(parts_k + [empty], axis=0), np.concatenate(parts_v + [empty.astype(V.dtype)], axis=0), cu_k)
+
+
 def compress_request(h: np.ndarray, W_q: np.ndarray, b_q: Optional[np.ndarray], K: np.ndarray,
                      *, n_q_heads: int, d_k: int, theta: float, S: int, p_nuc: float, n_f: int,
                      n_s: int, seed: int, layer_id: int, request_id: int,

@@ -438,3 +438,41 @@ def test_compress_layer_ragged_requests_are_independent():
             assert Kc[r][kh].shape[0] == res[r].budget[kh]
             assert np.array_equal(Kc[r][kh], li.K[kh, a:b][res[r].mask[kh]])
             assert np.array_equal(Vc[r][kh], li.V[kh, a:b][res[r].mask[kh]])
+
+
+# ----------------------------------------------------------------------------- varlen packing
+def test_pack_varlen_hand_example():
+    # two requests (3 and 2 tokens), two heads, d_k = 1: rows are labelled head * 100 + token
+    K = np.array([[[0], [1], [2], [3], [4]], [[100], [101], [102], [103], [104]]], dtype=np.int32)
+    V = K + 1000
+    cu = np.array([0, 3, 5])
+    masks = [np.array([[1, 0, 1], [0, 0, 0]], bool), np.array([[0, 1], [1, 1]], bool)]
+    Kp, Vp, cu_k = o.pack_varlen(K, V, cu, masks)
+    assert Kp[:, 0].tolist() == [0, 2, 4, 103, 104]          # (r0,h0) (r0,h1: none) (r1,h0) (r1,h1)
+    assert Vp[:, 0].tolist() == [1000, 1002, 1004, 1103, 1104]
+    assert cu_k.tolist() == [0, 2, 2, 3, 5]
+
+
+def test_pack_varlen_slices_are_the_compacted_heads_and_identity():
+    rng = np.random.default_rng(21)
+    H, d = 3, 4
+    lens = [7, 1, 12]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    K = rng.integers(0, 1000, size=(H, cu[-1], d))
+    V = rng.integers(0, 1000, size=(H, cu[-1], d))
+    masks = [rng.random((H, n)) < 0.5 for n in lens]
+    Kp, Vp, cu_k = o.pack_varlen(K, V, cu, masks)
+    assert cu_k[-1] == sum(int(m.sum()) for m in masks) == Kp.shape[0] == Vp.shape[0]
+    for r, n in enumerate(lens):
+        Kc, Vc = o.compact(K[:, cu[r]:cu[r + 1]], V[:, cu[r]:cu[r + 1]], masks[r])
+        for h in range(H):
+            s = r * H + h
+            assert np.array_equal(Kp[cu_k[s]:cu_k[s + 1]], Kc[h]) and np.array_equal(Vp[cu_k[s]:cu_k[s + 1]], Vc[h])
+    # keeping everything just re-orders the cache request-major, head-minor
+    full = [np.ones((H, n), bool) for n in lens]
+    Kf, _, cu_f = o.pack_varlen(K, V, cu, full)
+    assert np.array_equal(Kf, np.concatenate([K[h, cu[r]:cu[r + 1]] for r in range(3) for h in range(H)]))
+    assert np.array_equal(np.diff(cu_f), np.repeat(lens, H))
+    # keeping nothing gives empty buffers
+    Ke, Ve, cu_e = o.pack_varlen(K, V, cu, [np.zeros((H, n), bool) for n in lens])
+    assert Ke.shape == (0, d) and cu_e.tolist() == [0] * (3 * H + 1)
