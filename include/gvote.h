@@ -176,6 +176,20 @@ GVOTE_API int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t
                       int64_t total_tokens, int64_t max_N, int32_t* budget,
                       void* ws, size_t ws_bytes, void* stream);
 
+/* Section 3.4: the pruned cache in the layout a variable-length attention kernel consumes, written
+ * out of place from the UNPRUNED K and V and the keep-mask (use it instead of gvote_compact when
+ * the engine wants one dense buffer rather than per-head slabs).  "Sequence" s = r * n_kv_heads + h
+ * (request r, KV head h) owns rows cu_seqlens_k[s] .. cu_seqlens_k[s+1]-1 of K_packed and V_packed
+ * ([capacity_rows, d_k] bf16, dense), kept rows in ascending key order; cu_seqlens_k
+ * [batch*n_kv_heads + 1] int32 and budget [batch, n_kv_heads] are written.  The buffers need
+ * cu_seqlens_k[last] rows, at most n_kv_heads * total_tokens; if capacity_rows is smaller than what the
+ * mask keeps, the rows that do not fit are not written and the workspace status word reads
+ * GVOTE_ERR_WORKSPACE_TOO_SMALL (gvote_poll_status).  K and V are not modified. */
+GVOTE_API int32_t gvote_pack(const gvote_params* p, const void* K, const void* V, int64_t tok_stride, int64_t head_stride,
+                   const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch,
+                   int64_t total_tokens, int64_t max_N, void* K_packed, void* V_packed, int64_t capacity_rows,
+                   int32_t* cu_seqlens_k, int32_t* budget, void* ws, size_t ws_bytes, void* stream);
+
 /* Algorithm 1, whole: fit, sample, project, vote, compact for one layer.  The current query's
  * hidden state is the last row of each request in h unless h_last_or_null is given.
  * Outputs: mask, budget, b_step as in gvote_vote; K and V compacted in place. */

@@ -209,6 +209,23 @@ int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t tok_strid
                         total_tokens, max_N, budget, m, (char*)ws, (cudaStream_t)stream);
 }
 
+int32_t gvote_pack(const gvote_params* p, const void* K, const void* V, int64_t tok_stride, int64_t head_stride,
+                   const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                   void* K_packed, void* V_packed, int64_t capacity_rows, int32_t* cu_seqlens_k, int32_t* budget,
+                   void* ws, size_t ws_bytes, void* stream) {
+  PROPAGATE(validate_params(p));
+  PROPAGATE(validate_batch(batch, total_tokens, max_N));
+  REQUIRE_PTR(K); REQUIRE_PTR(V); REQUIRE_PTR(mask); REQUIRE_PTR(cu_seqlens); REQUIRE_PTR(K_packed);
+  REQUIRE_PTR(V_packed); REQUIRE_PTR(cu_seqlens_k); REQUIRE_PTR(budget); REQUIRE_PTR(ws);
+  if (tok_stride < p->d_k || tok_stride % 8 != 0 || head_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  if (capacity_rows < 0) return GVOTE_ERR_INVALID_ARG;
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
+  if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
+  return launch_pack(p, (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens,
+                     batch, total_tokens, max_N, (__nv_bfloat16*)K_packed, (__nv_bfloat16*)V_packed, capacity_rows,
+                     cu_seqlens_k, budget, m, (char*)ws, (cudaStream_t)stream);
+}
+
 int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_stride, const void* h_last_or_null,
                        const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
                        int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens, int32_t batch,

@@ -115,6 +115,11 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
                        const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens,
                        int64_t max_N, int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
 
+int32_t launch_pack(const gvote_params* p, const __nv_bfloat16* K, const __nv_bfloat16* V, int64_t tok, int64_t head,
+                    const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                    __nv_bfloat16* K_packed, __nv_bfloat16* V_packed, int64_t capacity_rows, int32_t* cu_seqlens_k,
+                    int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
+
 // ---------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 

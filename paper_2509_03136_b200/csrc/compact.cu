@@ -179,28 +179,39 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
 
 }  // namespace
 
-int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
-                       const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                       int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st) {
+int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int32_t* cu, int32_t batch,
+                         int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st) {
   const int Hkv = p->n_kv_heads;
   int32_t* prefix = reinterpret_cast<int32_t*>(ws + m.prefix);
   int32_t* flags = reinterpret_cast<int32_t*>(ws + m.flags);
   int32_t* ticket = flags + (size_t)2 * Hkv * m.n_tiles;
-  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
   dim3 gs(Hkv, batch);
   {
     LaunchScope scope_("mask_scan_kernel", st);
-  mask_scan_kernel<<<gs, kScanThreads, 0, st>>>(mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
+    mask_scan_kernel<<<gs, kScanThreads, 0, st>>>(mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
   }
   GVOTE_LAUNCH_CHECK("mask_scan_kernel");
+  return GVOTE_OK;
+}
+
+int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
+                       const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                       int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st) {
+  const int Hkv = p->n_kv_heads;
+  const int32_t* prefix = reinterpret_cast<const int32_t*>(ws + m.prefix);
+  int32_t* flags = reinterpret_cast<int32_t*>(ws + m.flags);
+  int32_t* ticket = flags + (size_t)2 * Hkv * m.n_tiles;
+  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
+  const int32_t rc = launch_mask_scan(p, mask, cu, batch, budget, m, ws, st);
+  if (rc != GVOTE_OK) return rc;
   const size_t smem = (size_t)kCompactTile * p->d_k * sizeof(__nv_bfloat16);
   if (smem > 48 * 1024)
     GVOTE_CUDA_CHECK(cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int64_t ctas = m.n_tiles * 2 * Hkv;
   {
     LaunchScope scope_("compact_kernel", st);
-  compact_kernel<<<(unsigned)ctas, kCompactThreads, smem, st>>>(K, V, tok, head, mask, prefix, cu, budget, batch, Hkv,
-                                                                p->d_k, m.row_words, m.n_tiles, flags, ticket, status);
+    compact_kernel<<<(unsigned)ctas, kCompactThreads, smem, st>>>(K, V, tok, head, mask, prefix, cu, budget, batch, Hkv,
+                                                                  p->d_k, m.row_words, m.n_tiles, flags, ticket, status);
   }
   GVOTE_LAUNCH_CHECK("compact_kernel");
   return GVOTE_OK;

@@ -23,7 +23,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
     "gvote_workspace_bytes", "gvote_fit", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
-    "gvote_compact", "gvote_compress", "gvote_compress_host", "gvote_host_arena_release",
+    "gvote_compact", "gvote_pack", "gvote_compress", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
@@ -74,6 +74,8 @@ def load():
     lib.gvote_select.argtypes = [P, vp, vp, vp, i64, vp, vp, i64, i64, vp, i32, i64, i64, vp, vp, vp, vp, vp, sz, vp]
     lib.gvote_compact.restype = i32
     lib.gvote_compact.argtypes = [P, vp, vp, i64, i64, vp, vp, i32, i64, i64, vp, vp, sz, vp]
+    lib.gvote_pack.restype = i32
+    lib.gvote_pack.argtypes = [P, vp, vp, i64, i64, vp, vp, i32, i64, i64, vp, vp, i64, vp, vp, vp, sz, vp]
     lib.gvote_compress.restype = i32
     lib.gvote_compress.argtypes = [P, vp, i64, vp, vp, i64, vp, vp, vp, i64, i64, vp, i32, i64, i64, vp, vp, vp,
                                    vp, sz, vp]
@@ -226,6 +228,20 @@ def gvote_compact(p, K, V, mask, cu_seqlens, geom, budget, ws) -> None:
     _check(load().gvote_compact(ctypes.byref(p), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(mask),
                                 _ptr(cu_seqlens), batch, total, max_N, _ptr(budget), _ptr(ws), ws.numel(), _stream()),
            "gvote_compact")
+
+
+def gvote_pack(p, K, V, mask, cu_seqlens, geom, K_packed, V_packed, cu_seqlens_k, budget, ws) -> None:
+    batch, total, max_N = geom
+    _dev(K, torch.bfloat16, "K", dense=False); _dev(V, torch.bfloat16, "V", dense=False); _dev(mask, torch.int32, "mask")
+    _dev(K_packed, torch.bfloat16, "K_packed"); _dev(V_packed, torch.bfloat16, "V_packed")
+    _dev(cu_seqlens_k, torch.int32, "cu_seqlens_k"); _dev(budget, torch.int32, "budget")
+    if K.stride() != V.stride():
+        raise ValueError("K and V must share strides")
+    if K_packed.shape != V_packed.shape or K_packed.dim() != 2 or K_packed.shape[1] != p.d_k:
+        raise ValueError("K_packed and V_packed must be [rows, d_k]")
+    _check(load().gvote_pack(ctypes.byref(p), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(mask), _ptr(cu_seqlens),
+                             batch, total, max_N, _ptr(K_packed), _ptr(V_packed), K_packed.shape[0],
+                             _ptr(cu_seqlens_k), _ptr(budget), _ptr(ws), ws.numel(), _stream()), "gvote_pack")
 
 
 def gvote_compress(p, h, W_q, b_q, K, V, cu_seqlens, geom, mask, budget, b_step, ws, h_last=None) -> None:

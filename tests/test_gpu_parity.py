@@ -323,6 +323,68 @@ def test_compact_strided_heads(gv):
         assert np.array_equal(out[0, :n, h], base[0, keep[h], h]) and np.array_equal(out[1, :n, h], base[1, keep[h], h])
 
 
+# ----------------------------------------------------------------------------- varlen packing
+@pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
+                                                  ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
+                                                  ((1000,), 1, 8, 1.0), ((1000, 77), 2, 16, 0.0)])
+def test_pack_varlen_bit_exact(gv, lens, Hkv, d_k, density):
+    """gvote_pack against the oracle's packing, bit for bit, with K and V left untouched."""
+    rng = np.random.default_rng(31)
+    T, B = sum(lens), len(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    K = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
+    V = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
+    keep = rng.random((Hkv, T)) < density
+    words = np.zeros((Hkv, gv.mask_row_words(T, B)), dtype=np.uint32)
+    for r in range(B):
+        for h in range(Hkv):
+            w = o.pack_mask_bits(keep[h, cu[r]:cu[r + 1]])
+            off = gv.mask_word_offset(int(cu[r]), r)
+            words[h, off:off + len(w)] = w
+    Ko, Vo, cu_k = o.pack_varlen(K, V, cu, [keep[:, cu[r]:cu[r + 1]] for r in range(B)])
+    p = gv.make_params(d_h=64, n_q_heads=Hkv, n_kv_heads=Hkv, d_k=d_k, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=0,
+                       seed=0)
+    geom = (B, T, max(lens))
+    ws = gv.alloc_workspace(p, *geom)
+    Kd, Vd = gv.bf16_from_bits(K), gv.bf16_from_bits(V)
+    rows = max(int(cu_k[-1]), 1)
+    Kp = torch.zeros(rows, d_k, dtype=torch.bfloat16, device="cuda"); Vp = torch.zeros_like(Kp)
+    cuk = torch.full((B * Hkv + 1,), -1, dtype=torch.int32, device="cuda")
+    budget = torch.empty(B, Hkv, dtype=torch.int32, device="cuda")
+    md = torch.from_numpy(words.view(np.int32)).cuda()
+    for rep in range(2):
+        gv.gvote_pack(p, Kd, Vd, md, torch.from_numpy(cu).cuda(), geom, Kp, Vp, cuk, budget, ws)
+        assert gv.gvote_poll_status(ws) == 0
+        assert np.array_equal(cuk.cpu().numpy(), cu_k)
+        assert np.array_equal(budget.cpu().numpy().ravel(), np.diff(cu_k))
+        n = int(cu_k[-1])
+        assert np.array_equal(gv.bits_from_bf16(Kp)[:n], Ko) and np.array_equal(gv.bits_from_bf16(Vp)[:n], Vo)
+        assert np.array_equal(gv.bits_from_bf16(Kd), K) and np.array_equal(gv.bits_from_bf16(Vd), V)
+
+
+def test_pack_varlen_reports_buffers_that_are_too_small(gv):
+    rng = np.random.default_rng(32)
+    T, Hkv, d_k = 600, 2, 32
+    K = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
+    keep = np.ones((Hkv, T), dtype=bool)
+    words = np.stack([np.concatenate([o.pack_mask_bits(keep[h]), np.zeros(1, np.uint32)]) for h in range(Hkv)])
+    words = words[:, :gv.mask_row_words(T, 1)]
+    p = gv.make_params(d_h=64, n_q_heads=Hkv, n_kv_heads=Hkv, d_k=d_k, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=0,
+                       seed=0)
+    geom = (1, T, T)
+    ws = gv.alloc_workspace(p, *geom)
+    Kd = gv.bf16_from_bits(K)
+    Kp = torch.zeros(700, d_k, dtype=torch.bfloat16, device="cuda"); Vp = torch.zeros_like(Kp)   # 1200 rows are kept
+    cuk = torch.empty(Hkv + 1, dtype=torch.int32, device="cuda")
+    budget = torch.empty(1, Hkv, dtype=torch.int32, device="cuda")
+    gv.gvote_pack(p, Kd, Kd, torch.from_numpy(np.ascontiguousarray(words).view(np.int32)).cuda(),
+                  torch.tensor([0, T], dtype=torch.int32, device="cuda"), geom, Kp, Vp, cuk, budget, ws)
+    assert gv.gvote_poll_status(ws) == -3
+    assert cuk.cpu().numpy().tolist() == [0, 600, 1200]
+    assert np.array_equal(gv.bits_from_bf16(Kp)[:600], K[0])          # what fits is written
+    ws.zero_()
+
+
 # ----------------------------------------------------------------------------- whole pass
 def _run_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
     p = gv.params_from_config(cfg, layer_id=layer_id, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0)
