@@ -131,6 +131,47 @@ def fit(h: np.ndarray, n_s: int) -> Tuple[np.ndarray, np.ndarray]:
     return mu, var
 
 
+@dataclass
+class FitState:
+    """Running moments of the hidden states seen so far (per channel): count, mean and the sum of
+    squared deviations from the mean."""
+    n: int
+    mean: np.ndarray
+    m2: np.ndarray
+
+
+def fit_state(rows: np.ndarray) -> FitState:
+    """Moments of a block of hidden-state rows [T, d_h] (T may be 0)."""
+    x = np.asarray(rows, dtype=np.float64)
+    T = x.shape[0]
+    if T == 0:
+        z = np.zeros(x.shape[1])
+        return FitState(0, z, z.copy())
+    mean = x.sum(axis=0) / T
+    d = x - mean
+    return FitState(T, mean, (d * d).sum(axis=0))
+
+
+def fit_merge(a: FitState, b: FitState) -> FitState:
+    """Moments of the union of two disjoint blocks from their moments (the pairwise update of
+    Chan, Golub and LeVeque): the Gaussian of Step 2 can be fitted while the prompt streams by,
+    block by block, without keeping the hidden states."""
+    if a.n == 0:
+        return FitState(b.n, b.mean.copy(), b.m2.copy())
+    if b.n == 0:
+        return FitState(a.n, a.mean.copy(), a.m2.copy())
+    n = a.n + b.n
+    delta = b.mean - a.mean
+    return FitState(n, a.mean + delta * (b.n / n), a.m2 + b.m2 + delta * delta * (a.n * b.n / n))
+
+
+def fit_finish(s: FitState) -> Tuple[np.ndarray, np.ndarray]:
+    """Step 2's (mu, unbiased variance) from running moments."""
+    if s.n < 2:
+        raise ValueError("fit needs at least two rows")
+    return s.mean.copy(), s.m2 / (s.n - 1)
+
+
 # ----------------------------------------------------------------------------- Step 3: sample
 def sample(mu: np.ndarray, var: np.ndarray, S: int, seed: int, layer_id: int,
            request_id: int) -> Tuple[np.ndarray, np.ndarray]:

@@ -476,3 +476,34 @@ def test_pack_varlen_slices_are_the_compacted_heads_and_identity():
     # keeping nothing gives empty buffers
     Ke, Ve, cu_e = o.pack_varlen(K, V, cu, [np.zeros((H, n), bool) for n in lens])
     assert Ke.shape == (0, d) and cu_e.tolist() == [0] * (3 * H + 1)
+
+
+# ----------------------------------------------------------------------------- streaming fit
+def test_fit_merge_equals_fit_of_the_concatenation():
+    rng = np.random.default_rng(41)
+    h = rng.normal(size=(97, 6)) * rng.uniform(0.1, 5, size=6) + rng.normal(size=6) * 20
+    n_s = 4
+    cuts = [n_s, 10, 11, 50, 97]                                  # uneven blocks, one of a single row
+    st = o.fit_state(h[0:0])
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        st = o.fit_merge(st, o.fit_state(h[a:b]))
+    mu, var = o.fit_finish(st)
+    assert st.n == 97 - n_s
+    assert np.allclose(mu, h[n_s:].mean(axis=0), rtol=1e-13) and np.allclose(var, h[n_s:].var(axis=0, ddof=1), rtol=1e-12)
+    mu2, var2 = o.fit(h, n_s)                                     # the one-shot fit of Step 2
+    assert np.allclose(mu, mu2, rtol=1e-13) and np.allclose(var, var2, rtol=1e-12)
+
+
+def test_fit_merge_is_symmetric_and_has_an_identity():
+    rng = np.random.default_rng(42)
+    A, B = rng.normal(size=(5, 3)), rng.normal(size=(9, 3)) + 3
+    ab, ba = o.fit_merge(o.fit_state(A), o.fit_state(B)), o.fit_merge(o.fit_state(B), o.fit_state(A))
+    assert ab.n == ba.n == 14 and np.allclose(ab.mean, ba.mean, rtol=1e-14) and np.allclose(ab.m2, ba.m2, rtol=1e-13)
+    e = o.fit_state(A[0:0])
+    same = o.fit_merge(e, o.fit_state(A))
+    assert same.n == 5 and np.array_equal(same.mean, o.fit_state(A).mean) and np.array_equal(same.m2, o.fit_state(A).m2)
+    # two blocks of one row each: variance of two points is (x - y)^2 / 2
+    two = o.fit_merge(o.fit_state(A[:1]), o.fit_state(A[1:2]))
+    assert np.allclose(o.fit_finish(two)[1], (A[0] - A[1]) ** 2 / 2, rtol=1e-13)
+    with pytest.raises(ValueError):
+        o.fit_finish(o.fit_state(A[:1]))
