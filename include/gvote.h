@@ -105,6 +105,23 @@ GVOTE_API int32_t gvote_fit(const gvote_params* p, const void* h, int64_t h_row_
                   const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
                   float* mu, float* var, void* ws, size_t ws_bytes, void* stream);
 
+/* Step 2 while the prompt streams by (the Gaussian needs only running moments, not the hidden states:
+ * an engine can feed each prefill chunk's layer-norm output and drop it, which takes the fit's read of
+ * all hidden states out of the compression pass).
+ * state: [batch, 3, d_h] double, zero-filled before the first block; per request and channel it
+ * holds the number of rows seen, their mean and their sum of squared deviations.
+ * gvote_fit_update folds one block of rows into the state: h_block [total_rows, d_h] holds the new rows
+ * of every request, request r owning rows cu_block[r] .. cu_block[r+1]-1 (a request may have none).
+ * Every row given is counted: leaving out the n_s sink tokens is the caller's doing here (p->n_s is not
+ * used).  Blocks are merged with the pairwise update of Chan, Golub and LeVeque in fp64.
+ * gvote_fit_finish turns the state into mu and the unbiased variance (NaN below two rows), the inputs
+ * of gvote_sample and gvote_compress_moments. */
+GVOTE_API int32_t gvote_fit_update(const gvote_params* p, const void* h_block, int64_t h_row_stride,
+                         const int32_t* cu_block, int32_t batch, int64_t total_rows, int64_t max_rows,
+                         double* state, void* ws, size_t ws_bytes, void* stream);
+GVOTE_API int32_t gvote_fit_finish(const gvote_params* p, const double* state, int32_t batch,
+                         float* mu, float* var, void* stream);
+
 /* Fit without any allocation (the paper has no counterpart: this entry point exists for the
  * integration, not for the method).  Same result as gvote_fit, but the per-chunk partial moments
  * live in a fixed 1 MiB array inside the library's device image (GVOTE_FIT_STATIC_MAX_ENTRIES
@@ -199,6 +216,16 @@ GVOTE_API int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h
                        const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
                        uint32_t* mask, int32_t* budget, int32_t* b_step,
                        void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 from line 5 on, for a caller that already has the Gaussian (gvote_fit_finish): sample,
+ * project, vote, compact.  mu, var [batch, d_h] float; h_last [batch, d_h] of p->h_dtype is the current
+ * query's hidden state.  Other arguments and outputs as in gvote_compress. */
+GVOTE_API int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                               const void* W_q, int64_t wq_ld, const float* b_q_or_null,
+                               void* K, void* V, int64_t tok_stride, int64_t head_stride,
+                               const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
+                               uint32_t* mask, int32_t* budget, int32_t* b_step,
+                               void* ws, size_t ws_bytes, void* stream);
 
 /* The same pass for a caller whose tensors live in HOST memory (pinned memory gives full copy
  * speed): all pointers are host pointers, K and V are dense ([n_kv_heads, total_tokens, d_k]),

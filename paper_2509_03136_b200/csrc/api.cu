@@ -209,6 +209,53 @@ int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t tok_strid
                         total_tokens, max_N, budget, m, (char*)ws, (cudaStream_t)stream);
 }
 
+int32_t gvote_fit_update(const gvote_params* p, const void* h_block, int64_t h_row_stride,
+                         const int32_t* cu_block, int32_t batch, int64_t total_rows, int64_t max_rows, double* state,
+                         void* ws, size_t ws_bytes, void* stream) {
+  PROPAGATE(validate_params(p));
+  PROPAGATE(validate_batch(batch, total_rows, max_rows));
+  REQUIRE_PTR(h_block); REQUIRE_PTR(cu_block); REQUIRE_PTR(state); REQUIRE_PTR(ws);
+  if (h_row_stride < p->d_h || h_row_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  const WorkspaceMap m = workspace_map(p, batch, total_rows, max_rows);
+  if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
+  return launch_fit_state_update(p, h_block, h_row_stride, cu_block, batch, m.fit_chunks,
+                                 reinterpret_cast<float2*>((char*)ws + m.fit_partial), state, (cudaStream_t)stream);
+}
+
+int32_t gvote_fit_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
+                         void* stream) {
+  PROPAGATE(validate_params(p));
+  if (batch < 1) return GVOTE_ERR_INVALID_ARG;
+  REQUIRE_PTR(state); REQUIRE_PTR(mu); REQUIRE_PTR(var);
+  return launch_fit_state_finish(p, state, batch, mu, var, (cudaStream_t)stream);
+}
+
+int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                               const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
+                               int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens, int32_t batch,
+                               int64_t total_tokens, int64_t max_N, uint32_t* mask, int32_t* budget, int32_t* b_step,
+                               void* ws, size_t ws_bytes, void* stream) {
+  PROPAGATE(validate_params(p));
+  PROPAGATE(validate_batch(batch, total_tokens, max_N));
+  REQUIRE_PTR(mu); REQUIRE_PTR(var); REQUIRE_PTR(h_last); REQUIRE_PTR(W_q); OPTIONAL_PTR(b_q_or_null); REQUIRE_PTR(K);
+  REQUIRE_PTR(V); REQUIRE_PTR(cu_seqlens); REQUIRE_PTR(mask); REQUIRE_PTR(budget); REQUIRE_PTR(b_step);
+  REQUIRE_PTR(ws);
+  if (wq_ld < p->d_h || wq_ld % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  if (tok_stride < p->d_k || tok_stride % 8 != 0 || head_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
+  if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
+  char* w = (char*)ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* Ht = reinterpret_cast<float*>(w + m.h_tilde);
+  __nv_bfloat16* Q = reinterpret_cast<__nv_bfloat16*>(w + m.q_bf16);
+  PROPAGATE(launch_sample(p, mu, var, batch, Ht, nullptr, st));
+  PROPAGATE(launch_project(p, Ht, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q, st));
+  PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
+                        max_N, mask, nullptr, b_step, nullptr, m, w, st));
+  return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
+                        total_tokens, max_N, budget, m, w, st);
+}
+
 int32_t gvote_pack(const gvote_params* p, const void* K, const void* V, int64_t tok_stride, int64_t head_stride,
                    const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
                    void* K_packed, void* V_packed, int64_t capacity_rows, int32_t* cu_seqlens_k, int32_t* budget,

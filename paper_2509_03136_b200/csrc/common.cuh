@@ -91,6 +91,10 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
                    int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st);
 int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
                            int fit_chunks, float2* partial, cudaStream_t st);
+int32_t launch_fit_state_update(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                                int fit_chunks, float2* partial, double* state, cudaStream_t st);
+int32_t launch_fit_state_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
+                                cudaStream_t st);
 int32_t launch_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch,
                       float* H_tilde, uint32_t* raw, cudaStream_t st);
 // Fused middle of the whole pass: merges the fit partials (mu, var), draws the S samples and writes

@@ -119,6 +119,52 @@ fit_finalize_kernel(const float2* __restrict__ partial, const int32_t* __restric
   }
 }
 
+// ---------------------------------------------------------------------------------- streaming fit
+// Running moments per request and channel, fp64: state[r][0][c] = rows seen, [1][c] = mean, [2][c] =
+// sum of squared deviations.  One block of rows is reduced by fit_partial_kernel as usual; this kernel
+// merges the block's chunks and folds them into the state with the pairwise update of Chan, Golub
+// and LeVeque.
+__global__ void __launch_bounds__(256)
+fit_state_update_kernel(const float2* __restrict__ partial, const int32_t* __restrict__ cu, int d_h, int chunks,
+                        double* __restrict__ state) {
+  __shared__ FitMoments sm[8][32];
+  const int r = blockIdx.y;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int col = blockIdx.x * 32 + tx;
+  const int first = cu[r], last = cu[r + 1];
+  FitMoments acc{0.0, 0.0, 0.0};
+  double ref = 0.0;
+  if (col < d_h && last > first) {
+    ref = (double)partial[((int64_t)r * chunks) * d_h + col].x;
+    acc = fit_merge_lane(partial, r, chunks, d_h, col, first, last, ty, 8, ref);
+  }
+  sm[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && col < d_h && last > first) {
+    for (int j = 1; j < 8; ++j) { acc.n += sm[j][tx].n; acc.a += sm[j][tx].a; acc.bc += sm[j][tx].bc; }
+    const double nb = acc.n, mean_b = ref + acc.a / acc.n, m2_b = fmax(acc.bc - acc.a * acc.a / acc.n, 0.0);
+    double* st = state + (int64_t)r * 3 * d_h;
+    const double na = st[col];
+    if (na <= 0.0) {
+      st[col] = nb; st[d_h + col] = mean_b; st[2 * d_h + col] = m2_b;
+    } else {
+      const double n = na + nb, delta = mean_b - st[d_h + col];
+      st[col] = n;
+      st[d_h + col] += delta * (nb / n);
+      st[2 * d_h + col] += m2_b + delta * delta * (na * nb / n);
+    }
+  }
+}
+
+__global__ void fit_state_finish_kernel(const double* __restrict__ state, int d_h, float* __restrict__ mu,
+                                        float* __restrict__ var) {
+  const int r = blockIdx.y, col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= d_h) return;
+  const double* st = state + (int64_t)r * 3 * d_h;
+  mu[(int64_t)r * d_h + col] = (float)st[d_h + col];
+  var[(int64_t)r * d_h + col] = (float)(st[2 * d_h + col] / (st[col] - 1.0));   // NaN/inf below two rows
+}
+
 }  // namespace
 
 int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
@@ -148,6 +194,32 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
     fit_finalize_kernel<<<g2, 256, 0, st>>>(partial, cu, p->n_s, p->d_h, fit_chunks, mu, var);
   }
   GVOTE_LAUNCH_CHECK("fit_finalize_kernel");
+  return GVOTE_OK;
+}
+
+int32_t launch_fit_state_update(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
+                                int fit_chunks, float2* partial, double* state, cudaStream_t st) {
+  gvote_params q = *p;
+  q.n_s = 0;                                   // which rows to leave out is the caller's choice here
+  const int32_t rc = launch_fit_partial(&q, h, ld, cu, batch, fit_chunks, partial, st);
+  if (rc != GVOTE_OK) return rc;
+  dim3 g2((unsigned)ceil_div(p->d_h, 32), batch);
+  {
+    LaunchScope scope_("fit_state_update_kernel", st);
+    fit_state_update_kernel<<<g2, 256, 0, st>>>(partial, cu, p->d_h, fit_chunks, state);
+  }
+  GVOTE_LAUNCH_CHECK("fit_state_update_kernel");
+  return GVOTE_OK;
+}
+
+int32_t launch_fit_state_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
+                                cudaStream_t st) {
+  dim3 g((unsigned)ceil_div(p->d_h, 256), batch);
+  {
+    LaunchScope scope_("fit_state_finish_kernel", st);
+    fit_state_finish_kernel<<<g, 256, 0, st>>>(state, p->d_h, mu, var);
+  }
+  GVOTE_LAUNCH_CHECK("fit_state_finish_kernel");
   return GVOTE_OK;
 }
 

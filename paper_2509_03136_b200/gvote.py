@@ -22,8 +22,8 @@ SEL_TOPK_C0, SEL_TOPP = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
-    "gvote_workspace_bytes", "gvote_fit", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
-    "gvote_compact", "gvote_pack", "gvote_compress", "gvote_compress_host", "gvote_host_arena_release",
+    "gvote_workspace_bytes", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
+    "gvote_compact", "gvote_pack", "gvote_compress", "gvote_compress_moments", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
@@ -62,6 +62,13 @@ def load():
     lib.gvote_workspace_bytes.argtypes = [P, i32, i64, i64]
     lib.gvote_fit.restype = i32
     lib.gvote_fit.argtypes = [P, vp, i64, vp, i32, i64, i64, vp, vp, vp, sz, vp]
+    lib.gvote_fit_update.restype = i32
+    lib.gvote_fit_update.argtypes = [P, vp, i64, vp, i32, i64, i64, vp, vp, sz, vp]
+    lib.gvote_fit_finish.restype = i32
+    lib.gvote_fit_finish.argtypes = [P, vp, i32, vp, vp, vp]
+    lib.gvote_compress_moments.restype = i32
+    lib.gvote_compress_moments.argtypes = [P, vp, vp, vp, vp, i64, vp, vp, vp, i64, i64, vp, i32, i64, i64, vp, vp, vp,
+                                           vp, sz, vp]
     lib.gvote_fit_static.restype = i32
     lib.gvote_fit_static.argtypes = [P, vp, i64, vp, i32, i64, vp, vp, vp]
     lib.gvote_sample.restype = i32
@@ -171,6 +178,36 @@ def gvote_fit(p, h, cu_seqlens, geom, mu, var, ws) -> None:
     _dev(cu_seqlens, torch.int32, "cu_seqlens"); _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
     _check(load().gvote_fit(ctypes.byref(p), _ptr(h), h.stride(0), _ptr(cu_seqlens), batch, total, max_N,
                             _ptr(mu), _ptr(var), _ptr(ws), ws.numel(), _stream()), "gvote_fit")
+
+
+def gvote_fit_update(p, h_block, cu_block, geom, state, ws) -> None:
+    """Fold one block of hidden-state rows (requests packed by cu_block) into the running moments
+    `state` [batch, 3, d_h] float64 (zero-filled before the first block)."""
+    batch, total, max_rows = geom
+    _dev(h_block, torch.float32 if p.h_dtype == DTYPE_F32 else torch.bfloat16, "h_block", dense=False)
+    _dev(cu_block, torch.int32, "cu_block"); _dev(state, torch.float64, "state")
+    _check(load().gvote_fit_update(ctypes.byref(p), _ptr(h_block), h_block.stride(0), _ptr(cu_block), batch, total,
+                                   max_rows, _ptr(state), _ptr(ws), ws.numel(), _stream()), "gvote_fit_update")
+
+
+def gvote_fit_finish(p, state, batch, mu, var) -> None:
+    _dev(state, torch.float64, "state"); _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
+    _check(load().gvote_fit_finish(ctypes.byref(p), _ptr(state), batch, _ptr(mu), _ptr(var), _stream()),
+           "gvote_fit_finish")
+
+
+def gvote_compress_moments(p, mu, var, h_last, W_q, b_q, K, V, cu_seqlens, geom, mask, budget, b_step, ws) -> None:
+    batch, total, max_N = geom
+    _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
+    _dev(h_last, torch.float32 if p.h_dtype == DTYPE_F32 else torch.bfloat16, "h_last")
+    _dev(W_q, torch.bfloat16, "W_q", dense=False); _dev(K, torch.bfloat16, "K", dense=False); _dev(V, torch.bfloat16, "V", dense=False)
+    _dev(mask, torch.int32, "mask"); _dev(budget, torch.int32, "budget"); _dev(b_step, torch.int32, "b_step")
+    if K.stride() != V.stride():
+        raise ValueError("K and V must share strides")
+    _check(load().gvote_compress_moments(ctypes.byref(p), _ptr(mu), _ptr(var), _ptr(h_last), _ptr(W_q), W_q.stride(0),
+                                         _ptr(b_q), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(cu_seqlens),
+                                         batch, total, max_N, _ptr(mask), _ptr(budget), _ptr(b_step), _ptr(ws),
+                                         ws.numel(), _stream()), "gvote_compress_moments")
 
 
 FIT_STATIC_MAX_ENTRIES = 131072

@@ -400,11 +400,11 @@ def _run_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
             gv.bits_from_bf16(d["V"]))
 
 
-def _check_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
+def _check_compress(gv, cfg, li, sel_mode="topk", layer_id=0, runner=None):
     """End to end.  The GPU draws its own samples (fp32 fit and Box-Muller), so a few query values
     land on the neighbouring bf16 step; masks are compared inside the score tolerance (2e-2) band
     and budgets to 0.5 % of N.  Compaction is checked bit-exactly against the GPU's own mask."""
-    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li, sel_mode, layer_id)
+    mask, budget, b_step, Kg, Vg = (runner or _run_compress)(gv, cfg, li, sel_mode, layer_id)
     kw = pu.oracle_kwargs(cfg, layer_id)
     res, _, _ = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, sel_mode=sel_mode, **kw)
     pf = kw["p_nuc"]
@@ -432,6 +432,70 @@ def test_compress_small(gv, idx):
 def test_compress_configs(gv, name, mode):
     cfg = synth.make_config(name)
     _check_compress(gv, cfg, synth.make_layer(cfg, 0), mode)
+
+
+# ----------------------------------------------------------------------------- streaming fit
+def _stream_fit(gv, p, cfg, li, n_blocks, rng):
+    """Feed every request's rows after the sinks in n_blocks uneven blocks; returns (mu, var) tensors."""
+    cu = li.cu_seqlens
+    B = cfg.batch
+    state = torch.zeros(B, 3, cfg.d_h, dtype=torch.float64, device="cuda")
+    cuts = []
+    for r in range(B):
+        a, b = int(cu[r]) + cfg.n_s, int(cu[r + 1])
+        inner = np.sort(rng.integers(a, b + 1, size=n_blocks - 1))
+        cuts.append(np.concatenate([[a], inner, [b]]))
+    for k in range(n_blocks):
+        rows = [li.h[cuts[r][k]:cuts[r][k + 1]] for r in range(B)]
+        lens = [x.shape[0] for x in rows]
+        if sum(lens) == 0:
+            continue
+        block = torch.from_numpy(np.concatenate(rows)).cuda()
+        cub = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).cuda()
+        geom = (B, sum(lens), max(lens))
+        ws = gv.alloc_workspace(p, *geom)
+        gv.gvote_fit_update(p, block, cub, geom, state, ws)
+    mu = torch.empty(B, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit_finish(p, state, B, mu, var)
+    return mu, var
+
+
+@pytest.mark.parametrize("idx,n_blocks", [(0, 1), (1, 3), (2, 4), (3, 7)])
+def test_streaming_fit_matches_one_shot_fit(gv, idx, n_blocks):
+    """Moments accumulated block by block (Chan merge, fp64 state) against the oracle's one-shot fit:
+    1e-5 relative on the variance, 1e-5 of the largest standard deviation on the mean."""
+    cfg = _small_cfgs()[idx]
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg)
+    mu, var = _stream_fit(gv, p, cfg, li, n_blocks, np.random.default_rng(50 + idx))
+    for r in range(cfg.batch):
+        m, v = o.fit(li.h[li.cu_seqlens[r]:li.cu_seqlens[r + 1]], cfg.n_s)
+        assert np.allclose(var[r].cpu().numpy(), v, rtol=1e-5, atol=0)
+        assert np.abs(mu[r].cpu().numpy() - m).max() <= 1e-5 * np.sqrt(v).max() + 1e-6 * np.abs(m).max()
+
+
+def _run_compress_moments(gv, cfg, li, sel_mode="topk", layer_id=0):
+    p = gv.params_from_config(cfg, layer_id=layer_id, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mu, var = _stream_fit(gv, p, cfg, li, 3, np.random.default_rng(60))
+    h_last = torch.from_numpy(np.stack([li.h[int(li.cu_seqlens[r + 1]) - 1] for r in range(cfg.batch)])).cuda()
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_compress_moments(p, mu, var, h_last, d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget,
+                              b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
+            gv.bits_from_bf16(d["V"]))
+
+
+@pytest.mark.parametrize("name", ["small2", "c0", "c1", "c3"])
+def test_compress_from_streamed_moments(gv, name):
+    """The pass with the Gaussian fitted upstream, block by block, against the oracle's whole pass."""
+    cfg = _small_cfgs()[2] if name == "small2" else synth.make_config(name)
+    _check_compress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(name == "small2")), runner=_run_compress_moments)
 
 
 def test_compress_is_deterministic(gv):
