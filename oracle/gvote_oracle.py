@@ -318,6 +318,20 @@ def vote(Q: np.ndarray, K: np.ndarray, *, p_nuc: float, sel_mode: str = "topk",
     return mask, budget, b_step, row_sets, probs
 
 
+def attention_overlap(Q: np.ndarray, K: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """Section 3.3's yardstick, applied to the pass's own output: the share of the current query's
+    attention (softmax weights of Eq. 1) that falls on the keys the pass keeps, per query head.
+    Q [H_q, S+1, d_k] (row 0 of each head is the current query), K [H_kv, N, d_k], mask [H_kv, N]."""
+    H_q, _, d_k = Q.shape
+    G = H_q // K.shape[0]
+    out = np.zeros(H_q)
+    for g in range(H_q):
+        kh = g // G
+        a0 = softmax_rows((Q[g, :1] @ K[kh].T) / math.sqrt(d_k))[0]
+        out[g] = a0[mask[kh]].sum()
+    return out
+
+
 def compact(K: np.ndarray, V: np.ndarray, mask: np.ndarray):
     """Algorithm 1 line 11: keep the rows of the keep-set, in ascending index order.
     K, V [H_kv, N, d_k] (any dtype; moved, not computed on); returns lists per head."""

@@ -507,3 +507,29 @@ def test_fit_merge_is_symmetric_and_has_an_identity():
     assert np.allclose(o.fit_finish(two)[1], (A[0] - A[1]) ** 2 / 2, rtol=1e-13)
     with pytest.raises(ValueError):
         o.fit_finish(o.fit_state(A[:1]))
+
+
+# ----------------------------------------------------------------------------- attention overlap
+def test_attention_overlap_special_cases():
+    rng = np.random.default_rng(51)
+    H_q, H_kv, S1, d_k, N = 4, 2, 3, 8, 50
+    Q = rng.normal(size=(H_q, S1, d_k)) * 2
+    K = rng.normal(size=(H_kv, N, d_k))
+    ones, none = np.ones((H_kv, N), bool), np.zeros((H_kv, N), bool)
+    assert np.allclose(o.attention_overlap(Q, K, ones), 1.0, rtol=1e-14) and np.all(o.attention_overlap(Q, K, none) == 0)
+    m = rng.random((H_kv, N)) < 0.4
+    assert np.allclose(o.attention_overlap(Q, K, m) + o.attention_overlap(Q, K, ~m), 1.0, rtol=1e-13)   # additivity
+    # keeping exactly the top-p set of the current query keeps at least p of its attention, and
+    # dropping that set's last key falls below p (minimality)
+    for g in range(H_q):
+        kh = g // 2
+        a0 = o.softmax_rows((Q[g, :1] @ K[kh].T) / math.sqrt(d_k))[0]
+        C0 = o.top_p_set(a0, 0.9)
+        mk = none.copy(); mk[kh, C0] = True
+        assert o.attention_overlap(Q, K, mk)[g] >= 0.9
+        mk[kh, C0[-1]] = False
+        assert o.attention_overlap(Q, K, mk)[g] < 0.9
+    # by hand: two keys with logits 0 and ln 3 -> weights 1/4 and 3/4
+    Q1 = np.zeros((1, 1, 4)); Q1[0, 0, 0] = 2.0
+    K1 = np.zeros((1, 2, 4)); K1[0, 1, 0] = math.log(3.0)         # logit = 2 * ln3 / sqrt(4) = ln 3
+    assert o.attention_overlap(Q1, K1, np.array([[False, True]]))[0] == pytest.approx(0.75, rel=1e-14)
