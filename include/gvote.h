@@ -193,6 +193,17 @@ GVOTE_API int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t
                       int64_t total_tokens, int64_t max_N, int32_t* budget,
                       void* ws, size_t ws_bytes, void* stream);
 
+/* Section 3.3's yardstick applied to a keep-mask: overlap[r][g] = the share of the current query's
+ * attention (softmax weights of Eq. 1 over all N_r keys) of query head g that falls on the keys its
+ * KV head keeps; 1 means nothing the query looks at was pruned.  Q as written by gvote_project (the
+ * current-query rows are used), K the UNPRUNED keys, mask as written by gvote_vote.  overlap:
+ * [batch, n_q_heads] float.  A diagnostic: fp32 logits, not on the compression path. */
+GVOTE_API int32_t gvote_overlap(const gvote_params* p, const void* Q,
+                      const void* K, int64_t k_tok_stride, int64_t k_head_stride,
+                      const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch,
+                      int64_t total_tokens, int64_t max_N, float* overlap,
+                      void* ws, size_t ws_bytes, void* stream);
+
 /* Section 3.4: the pruned cache in the layout a variable-length attention kernel consumes, written
  * out of place from the UNPRUNED K and V and the keep-mask (use it instead of gvote_compact when
  * the engine wants one dense buffer rather than per-head slabs).  "Sequence" s = r * n_kv_heads + h

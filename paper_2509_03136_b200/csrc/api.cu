@@ -256,6 +256,19 @@ int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const flo
                         total_tokens, max_N, budget, m, w, st);
 }
 
+int32_t gvote_overlap(const gvote_params* p, const void* Q, const void* K, int64_t k_tok_stride, int64_t k_head_stride,
+                      const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens,
+                      int64_t max_N, float* overlap, void* ws, size_t ws_bytes, void* stream) {
+  PROPAGATE(validate_params(p));
+  PROPAGATE(validate_batch(batch, total_tokens, max_N));
+  REQUIRE_PTR(Q); REQUIRE_PTR(K); REQUIRE_PTR(mask); REQUIRE_PTR(cu_seqlens); REQUIRE_PTR(overlap); REQUIRE_PTR(ws);
+  if (k_tok_stride < p->d_k || k_tok_stride % 8 != 0 || k_head_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
+  if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
+  return launch_overlap(p, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, k_tok_stride, k_head_stride, mask,
+                        cu_seqlens, batch, max_N, overlap, m, (char*)ws, (cudaStream_t)stream);
+}
+
 int32_t gvote_pack(const gvote_params* p, const void* K, const void* V, int64_t tok_stride, int64_t head_stride,
                    const uint32_t* mask, const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int64_t max_N,
                    void* K_packed, void* V_packed, int64_t capacity_rows, int32_t* cu_seqlens_k, int32_t* budget,

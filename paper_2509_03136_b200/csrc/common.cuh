@@ -124,6 +124,10 @@ int32_t launch_pack(const gvote_params* p, const __nv_bfloat16* K, const __nv_bf
                     __nv_bfloat16* K_packed, __nv_bfloat16* V_packed, int64_t capacity_rows, int32_t* cu_seqlens_k,
                     int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
 
+int32_t launch_overlap(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                       int64_t k_head, const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t max_N,
+                       float* overlap, const WorkspaceMap& m, char* ws, cudaStream_t st);
+
 // ---------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 

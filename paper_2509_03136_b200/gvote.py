@@ -23,7 +23,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
     "gvote_workspace_bytes", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
-    "gvote_compact", "gvote_pack", "gvote_compress", "gvote_compress_moments", "gvote_compress_host", "gvote_host_arena_release",
+    "gvote_compact", "gvote_pack", "gvote_overlap", "gvote_compress", "gvote_compress_moments", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
@@ -81,6 +81,8 @@ def load():
     lib.gvote_select.argtypes = [P, vp, vp, vp, i64, vp, vp, i64, i64, vp, i32, i64, i64, vp, vp, vp, vp, vp, sz, vp]
     lib.gvote_compact.restype = i32
     lib.gvote_compact.argtypes = [P, vp, vp, i64, i64, vp, vp, i32, i64, i64, vp, vp, sz, vp]
+    lib.gvote_overlap.restype = i32
+    lib.gvote_overlap.argtypes = [P, vp, vp, i64, i64, vp, vp, i32, i64, i64, vp, vp, sz, vp]
     lib.gvote_pack.restype = i32
     lib.gvote_pack.argtypes = [P, vp, vp, i64, i64, vp, vp, i32, i64, i64, vp, vp, i64, vp, vp, vp, sz, vp]
     lib.gvote_compress.restype = i32
@@ -265,6 +267,16 @@ def gvote_compact(p, K, V, mask, cu_seqlens, geom, budget, ws) -> None:
     _check(load().gvote_compact(ctypes.byref(p), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(mask),
                                 _ptr(cu_seqlens), batch, total, max_N, _ptr(budget), _ptr(ws), ws.numel(), _stream()),
            "gvote_compact")
+
+
+def gvote_overlap(p, Q, K, mask, cu_seqlens, geom, overlap, ws) -> None:
+    """Share of each query head's current-query attention that falls on the kept keys (Section 3.3)."""
+    batch, total, max_N = geom
+    _dev(Q, torch.bfloat16, "Q"); _dev(K, torch.bfloat16, "K", dense=False); _dev(mask, torch.int32, "mask")
+    _dev(overlap, torch.float32, "overlap")
+    _check(load().gvote_overlap(ctypes.byref(p), _ptr(Q), _ptr(K), K.stride(1), K.stride(0), _ptr(mask),
+                                _ptr(cu_seqlens), batch, total, max_N, _ptr(overlap), _ptr(ws), ws.numel(), _stream()),
+           "gvote_overlap")
 
 
 def gvote_pack(p, K, V, mask, cu_seqlens, geom, K_packed, V_packed, cu_seqlens_k, budget, ws) -> None:

@@ -323,6 +323,31 @@ def test_compact_strided_heads(gv):
         assert np.array_equal(out[0, :n, h], base[0, keep[h], h]) and np.array_equal(out[1, :n, h], base[1, keep[h], h])
 
 
+# ----------------------------------------------------------------------------- attention overlap
+@pytest.mark.parametrize("idx", range(4))
+def test_overlap_matches_oracle(gv, idx):
+    """gvote_overlap on the mask gvote_vote produced, against the oracle on the same mask: fp32 logits
+    of bf16 operands against fp64, 1e-4 absolute on a number in [0, 1]."""
+    cfg = _small_cfgs()[idx]
+    li = synth.make_layer(cfg, 0)
+    Q_or = _oracle_queries(cfg, li)
+    mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    p = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    Qgm = np.ascontiguousarray(np.stack([pu.to_group_major(q, cfg.G) for q in Q_or]))
+    Qd = torch.from_numpy(Qgm).to(torch.bfloat16).contiguous().cuda()
+    ov = torch.empty(cfg.batch, cfg.n_q_heads, device="cuda")
+    gv.gvote_overlap(p, Qd, gv.bf16_from_bits(li.K), torch.from_numpy(mask).cuda(), torch.from_numpy(li.cu_seqlens).cuda(),
+                     geom, ov, ws)
+    ov = ov.cpu().numpy()
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), b - a) for h in range(cfg.n_kv_heads)])
+        ref = o.attention_overlap(Q_or[r], o.bf16_bits_to_f64(li.K[:, a:b]), gm)
+        assert np.abs(ov[r] - ref).max() < 1e-4, (ov[r], ref)
+
+
 # ----------------------------------------------------------------------------- varlen packing
 @pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
                                                   ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
