@@ -532,17 +532,31 @@ def test_compress_is_deterministic(gv):
         assert np.array_equal(x, y)
 
 
+def _layers_to_check(default):
+    """GVOTE_PARITY_LAYERS=a,b,... or "all" widens the full-size checks beyond the default layer (each
+    layer costs the oracle some tens of seconds of CPU)."""
+    import os
+    want = os.environ.get("GVOTE_PARITY_LAYERS", "")
+    if not want:
+        return [default]
+    return None if want == "all" else [int(x) for x in want.split(",")]
+
+
 def test_compress_full_size_c2_layer(gv):
-    """One layer of the 32K workload, in the launch configuration the benchmark times."""
+    """A layer of the 32K workload, in the launch configuration the benchmark times."""
     cfg = synth.make_config("c2")
-    _check_compress(gv, cfg, synth.make_layer(cfg, 3), layer_id=3)
+    layers = _layers_to_check(3)
+    for layer in (range(cfg.n_layers) if layers is None else layers):
+        _check_compress(gv, cfg, synth.make_layer(cfg, layer), layer_id=layer)
 
 
 def test_compress_full_size_c4_layer(gv):
     """One layer of the 128K-context Qwen2.5-7B-shaped workload (N = 131072, G = 7, S = 64, p = 0.98):
     two row chunks per KV head in the score contraction, 2 MB of mask bits, 1.9 GB of hidden states."""
     cfg = synth.make_config("c4")
-    _check_compress(gv, cfg, synth.make_layer(cfg, 1), layer_id=1)
+    layers = _layers_to_check(1)
+    for layer in (range(cfg.n_layers) if layers is None else layers):
+        _check_compress(gv, cfg, synth.make_layer(cfg, layer), layer_id=layer)
 
 
 def test_compress_host_variant_matches_device_variant(gv):
