@@ -121,7 +121,10 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
                  uint32_t* __restrict__ mask, int32_t* __restrict__ b_step) {
   extern __shared__ __align__(16) uint8_t dyn[];
   ClusterShared& cs = *reinterpret_cast<ClusterShared*>(dyn);
-  __shared__ SelShared sh;               // only the generic radix search and the emission use it
+  // The generic radix search and the emission (rare routes of the first CTA) work in the space of the
+  // candidate list, which is dead by the time they run.
+  static_assert(sizeof(SelShared) <= sizeof(float) * kListCap + sizeof(int) * kListCap, "list area too small");
+  SelShared& sh = *reinterpret_cast<SelShared*>(cs.val);
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
   ClusterShared& lead = *cluster.map_shared_rank(&cs, 0);
@@ -349,8 +352,9 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
       __syncthreads();
       const float v_t = cs.v_t;
       const uint32_t eq = (tid < m && cs.val[tid] == v_t) ? 1u : 0u, gt = (tid < m && cs.val[tid] > v_t) ? 1u : 0u;
-      eq_cnt = block_sum_u32(eq, sh.red32);
-      const uint32_t gt_cnt = block_sum_u32(gt, sh.red32);
+      eq_cnt = block_sum_u32(eq, cs.red32);
+      const uint32_t gt_cnt = block_sum_u32(gt, cs.red32);
+      __syncthreads();                                    // the list is dead from here on (sh takes its place)
       t_key = ordered_key(v_t);
       ties = (uint32_t)pick - gt_cnt;
       settled = true;
