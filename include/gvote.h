@@ -24,6 +24,8 @@
  *    (device) holds the prefix sums of the request lengths N_r (request r owns tokens
  *    cu_seqlens[r] .. cu_seqlens[r+1]-1).  `total_tokens` = cu_seqlens[batch] and `max_N` =
  *    the longest request are passed from the host so that no call has to read the device.
+ *    A request may be empty (N_r = 0): nothing is read or written for it, its budgets and |C0| are 0.
+ *    A non-empty request needs N_r - n_s >= 2 rows for the fit.
  *  - bf16 tensors: W_q [n_q_heads*d_k, d_h], one row per output feature (the paper's W_q
  *    stored transposed, as linear layers keep it), row stride wq_ld elements;
  *    K and V [n_kv_heads, total_tokens, d_k] with element strides (head_stride, tok_stride),

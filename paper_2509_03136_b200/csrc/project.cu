@@ -27,8 +27,10 @@ __global__ void xstage_kernel(const float* __restrict__ H, const T* __restrict__
   if (c >= d_h) return;
   float v;
   if (row == 0) {
+    // the current query is the request's last row; a request without rows has none (zeros stand in)
+    const bool empty = cu_rows && cu_rows[r + 1] <= cu_rows[r];
     const int64_t src_row = cu_rows ? (int64_t)cu_rows[r + 1] - 1 : (int64_t)r;
-    v = to_f32<T>(h_last[src_row * h_last_ld + c]);
+    v = empty ? 0.f : to_f32<T>(h_last[src_row * h_last_ld + c]);
   } else {
     v = H[((int64_t)r * S + (row - 1)) * d_h + c];
   }

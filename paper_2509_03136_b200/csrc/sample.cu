@@ -94,9 +94,12 @@ prep_kernel(const float2* __restrict__ partial, int chunks, const T* __restrict_
       fit_merge_finish(acc, ref, m, v);
       mu[(int64_t)r * d_h + col] = m;
       var[(int64_t)r * d_h + col] = v;
+      // the current query is the request's last row; a request without rows has none (zeros stand in)
+      const bool empty = cu_rows && cu_rows[r + 1] <= cu_rows[r];
       const int64_t src_row = cu_rows ? (int64_t)cu_rows[r + 1] - 1 : (int64_t)r;
       float x0;
-      if (sizeof(T) == 4) x0 = reinterpret_cast<const float*>(h_last)[src_row * h_last_ld + col];
+      if (empty) x0 = 0.f;
+      else if (sizeof(T) == 4) x0 = reinterpret_cast<const float*>(h_last)[src_row * h_last_ld + col];
       else x0 = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(h_last)[src_row * h_last_ld + col]);
       X[((int64_t)r * (S + 1)) * d_h + col] = __float2bfloat16_rn(x0);
     }

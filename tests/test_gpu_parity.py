@@ -523,6 +523,30 @@ def test_compress_from_streamed_moments(gv, name):
     _check_compress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(name == "small2")), runner=_run_compress_moments)
 
 
+def test_compress_with_an_empty_request(gv):
+    """A request without cached tokens in the middle of a batch: nothing is read or written for it
+    (budget 0, |C0| 0) and its neighbours are unaffected."""
+    cfg = synth.make_small(8, seq_lens=(40, 0, 33), S=4, d_h=64, n_q_heads=4, n_kv_heads=2, d_k=64)
+    full = synth.make_small(8, seq_lens=(40, 33), S=4, d_h=64, n_q_heads=4, n_kv_heads=2, d_k=64)
+    li = synth.make_layer(full, 0)
+    li.cu_seqlens = np.array([0, 40, 40, 73], dtype=np.int32)
+    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li)
+    assert budget[1].tolist() == [0, 0] and b_step[1].tolist() == [0] * 4
+    W = o.bf16_bits_to_f64(li.W_q)
+    kw = pu.oracle_kwargs(cfg)
+    for r, (a, b) in ((0, (0, 40)), (2, (40, 73))):
+        res = o.compress_request(li.h[a:b].astype(np.float64), W, li.b_q, o.bf16_bits_to_f64(li.K[:, a:b]),
+                                 request_id=r, **kw)
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), b - a) for h in range(cfg.n_kv_heads)])
+        pu.check_vote_against_oracle(res.Q, o.bf16_bits_to_f64(li.K[:, a:b]), kw["p_nuc"], "topk", False, gm, b_step[r],
+                                     mass_band=2e-2, logit_band=2e-2)
+        assert np.all(np.abs(budget[r] - res.budget) <= 2)
+        Kc, Vc = o.compact(li.K[:, a:b], li.V[:, a:b], gm)
+        for h in range(cfg.n_kv_heads):
+            n = int(gm[h].sum())
+            assert np.array_equal(Kg[h, a:a + n], Kc[h]) and np.array_equal(Vg[h, a:a + n], Vc[h])
+
+
 def test_compress_is_deterministic(gv):
     cfg = synth.make_config("c1")
     li = synth.make_layer(cfg, 0)
