@@ -139,6 +139,7 @@ GVOTE_API int32_t gvote_fit_finish(const gvote_params* p, const double* state, i
  *  - All calls on a device share the one array.  It needs no clearing (every entry a call reads
  *    it has written itself), but two calls whose kernels may overlap on the GPU (different
  *    streams, no dependency) race on it: serialise them.
+ *  - There is no status word here: a bounded device-side wait that ran out shows as NaN in mu.
  * Arguments as in gvote_fit, minus the workspace and total_tokens. */
 #define GVOTE_FIT_STATIC_MAX_ENTRIES 131072
 GVOTE_API int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_t h_row_stride,

@@ -76,12 +76,7 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   WorkspaceMap m;
   memset(&m, 0, sizeof(m));
   const int64_t S1 = p->S + 1, F = (int64_t)p->n_q_heads * p->d_k;
-  const int strips = (int)ceil_div(p->d_h, kFitStripCols);
-  // about eight CTAs per SM on a 148-SM part, at least 32 rows per chunk
-  int64_t chunks = 1184 / ((int64_t)strips * batch);
-  const int64_t max_chunks = ceil_div(max_N > 0 ? max_N : 1, 32);
-  if (chunks > max_chunks) chunks = max_chunks;
-  if (chunks < 1) chunks = 1;
+  const int64_t chunks = fit_chunk_count(p, batch, max_N);
   m.fit_chunks = (int)chunks;
   m.proj_splits = project_umma_splits(p, batch * (p->S + 1));
   m.n_tiles = (total_tokens >> 7) + batch;
@@ -132,8 +127,9 @@ int32_t gvote_fit(const gvote_params* p, const void* h, int64_t h_row_stride, co
   if (max_N - p->n_s < 2) return GVOTE_ERR_INVALID_ARG;
   const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
   if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
-  return launch_fit(p, h, h_row_stride, cu_seqlens, batch, m.fit_chunks,
-                    reinterpret_cast<float2*>((char*)ws + m.fit_partial), mu, var, (cudaStream_t)stream);
+  return launch_fit(p, h, h_row_stride, cu_seqlens, batch, total_tokens, m.fit_chunks,
+                    reinterpret_cast<float2*>((char*)ws + m.fit_partial), reinterpret_cast<int32_t*>((char*)ws + m.status),
+                    mu, var, (cudaStream_t)stream);
 }
 
 int32_t gvote_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch, float* H_tilde,
@@ -218,8 +214,9 @@ int32_t gvote_fit_update(const gvote_params* p, const void* h_block, int64_t h_r
   if (h_row_stride < p->d_h || h_row_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
   const WorkspaceMap m = workspace_map(p, batch, total_rows, max_rows);
   if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
-  return launch_fit_state_update(p, h_block, h_row_stride, cu_block, batch, m.fit_chunks,
-                                 reinterpret_cast<float2*>((char*)ws + m.fit_partial), state, (cudaStream_t)stream);
+  return launch_fit_state_update(p, h_block, h_row_stride, cu_block, batch, total_rows, m.fit_chunks,
+                                 reinterpret_cast<float2*>((char*)ws + m.fit_partial),
+                                 reinterpret_cast<int32_t*>((char*)ws + m.status), state, (cudaStream_t)stream);
 }
 
 int32_t gvote_fit_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
@@ -307,8 +304,8 @@ int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_strid
   float* mu = reinterpret_cast<float*>(w + m.mu);
   float* var = reinterpret_cast<float*>(w + m.var);
   __nv_bfloat16* Q = reinterpret_cast<__nv_bfloat16*>(w + m.q_bf16);
-  PROPAGATE(launch_fit_partial(p, h, h_row_stride, cu_seqlens, batch, m.fit_chunks,
-                               reinterpret_cast<float2*>(w + m.fit_partial), st));
+  PROPAGATE(launch_fit_partial(p, h, h_row_stride, cu_seqlens, batch, total_tokens, m.fit_chunks,
+                               reinterpret_cast<float2*>(w + m.fit_partial), reinterpret_cast<int32_t*>(w + m.status), st));
   __nv_bfloat16* X = reinterpret_cast<__nv_bfloat16*>(w + m.x_bf16);
   float* rope = reinterpret_cast<float*>(w + m.rope);
   if (h_last_or_null)

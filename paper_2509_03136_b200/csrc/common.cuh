@@ -53,7 +53,7 @@ int32_t validate_params(const gvote_params* p);
 // Status block (first 256 bytes): word 0 = sticky error status, word 1 = where it was raised.
 constexpr size_t kStatusBytes = 256;
 constexpr int kCompactTile = 128;   // tokens per compaction tile
-constexpr int kFitStripCols = 256;  // channels per fit CTA (64 threads x float4)
+constexpr int kFitStripCols = 256;  // channels per fit CTA (64 column threads x 4 channels)
 
 struct WorkspaceMap {
   size_t status;        // int32[64]
@@ -88,11 +88,15 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
 // ---------------------------------------------------------------------------------- stage launchers
 // (each enqueues kernels on `st`; pointers are device pointers; see gvote.h for the layouts)
 int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                   int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st);
+                   int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, float* mu, float* var,
+                   cudaStream_t st);
 int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                           int fit_chunks, float2* partial, cudaStream_t st);
+                           int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, cudaStream_t st);
 int32_t launch_fit_state_update(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                                int fit_chunks, float2* partial, double* state, cudaStream_t st);
+                                int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, double* state,
+                                cudaStream_t st);
+// Row chunks per request for the fit (see fit.cu).
+int fit_chunk_count(const gvote_params* p, int32_t batch, int64_t max_N);
 int32_t launch_fit_state_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
                                 cudaStream_t st);
 int32_t launch_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch,

@@ -2,29 +2,44 @@
 // hidden states along the sequence axis, skipping the first n_s sink tokens of every request.
 //
 // The hidden-state matrix is the largest tensor the pass touches (16 KiB per token at d_h = 4096
-// in fp32), so this is a pure HBM stream: each CTA owns a strip of 256 channels and a chunk of
-// rows, every thread keeps shifted first and second moments of four channels in registers, and
-// one (mean, M2) pair per channel and chunk goes to scratch.  A second, tiny kernel merges the
-// chunks with Chan's parallel-variance update in fp64.
+// in fp32), so this is a pure HBM stream.  Each CTA owns a strip of 256 channels and a chunk of
+// rows and pulls them through a ring of shared-memory stages: one thread asks the TMA unit for a
+// [32 rows x 256 channels] box per stage (marked evict-first in L2: the data is read once), four
+// warps take the stages as they land and keep shifted first and second moments of four channels
+// per thread in registers.  Few threads and registers per SM stay busy that way, which leaves room
+// for the kernels of other layers that run beside the fit on other streams.  One (mean, M2) pair
+// per channel and chunk goes to scratch; a second, tiny kernel merges the chunks with Chan's
+// parallel-variance update in fp64.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises GVOTE_ERR_TIMEOUT in the status word
+// (where the caller gave one), lets its copies in flight land, and writes NaN partials so that the
+// failure cannot pass for a result.
 #include <mutex>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace gvote {
 namespace {
 
-constexpr int kFitTx = 64;   // column threads (x4 channels each)
-constexpr int kFitTy = 4;    // row lanes
+constexpr int kFitTx = 64;                 // column threads (x4 channels each)
+constexpr int kFitTy = 2;                  // row lanes
+constexpr int kFitRows = 32;               // rows per stage (one lane of the producer warp per row in the tail)
+constexpr int kFitConsumers = kFitTx * kFitTy;
+constexpr int kFitThreads = kFitConsumers + 32;    // + the producer warp
+constexpr int kFitMaxStages = 8;
+constexpr int kFitFlushStages = 4;         // fold the running sums into a second level every so many stages
+constexpr uint32_t kFitWaitPolls = 1u << 22;
 
 template <typename T>
-__device__ __forceinline__ float4 load4(const T* p);
+__device__ __forceinline__ float4 lds4(const T* p);
 template <>
-__device__ __forceinline__ float4 load4<float>(const float* p) {
-  return __ldcs(reinterpret_cast<const float4*>(p));
+__device__ __forceinline__ float4 lds4<float>(const float* p) {
+  return *reinterpret_cast<const float4*>(p);
 }
 template <>
-__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
-  uint2 u = __ldcs(reinterpret_cast<const uint2*>(p));
+__device__ __forceinline__ float4 lds4<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 u = *reinterpret_cast<const uint2*>(p);
   float4 r;
   r.x = __uint_as_float(u.x << 16);
   r.y = __uint_as_float(u.x & 0xffff0000u);
@@ -39,40 +54,116 @@ __device__ __forceinline__ void acc4(float4& s1, float4& s2, const float4& v, co
   s2.x = fmaf(dx, dx, s2.x); s2.y = fmaf(dy, dy, s2.y);
   s2.z = fmaf(dz, dz, s2.z); s2.w = fmaf(dw, dw, s2.w);
 }
+__device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
+// tmH describes h as [rows][d_h] with a [kFitRows x 256] box.  Its row extent may be an upper bound:
+// a stage that would reach past the chunk's last row is fetched row by row instead, so no load
+// touches a row the chunk does not own.
 template <typename T>
-__global__ void __launch_bounds__(kFitTx* kFitTy)
-fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restrict__ cu, int n_s, int d_h,
-                   int chunks, float2* __restrict__ partial) {
+__global__ void __launch_bounds__(kFitThreads)
+fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict__ h, int64_t ld,
+                   const int32_t* __restrict__ cu, int n_s, int d_h, int chunks, int stages,
+                   float2* __restrict__ partial, int32_t* __restrict__ status) {
+  extern __shared__ __align__(1024) uint8_t fit_ring[];
+  __shared__ uint64_t full[kFitMaxStages], empty[kFitMaxStages];
+  __shared__ int abort_flag;
+  __shared__ float4 sm1[kFitTy][kFitTx], sm2[kFitTy][kFitTx];
+  constexpr int R = kFitRows;
+  constexpr uint32_t pitch = kFitStripCols * sizeof(T);
+  constexpr uint32_t stage_bytes = R * pitch;
   const int r = blockIdx.z, c = blockIdx.y;
-  const int tx = threadIdx.x, ty = threadIdx.y;
-  const int col = (blockIdx.x * kFitTx + tx) * 4;
-  const bool active = col < d_h;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col0 = blockIdx.x * kFitStripCols;
+  const int width = min(kFitStripCols, d_h - col0);
   int a, b;
   fit_chunk_rows(cu[r] + n_s, cu[r + 1], chunks, c, a, b);
-
-  float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1, sh = s1;
-  if (active && a < b) {
-    const T* base = h + col;
-    sh = load4<T>(base + (int64_t)a * ld);   // shift: the chunk's first row (same for all row lanes)
-    int i = a + ty;
-    for (; i + 3 * kFitTy < b; i += 4 * kFitTy) {
-      float4 v0 = load4<T>(base + (int64_t)i * ld);
-      float4 v1 = load4<T>(base + (int64_t)(i + kFitTy) * ld);
-      float4 v2 = load4<T>(base + (int64_t)(i + 2 * kFitTy) * ld);
-      float4 v3 = load4<T>(base + (int64_t)(i + 3 * kFitTy) * ld);
-      acc4(s1, s2, v0, sh); acc4(s1, s2, v1, sh); acc4(s1, s2, v2, sh); acc4(s1, s2, v3, sh);
-    }
-    for (; i < b; i += kFitTy) {
-      float4 v = load4<T>(base + (int64_t)i * ld);
-      acc4(s1, s2, v, sh);
-    }
+  const int n_it = (b > a) ? (b - a + R - 1) / R : 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], kFitConsumers / 32); }
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmH);
   }
-  __shared__ float4 sm1[kFitTy][kFitTx], sm2[kFitTy][kFitTx];
-  sm1[ty][tx] = s1;
-  sm2[ty][tx] = s2;
   __syncthreads();
-  if (ty == 0 && active) {
+  const int tx = threadIdx.x % kFitTx, ty = (threadIdx.x / kFitTx) % kFitTy;
+  const bool active = tx * 4 < width;
+  float4 sh = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  if (warp == kFitConsumers / 32) {
+    // ------------------------------------------------------------ producer
+    const uint64_t pol = ptx::l2_policy_evict_first();
+    int issued = 0;
+    bool ok = true;
+    for (int it = 0; it < n_it; ++it) {
+      const int s = it % stages;
+      if (it >= stages) {
+        const uint32_t par = ((uint32_t)(it / stages) & 1u) ^ 1u;
+        ok = ptx::mbar_wait(&empty[s], par, kFitWaitPolls) && !*(volatile int*)&abort_flag;
+        if (!ok) break;
+      }
+      const int row = a + it * R;
+      const int rows_here = min(R, b - row);
+      uint8_t* dst = fit_ring + (size_t)s * stage_bytes;
+      if (rows_here == R) {
+        if (lane == 0) {
+          ptx::mbar_arrive_expect_tx(&full[s], stage_bytes);
+          ptx::tma_load_2d_hint(dst, &tmH, &full[s], col0, row, pol);
+        }
+      } else {
+        const uint32_t row_bytes = (uint32_t)width * sizeof(T);
+        if (lane == 0) ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)rows_here * row_bytes);
+        __syncwarp();
+        if (lane < rows_here) ptx::bulk_load(dst + (size_t)lane * pitch, h + (int64_t)(row + lane) * ld + col0, row_bytes, &full[s]);
+      }
+      issued = it + 1;
+    }
+    if (!ok) {
+      if (lane == 0) abort_flag = 1;
+      for (int it = max(issued - stages, 0); it < issued; ++it)      // let the copies in flight land
+        ptx::mbar_wait(&full[it % stages], (uint32_t)(it / stages) & 1u, kFitWaitPolls);
+    }
+  } else {
+    // ------------------------------------------------------------ consumers
+    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1, t1 = s1, t2 = s1;
+    for (int it = 0; it < n_it; ++it) {
+      const int s = it % stages;
+      if (!ptx::mbar_wait(&full[s], (uint32_t)(it / stages) & 1u, kFitWaitPolls) || *(volatile int*)&abort_flag) {
+        abort_flag = 1;
+        break;
+      }
+      const T* st = reinterpret_cast<const T*>(fit_ring + (size_t)s * stage_bytes);
+      const int rows_here = min(R, b - (a + it * R));
+      if (active) {
+        if (it == 0) sh = lds4<T>(st + tx * 4);     // shift: the chunk's first row (same for all row lanes)
+        if (rows_here == R) {
+          float4 v[R / kFitTy];
+#pragma unroll
+          for (int j = 0; j < R / kFitTy; ++j) v[j] = lds4<T>(st + (size_t)(ty + j * kFitTy) * kFitStripCols + tx * 4);
+#pragma unroll
+          for (int j = 0; j < R / kFitTy; ++j) acc4(s1, s2, v[j], sh);
+        } else {
+          for (int row = ty; row < rows_here; row += kFitTy)
+            acc4(s1, s2, lds4<T>(st + (size_t)row * kFitStripCols + tx * 4), sh);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&empty[s]);
+      if ((it + 1) % kFitFlushStages == 0) {        // short fp32 runs: the rounding error stays that of 64 terms
+        add4(t1, s1); add4(t2, s2);
+        s1 = make_float4(0.f, 0.f, 0.f, 0.f); s2 = s1;
+      }
+    }
+    add4(t1, s1); add4(t2, s2);
+    sm1[ty][tx] = t1;
+    sm2[ty][tx] = t2;
+  }
+  __syncthreads();
+  const bool failed = abort_flag != 0;
+  if (threadIdx.x == 0 && failed && status) {
+    atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
+    atomicExch(&status[1], 7);
+  }
+  if (threadIdx.x < kFitTx && active) {
     double t1[4] = {0, 0, 0, 0}, t2[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int j = 0; j < kFitTy; ++j) {
@@ -82,7 +173,7 @@ fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restric
     }
     const int n = b - a;
     const float shv[4] = {sh.x, sh.y, sh.z, sh.w};
-    float2* out = partial + ((int64_t)(r * chunks + c)) * d_h + col;
+    float2* out = partial + ((int64_t)(r * chunks + c)) * d_h + col0 + tx * 4;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       double mean = 0.0, m2 = 0.0;
@@ -90,7 +181,7 @@ fit_partial_kernel(const T* __restrict__ h, int64_t ld, const int32_t* __restric
         mean = (double)shv[j] + t1[j] / n;
         m2 = t2[j] - t1[j] * t1[j] / n;
       }
-      out[j] = make_float2((float)mean, (float)fmax(m2, 0.0));
+      out[j] = failed ? make_float2(nanf(""), nanf("")) : make_float2((float)mean, (float)fmax(m2, 0.0));
     }
   }
 }
@@ -167,17 +258,35 @@ __global__ void fit_state_finish_kernel(const double* __restrict__ state, int d_
 
 }  // namespace
 
+// `rows_bound`: an upper bound of the rows h holds (the packed token count, or batch x longest request).
 int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                           int fit_chunks, float2* partial, cudaStream_t st) {
+                           int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, cudaStream_t st) {
   const int strips = (int)ceil_div(p->d_h, kFitStripCols);
-  dim3 grid(strips, fit_chunks, batch), block(kFitTx, kFitTy);
+  const int elem = p->h_dtype == GVOTE_DTYPE_F32 ? 4 : 2;
+  if (rows_bound < 1) rows_bound = 1;
+  CUtensorMap tmH;
+  {
+    const uint64_t dims[2] = {(uint64_t)p->d_h, (uint64_t)rows_bound};
+    const uint64_t strides[1] = {(uint64_t)ld * elem};
+    const uint32_t box[2] = {(uint32_t)kFitStripCols, (uint32_t)kFitRows};
+    if (!encode_tensor_map_plain(&tmH, h, elem, 2, dims, strides, box)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  }
+  // 96 KB of stages per CTA: what keeps one CTA per SM at the HBM rate
+  const size_t stage_bytes = (size_t)kFitRows * kFitStripCols * elem;
+  int stages = (int)((96 * 1024) / stage_bytes);
+  if (stages > kFitMaxStages) stages = kFitMaxStages;
+  const size_t smem = stages * stage_bytes;
+  dim3 grid(strips, fit_chunks, batch);
   {
     LaunchScope scope_("fit_partial_kernel", st);
     if (p->h_dtype == GVOTE_DTYPE_F32) {
-      fit_partial_kernel<float><<<grid, block, 0, st>>>((const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks, partial);
+      GVOTE_CUDA_CHECK(cudaFuncSetAttribute(fit_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      fit_partial_kernel<float><<<grid, kFitThreads, smem, st>>>(tmH, (const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks,
+                                                                 stages, partial, status);
     } else {
-      fit_partial_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)h, ld, cu, p->n_s, p->d_h,
-                                                                fit_chunks, partial);
+      GVOTE_CUDA_CHECK(cudaFuncSetAttribute(fit_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      fit_partial_kernel<__nv_bfloat16><<<grid, kFitThreads, smem, st>>>((tmH), (const __nv_bfloat16*)h, ld, cu, p->n_s,
+                                                                         p->d_h, fit_chunks, stages, partial, status);
     }
   }
   GVOTE_LAUNCH_CHECK("fit_partial_kernel");
@@ -185,8 +294,9 @@ int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, con
 }
 
 int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                   int fit_chunks, float2* partial, float* mu, float* var, cudaStream_t st) {
-  const int32_t rc = launch_fit_partial(p, h, ld, cu, batch, fit_chunks, partial, st);
+                   int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, float* mu, float* var,
+                   cudaStream_t st) {
+  const int32_t rc = launch_fit_partial(p, h, ld, cu, batch, rows_bound, fit_chunks, partial, status, st);
   if (rc != GVOTE_OK) return rc;
   dim3 g2((unsigned)ceil_div(p->d_h, 32), batch);
   {
@@ -198,10 +308,11 @@ int32_t launch_fit(const gvote_params* p, const void* h, int64_t ld, const int32
 }
 
 int32_t launch_fit_state_update(const gvote_params* p, const void* h, int64_t ld, const int32_t* cu, int32_t batch,
-                                int fit_chunks, float2* partial, double* state, cudaStream_t st) {
+                                int64_t rows_bound, int fit_chunks, float2* partial, int32_t* status, double* state,
+                                cudaStream_t st) {
   gvote_params q = *p;
   q.n_s = 0;                                   // which rows to leave out is the caller's choice here
-  const int32_t rc = launch_fit_partial(&q, h, ld, cu, batch, fit_chunks, partial, st);
+  const int32_t rc = launch_fit_partial(&q, h, ld, cu, batch, rows_bound, fit_chunks, partial, status, st);
   if (rc != GVOTE_OK) return rc;
   dim3 g2((unsigned)ceil_div(p->d_h, 32), batch);
   {
@@ -210,6 +321,18 @@ int32_t launch_fit_state_update(const gvote_params* p, const void* h, int64_t ld
   }
   GVOTE_LAUNCH_CHECK("fit_state_update_kernel");
   return GVOTE_OK;
+}
+
+// One CTA per SM of a 148-SM part streams at the HBM rate when the batch is a single request (all
+// chunks alike); a batch of requests of different lengths gets eight times as many, so that the
+// longest chunk is a small part of the whole.  At least two stages of rows per chunk.
+int fit_chunk_count(const gvote_params* p, int32_t batch, int64_t max_N) {
+  const int64_t strips = ceil_div(p->d_h, kFitStripCols);
+  int64_t chunks = (batch == 1 ? 148 : 1184) / (strips * batch);
+  const int64_t by_rows = ceil_div(max_N > 0 ? max_N : 1, 2 * kFitRows);
+  if (chunks > by_rows) chunks = by_rows;
+  if (chunks < 1) chunks = 1;
+  return (int)chunks;
 }
 
 int32_t launch_fit_state_finish(const gvote_params* p, const double* state, int32_t batch, float* mu, float* var,
@@ -276,18 +399,16 @@ extern "C" int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_
   // one chunk per request is the least the kernels can run with
   const int64_t per_chunk = (int64_t)batch * p->d_h;
   if (per_chunk > (int64_t)kStaticFitEntries) return GVOTE_ERR_UNSUPPORTED_SHAPE;
-  // as many row chunks as fill the GPU, as few as the fixed array holds, at least 32 rows each
-  const int64_t strips = ceil_div(p->d_h, kFitStripCols);
-  int64_t chunks = 1184 / (strips * batch);
+  // as many row chunks as the fit wants, as few as the fixed array holds
+  int64_t chunks = fit_chunk_count(p, batch, max_N);
   const int64_t fit_in_array = (int64_t)kStaticFitEntries / per_chunk;
-  const int64_t by_rows = ceil_div(max_N > 0 ? max_N : 1, 32);
   if (chunks > fit_in_array) chunks = fit_in_array;
-  if (chunks > by_rows) chunks = by_rows;
-  if (chunks < 1) chunks = 1;
   float2* scratch = nullptr;
   const int32_t sv = static_scratch_for_current_device(&scratch);
   if (sv != GVOTE_OK) return sv;
   // every entry the merge kernel reads is written by the partial kernel of the same call, so the
   // array needs no clearing between calls
-  return launch_fit(p, h, h_row_stride, cu_seqlens, batch, (int)chunks, scratch, mu, var, (cudaStream_t)stream);
+  // no status word here: a wait that ran out shows as NaN in mu and var
+  return launch_fit(p, h, h_row_stride, cu_seqlens, batch, (int64_t)batch * max_N, (int)chunks, scratch, nullptr, mu, var,
+                    (cudaStream_t)stream);
 }
