@@ -20,7 +20,10 @@ Readings of the paper where it is silent (each is a parameter or stated where us
   * variance is the unbiased estimator; the first n_s rows are skipped (Step 2);
   * future positions are N .. N+n_f-1; RoPE is rotate-half with w_j = theta^(-2j/d_k);
   * top-p keeps the shortest prefix, in (weight desc, index asc) order, whose running sum
-    reaches p (the crossing element is kept); top-k ties go to the lower index.
+    reaches p (the crossing element is kept); top-k ties go to the lower index;
+  * applying the pass again to a pruned cache (`recompress_request`, beyond the paper): every
+    query head votes over the rows its own KV head still holds; positions come from the
+    number of tokens seen, not from the number of rows stored.
 
 Parity status: every function below is pinned by tests/ against closed forms, brute
 force, published known-answer vectors or textbook library routines, except the end-to-end
@@ -386,6 +389,57 @@ def compress_request(h: np.ndarray, W_q: np.ndarray, b_q: Optional[np.ndarray], 
                                              keep_probs=keep_probs)     # 1-3, 8-10
     return RequestResult(mu=mu, var=var, H_tilde=H_tilde, Q=Q, b_step=b_step, mask=mask,
                          budget=budget, row_sets=rows, probs=probs)
+
+
+@dataclass
+class RecompressResult:
+    b_step: np.ndarray                 # [H_q] int   k_g = |C0| of query head g over its KV head's keys
+    masks: List[np.ndarray]            # per KV head: [len_kh] bool over that head's cache slots
+    budget: np.ndarray                 # [H_kv] int
+    token_pos: Optional[List[np.ndarray]]   # per KV head: original positions of the slots that stay
+    Q: np.ndarray                      # [H_q, S+1, d_k]
+
+
+def recompress_request(mu: np.ndarray, var: np.ndarray, h_last: np.ndarray, W_q: np.ndarray,
+                       b_q: Optional[np.ndarray], K_heads: Sequence[np.ndarray], seq_len: int, *,
+                       n_q_heads: int, d_k: int, theta: float, S: int, p_nuc: float, n_f: int,
+                       seed: int, layer_id: int, request_id: int, sel_mode: str = "topk",
+                       include_c0: bool = False, mirror_rounding: bool = True,
+                       token_pos: Optional[Sequence[np.ndarray]] = None) -> RecompressResult:
+    """Algorithm 1 applied again to a cache that an earlier pass has already pruned and that has
+    grown since (the extension Section 3.4 leaves open: there the pass runs once, after prefill).
+
+    KV head kh now holds K_heads[kh] [len_kh, d_k]: the rows that survived plus the rows appended
+    since, each still rotated at the position it was written at, so head lengths differ and a
+    slot number no longer is a position.  What Algorithm 1 calls N splits in two: the keys a
+    query head sees are the len_kh rows of its own KV head (lines 1-3 and 8-10 run per head on
+    those), while the positions of lines 1 and 6 come from seq_len, the number of tokens the
+    request has seen: the current query sits at seq_len - 1 and the synthetic queries average
+    positions seq_len .. seq_len + n_f - 1.  mu and var are the caller's running fit (line 4).
+    token_pos[kh] [len_kh] (optional) maps slots to original positions; the result carries the
+    map of the slots that stay."""
+    H_kv = len(K_heads)
+    G = n_q_heads // H_kv
+    H_tilde, _ = sample(mu, var, S, seed, layer_id, request_id)                      # line 5
+    Q = queries_for_request(H_tilde, h_last, W_q, b_q, seq_len, n_q_heads=n_q_heads, d_k=d_k,
+                            theta=theta, n_f=n_f, mirror_rounding=mirror_rounding)   # 1, 6-7
+    masks: List[np.ndarray] = []
+    b_step = np.zeros(n_q_heads, dtype=np.int64)
+    budget = np.zeros(H_kv, dtype=np.int64)
+    for kh in range(H_kv):
+        Kh = np.asarray(K_heads[kh], dtype=np.float64)
+        if Kh.shape[0] == 0:
+            masks.append(np.zeros(0, dtype=bool))
+            continue
+        m, b, ks, _, _ = vote(Q[kh * G:(kh + 1) * G], Kh[None], p_nuc=p_nuc, sel_mode=sel_mode,
+                              include_c0=include_c0)                                  # 1-3, 8-10
+        masks.append(m[0])
+        budget[kh] = b[0]
+        b_step[kh * G:(kh + 1) * G] = ks
+    kept_pos = None
+    if token_pos is not None:
+        kept_pos = [np.asarray(token_pos[kh])[masks[kh]] for kh in range(H_kv)]      # line 11, on the map
+    return RecompressResult(b_step=b_step, masks=masks, budget=budget, token_pos=kept_pos, Q=Q)
 
 
 def compress_layer(h: np.ndarray, W_q_bits: np.ndarray, b_q: Optional[np.ndarray],

@@ -533,3 +533,116 @@ def test_attention_overlap_special_cases():
     Q1 = np.zeros((1, 1, 4)); Q1[0, 0, 0] = 2.0
     K1 = np.zeros((1, 2, 4)); K1[0, 1, 0] = math.log(3.0)         # logit = 2 * ln3 / sqrt(4) = ln 3
     assert o.attention_overlap(Q1, K1, np.array([[False, True]]))[0] == pytest.approx(0.75, rel=1e-14)
+
+
+# ----------------------------------------------------------------------------- the pass applied again
+def _recompress_problem(seed, H_q=4, H_kv=2, d_k=16, d_h=24, N0=30):
+    rng = np.random.default_rng(seed)
+    W = rng.normal(size=(H_q * d_k, d_h)) / math.sqrt(d_h)
+    mu, var = rng.normal(size=d_h), rng.uniform(0.5, 2.0, size=d_h)
+    h_last = rng.normal(size=d_h)
+    k0 = rng.normal(size=(H_kv, N0, d_k))                  # keys before rotation, one per position
+    return W, mu, var, h_last, k0
+
+
+def _keys_at(k0_head, pos, d_k, theta, shift=0):
+    """Rows `pos` of the unrotated keys, rotated at positions pos + shift."""
+    w = o.rope_frequencies(d_k, theta)
+    at = (np.asarray(pos, dtype=np.float64) + shift)[:, None]
+    return o.rope_apply(k0_head[np.asarray(pos, dtype=int)], np.cos(at * w), np.sin(at * w))
+
+
+def test_recompress_of_an_unpruned_cache_is_the_pass_itself():
+    rng = np.random.default_rng(40)
+    H_q, H_kv, d_k, d_h, N, S, n_s = 4, 2, 8, 12, 26, 5, 2
+    h = rng.normal(size=(N, d_h))
+    W = rng.normal(size=(H_q * d_k, d_h)) / math.sqrt(d_h)
+    K = rng.normal(size=(H_kv, N, d_k))
+    kw = dict(n_q_heads=H_q, d_k=d_k, theta=1e4, S=S, p_nuc=0.8, n_f=4, seed=9, layer_id=3, request_id=1)
+    first = o.compress_request(h, W, None, K, n_s=n_s, **kw)
+    mu, var = o.fit(h, n_s)
+    again = o.recompress_request(mu, var, h[-1], W, None, [K[0], K[1]], N, **kw)
+    for kh in range(H_kv):
+        assert np.array_equal(again.masks[kh], first.mask[kh])
+    assert np.array_equal(again.budget, first.budget) and np.array_equal(again.b_step, first.b_step)
+
+
+def test_recompress_positions_come_from_tokens_seen_not_rows_stored():
+    """RoPE scores depend on relative position only, so moving every stored key and the count of
+    tokens seen by the same offset changes nothing; a query placed by the number of rows stored
+    would not move with them."""
+    d_k, theta, N0 = 16, 1e4, 30
+    W, mu, var, h_last, k0 = _recompress_problem(41, d_k=d_k, N0=N0)
+    rng = np.random.default_rng(42)
+    pos = [np.sort(rng.choice(N0, size=n, replace=False)) for n in (17, 9)]
+    kw = dict(n_q_heads=4, d_k=d_k, theta=theta, S=3, p_nuc=0.5, n_f=4, seed=5, layer_id=0, request_id=0,
+              mirror_rounding=False)
+    base = o.recompress_request(mu, var, h_last, W, None, [_keys_at(k0[kh], pos[kh], d_k, theta) for kh in range(2)],
+                                N0, **kw)
+    for shift in (1, 57):
+        moved = o.recompress_request(mu, var, h_last, W, None,
+                                     [_keys_at(k0[kh], pos[kh], d_k, theta, shift) for kh in range(2)],
+                                     N0 + shift, **kw)
+        for kh in range(2):
+            assert np.array_equal(moved.masks[kh], base.masks[kh])
+        assert np.array_equal(moved.b_step, base.b_step)
+    # the control: keys moved, count of tokens seen left alone -> different logits, different queries
+    stale = o.recompress_request(mu, var, h_last, W, None,
+                                 [_keys_at(k0[kh], pos[kh], d_k, theta, 57) for kh in range(2)], N0, **kw)
+    assert np.array_equal(stale.Q, base.Q)
+    assert (not np.array_equal(stale.b_step, base.b_step)
+            or any(not np.array_equal(stale.masks[kh], base.masks[kh]) for kh in range(2)))
+
+
+def test_recompress_by_brute_force_each_head_over_its_own_rows():
+    d_k, theta = 4, 1e4
+    W, mu, var, h_last, k0 = _recompress_problem(43, H_q=2, H_kv=2, d_k=d_k, d_h=6, N0=12)
+    pos = [np.array([0, 2, 3, 5, 8, 9, 11]), np.array([1, 4, 6, 10])]
+    K_heads = [_keys_at(k0[kh], pos[kh], d_k, theta) for kh in range(2)]
+    p = 0.7
+    res = o.recompress_request(mu, var, h_last, W, None, K_heads, 12, n_q_heads=2, d_k=d_k, theta=theta, S=3,
+                               p_nuc=p, n_f=2, seed=1, layer_id=0, request_id=0, token_pos=pos)
+    for kh in range(2):
+        n = K_heads[kh].shape[0]
+        assert res.masks[kh].shape == (n,)
+        L = np.array([[sum(res.Q[kh, r, j] * K_heads[kh][i, j] for j in range(d_k)) / 2.0 for i in range(n)]
+                      for r in range(4)])
+        e = np.exp(L[0] - L[0].max())
+        k = _brute_min_subset_size(e / e.sum(), p)
+        assert res.b_step[kh] == k
+        expect = np.zeros(n, dtype=bool)
+        for s in range(1, 4):
+            best = max(itertools.combinations(range(n), k), key=lambda c: sum(L[s, list(c)]))
+            expect[list(best)] = True
+        assert np.array_equal(res.masks[kh], expect) and res.budget[kh] == expect.sum()
+        assert res.token_pos[kh].tolist() == [int(pos[kh][i]) for i in range(n) if expect[i]]
+
+
+def test_recompress_after_a_first_pass_shrinks_and_keeps_the_map_consistent():
+    rng = np.random.default_rng(44)
+    H_q, H_kv, d_k, d_h, N, n_s = 4, 2, 8, 12, 40, 2
+    h = rng.normal(size=(N, d_h))
+    W = rng.normal(size=(H_q * d_k, d_h)) / math.sqrt(d_h)
+    K = rng.normal(size=(H_kv, N, d_k)) * 1.5
+    kw = dict(n_q_heads=H_q, d_k=d_k, theta=1e4, S=4, p_nuc=0.6, n_f=4, layer_id=0, request_id=0, include_c0=True)
+    first = o.compress_request(h, W, None, K, n_s=n_s, seed=3, **kw)
+    pos1 = [np.nonzero(first.mask[kh])[0] for kh in range(H_kv)]
+    mu, var = o.fit(h, n_s)
+    again = o.recompress_request(mu, var, h[-1], W, None, [K[kh][pos1[kh]] for kh in range(H_kv)], N, seed=4,
+                                 token_pos=pos1, **kw)
+    for kh in range(H_kv):
+        assert again.budget[kh] <= first.budget[kh] and again.masks[kh].shape[0] == first.budget[kh]
+        assert set(again.token_pos[kh].tolist()) <= set(pos1[kh].tolist())
+        assert np.all(np.diff(again.token_pos[kh]) > 0)
+    # the first pass kept the current query's own nucleus (include_c0), and the weights of a subset that
+    # holds it only grow when renormalised: the nucleus cannot get larger
+    assert np.all(again.b_step <= first.b_step)
+
+
+def test_recompress_head_with_no_rows():
+    W, mu, var, h_last, k0 = _recompress_problem(45, d_k=8, d_h=10, N0=9)
+    K_heads = [_keys_at(k0[0], np.arange(9), 8, 1e4), np.zeros((0, 8))]
+    res = o.recompress_request(mu, var, h_last, W, None, K_heads, 9, n_q_heads=4, d_k=8, theta=1e4, S=3, p_nuc=0.9,
+                               n_f=2, seed=1, layer_id=0, request_id=0, token_pos=[np.arange(9), np.zeros(0, dtype=int)])
+    assert res.budget[1] == 0 and res.masks[1].shape == (0,) and res.token_pos[1].shape == (0,)
+    assert res.b_step[2] == 0 and res.b_step[3] == 0 and res.budget[0] >= res.b_step[:2].max() > 0
