@@ -241,6 +241,30 @@ GVOTE_API int32_t gvote_compress_moments(const gvote_params* p, const float* mu,
                                uint32_t* mask, int32_t* budget, int32_t* b_step,
                                void* ws, size_t ws_bytes, void* stream);
 
+/* The pass applied again to a cache it has pruned before and that has grown since (an extension: in
+ * Section 3.4 the pass runs once, after prefill).  The heads of such a cache differ in length, and a slot
+ * no longer is a position, so the N of Algorithm 1 splits in two:
+ *  - kv_len [batch, n_kv_heads] int32 (device): rows KV head h of request r holds (kept earlier plus
+ *    appended since), at the front of its slab cu_seqlens[r] .. ; rows beyond are ignored.  Every query
+ *    head votes over the rows of its own KV head only (lines 1-3, 8-10); kv_len may be 0 (budget 0).
+ *  - seq_len [batch] int32 (device): tokens the request has seen.  The current query is rotated at
+ *    position seq_len - 1, the synthetic queries with the mean over positions seq_len .. seq_len+n_f-1
+ *    (lines 1 and 6); keys stay rotated where they were written.
+ *  - cu_seqlens / total_tokens / max_N describe the slabs (capacity), as in gvote_compress.
+ *  - token_pos_or_null [n_kv_heads, total_tokens] int32 (device, in/out): the original position of every
+ *    slot; its kept entries move to the front of the slab with the rows (entries beyond the new budget
+ *    are left as they were).
+ * mu, var: the caller's running fit (gvote_fit_update / gvote_fit_finish over all tokens seen).
+ * Outputs as in gvote_compress: mask over slots, budget = new rows per head, b_step, K and V compacted
+ * in place. */
+GVOTE_API int32_t gvote_recompress(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                         const void* W_q, int64_t wq_ld, const float* b_q_or_null,
+                         void* K, void* V, int64_t tok_stride, int64_t head_stride,
+                         const int32_t* cu_seqlens, const int32_t* kv_len, const int32_t* seq_len,
+                         int32_t* token_pos_or_null, int32_t batch, int64_t total_tokens, int64_t max_N,
+                         uint32_t* mask, int32_t* budget, int32_t* b_step,
+                         void* ws, size_t ws_bytes, void* stream);
+
 /* The same pass for a caller whose tensors live in HOST memory (pinned memory gives full copy
  * speed): all pointers are host pointers, K and V are dense ([n_kv_heads, total_tokens, d_k]),
  * h is dense [total_tokens, d_h].  The call copies the inputs to device buffers it keeps in a

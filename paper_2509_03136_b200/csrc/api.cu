@@ -227,11 +227,15 @@ int32_t gvote_fit_finish(const gvote_params* p, const double* state, int32_t bat
   return launch_fit_state_finish(p, state, batch, mu, var, (cudaStream_t)stream);
 }
 
-int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
-                               const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
-                               int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens, int32_t batch,
-                               int64_t total_tokens, int64_t max_N, uint32_t* mask, int32_t* budget, int32_t* b_step,
-                               void* ws, size_t ws_bytes, void* stream) {
+namespace {
+// The pass from line 5 on, from fitted moments; kv_len / seq_len / token_pos are the extras of the
+// re-application (all null for a cache that has not been pruned before).
+int32_t compress_from_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                              const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
+                              int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens,
+                              const int32_t* kv_len, const int32_t* seq_len, int32_t* token_pos, int32_t batch,
+                              int64_t total_tokens, int64_t max_N, uint32_t* mask, int32_t* budget, int32_t* b_step,
+                              void* ws, size_t ws_bytes, void* stream) {
   PROPAGATE(validate_params(p));
   PROPAGATE(validate_batch(batch, total_tokens, max_N));
   REQUIRE_PTR(mu); REQUIRE_PTR(var); REQUIRE_PTR(h_last); REQUIRE_PTR(W_q); OPTIONAL_PTR(b_q_or_null); REQUIRE_PTR(K);
@@ -246,11 +250,37 @@ int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const flo
   float* Ht = reinterpret_cast<float*>(w + m.h_tilde);
   __nv_bfloat16* Q = reinterpret_cast<__nv_bfloat16*>(w + m.q_bf16);
   PROPAGATE(launch_sample(p, mu, var, batch, Ht, nullptr, st));
-  PROPAGATE(launch_project(p, Ht, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q, st));
+  PROPAGATE(launch_project(p, Ht, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q, st,
+                           seq_len));
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, nullptr, b_step, nullptr, m, w, st));
-  return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
-                        total_tokens, max_N, budget, m, w, st);
+                        max_N, mask, nullptr, b_step, nullptr, m, w, st, kv_len));
+  PROPAGATE(launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
+                           total_tokens, max_N, budget, m, w, st));
+  if (token_pos) PROPAGATE(launch_remap(p, token_pos, mask, cu_seqlens, batch, total_tokens, max_N, budget, m, w, st));
+  return GVOTE_OK;
+}
+}  // namespace
+
+int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                               const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
+                               int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens, int32_t batch,
+                               int64_t total_tokens, int64_t max_N, uint32_t* mask, int32_t* budget, int32_t* b_step,
+                               void* ws, size_t ws_bytes, void* stream) {
+  return compress_from_moments(p, mu, var, h_last, W_q, wq_ld, b_q_or_null, K, V, tok_stride, head_stride, cu_seqlens,
+                               nullptr, nullptr, nullptr, batch, total_tokens, max_N, mask, budget, b_step, ws,
+                               ws_bytes, stream);
+}
+
+int32_t gvote_recompress(const gvote_params* p, const float* mu, const float* var, const void* h_last,
+                         const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,
+                         int64_t tok_stride, int64_t head_stride, const int32_t* cu_seqlens, const int32_t* kv_len,
+                         const int32_t* seq_len, int32_t* token_pos_or_null, int32_t batch, int64_t total_tokens,
+                         int64_t max_N, uint32_t* mask, int32_t* budget, int32_t* b_step, void* ws, size_t ws_bytes,
+                         void* stream) {
+  REQUIRE_PTR(kv_len); REQUIRE_PTR(seq_len); OPTIONAL_PTR(token_pos_or_null);
+  return compress_from_moments(p, mu, var, h_last, W_q, wq_ld, b_q_or_null, K, V, tok_stride, head_stride, cu_seqlens,
+                               kv_len, seq_len, token_pos_or_null, batch, total_tokens, max_N, mask, budget, b_step, ws,
+                               ws_bytes, stream);
 }
 
 int32_t gvote_overlap(const gvote_params* p, const void* Q, const void* K, int64_t k_tok_stride, int64_t k_head_stride,

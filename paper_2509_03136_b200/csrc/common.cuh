@@ -114,11 +114,17 @@ int project_umma_splits(const gvote_params* p, int rows_total);
 int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* h_last, int64_t h_last_ld,
                        const int32_t* h_last_rows_from_cu,  // when non-null: row index = cu[r+1]-1 of h_last
                        const void* W_q, int64_t wq_ld, const float* b_q, const int32_t* cu, int32_t batch,
-                       const WorkspaceMap& m, char* ws, __nv_bfloat16* Q, cudaStream_t st);
+                       const WorkspaceMap& m, char* ws, __nv_bfloat16* Q, cudaStream_t st,
+                       const int32_t* seq_len = nullptr);  // [batch] tokens seen (positions), or the slab lengths
+// Moves the kept entries of a per-head slot -> position map to the front of each slab, like the rows.
+int32_t launch_remap(const gvote_params* p, int32_t* token_pos, const uint32_t* mask, const int32_t* cu, int32_t batch,
+                     int64_t total_tokens, int64_t max_N, const int32_t* budget, const WorkspaceMap& m, char* ws,
+                     cudaStream_t st);
 int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                     uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs,
-                    const WorkspaceMap& m, char* ws, cudaStream_t st);
+                    const WorkspaceMap& m, char* ws, cudaStream_t st,
+                    const int32_t* kv_len = nullptr);   // [batch][n_kv_heads] rows that count, or all
 int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
                        const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens,
                        int64_t max_N, int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
@@ -164,6 +170,14 @@ __device__ __forceinline__ int64_t tile_offset(int cu_r, int r) { return (int64_
 
 
 // Rows of chunk `c` of a request whose fitted rows are [first, last): [a, b).
+// Keys of KV head kh of request r that take part in the vote: all N rows of the request's slab, or
+// (a cache that was pruned before: heads differ in length) the head's own count kv_len[r][kh].
+__device__ __forceinline__ int valid_keys(const int32_t* __restrict__ kv_len, int r, int n_kv_heads, int kh, int N) {
+  if (!kv_len) return N;
+  const int v = kv_len[r * n_kv_heads + kh];
+  return v < 0 ? 0 : (v < N ? v : N);
+}
+
 __device__ __forceinline__ void fit_chunk_rows(int first, int last, int chunks, int c, int& a, int& b) {
   const int n = max(last - first, 0);
   const int per = (n + chunks - 1) / chunks;

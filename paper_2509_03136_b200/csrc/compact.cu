@@ -177,6 +177,36 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   }
 }
 
+// ---------------------------------------------------------------------------------- slot -> position map
+// A cache that has been pruned carries, per KV head, the original position of every slot.  Pruning it
+// again moves the kept entries of that map to the front of the slab exactly as the rows move:
+// entry n goes to prefix(n).  Done out of place (gather into scratch, copy back): the map is 4 bytes
+// per slot, and this way no ordering between CTAs is needed.
+__global__ void __launch_bounds__(256)
+remap_gather_kernel(const int32_t* __restrict__ token_pos, int64_t slab, const uint32_t* __restrict__ mask,
+                    const int32_t* __restrict__ prefix, const int32_t* __restrict__ cu, int64_t row_words,
+                    int32_t* __restrict__ tmp) {
+  const int r = blockIdx.z, h = blockIdx.y;
+  const int start = cu[r], N = cu[r + 1] - start;
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= N) return;
+  const int64_t woff = (int64_t)h * row_words + mask_word_offset(start, r);
+  const uint32_t bits = mask[woff + (n >> 5)];
+  if (!((bits >> (n & 31)) & 1u)) return;
+  const int dst = prefix[woff + (n >> 5)] + __popc(bits & ((1u << (n & 31)) - 1u));
+  tmp[(int64_t)h * slab + start + dst] = token_pos[(int64_t)h * slab + start + n];
+}
+
+__global__ void __launch_bounds__(256)
+remap_store_kernel(int32_t* __restrict__ token_pos, int64_t slab, const int32_t* __restrict__ tmp,
+                   const int32_t* __restrict__ cu, const int32_t* __restrict__ budget, int Hkv) {
+  const int r = blockIdx.z, h = blockIdx.y;
+  const int start = cu[r];
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= budget[r * Hkv + h]) return;
+  token_pos[(int64_t)h * slab + start + n] = tmp[(int64_t)h * slab + start + n];
+}
+
 }  // namespace
 
 int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int32_t* cu, int32_t batch,
@@ -214,6 +244,29 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
                                                                   p->d_k, m.row_words, m.n_tiles, flags, ticket, status);
   }
   GVOTE_LAUNCH_CHECK("compact_kernel");
+  return GVOTE_OK;
+}
+
+// After launch_compact (which leaves the prefix in the workspace and the budgets with the caller).  The
+// gather's scratch is the logits area of the workspace, dead once the vote is over.
+int32_t launch_remap(const gvote_params* p, int32_t* token_pos, const uint32_t* mask, const int32_t* cu, int32_t batch,
+                     int64_t total_tokens, int64_t max_N, const int32_t* budget, const WorkspaceMap& m, char* ws,
+                     cudaStream_t st) {
+  if (max_N <= 0 || total_tokens <= 0) return GVOTE_OK;
+  const int Hkv = p->n_kv_heads;
+  const int32_t* prefix = reinterpret_cast<const int32_t*>(ws + m.prefix);
+  int32_t* tmp = reinterpret_cast<int32_t*>(ws + m.logits);
+  dim3 grid((unsigned)ceil_div(max_N, 256), (unsigned)Hkv, (unsigned)batch);
+  {
+    LaunchScope scope_("remap_gather_kernel", st);
+    remap_gather_kernel<<<grid, 256, 0, st>>>(token_pos, total_tokens, mask, prefix, cu, m.row_words, tmp);
+  }
+  GVOTE_LAUNCH_CHECK("remap_gather_kernel");
+  {
+    LaunchScope scope_("remap_store_kernel", st);
+    remap_store_kernel<<<grid, 256, 0, st>>>(token_pos, total_tokens, tmp, cu, budget, Hkv);
+  }
+  GVOTE_LAUNCH_CHECK("remap_store_kernel");
   return GVOTE_OK;
 }
 

@@ -41,11 +41,11 @@ __global__ void xstage_kernel(const float* __restrict__ H, const T* __restrict__
 // table[r][0..3][j] = cos((N-1) w_j), sin((N-1) w_j), mean_i cos((N+i) w_j), mean_i sin((N+i) w_j).
 // The means use the closed form of a sum of equally spaced angles:
 //   sum_{i<n} e^{i(a + i w)} = e^{i(a + (n-1) w/2)} * sin(n w/2) / sin(w/2).
-__global__ void rope_table_kernel(const int32_t* __restrict__ cu, int d_k, double theta, int n_f,
-                                  float* __restrict__ table) {
+__global__ void rope_table_kernel(const int32_t* __restrict__ cu, const int32_t* __restrict__ seq_len, int d_k,
+                                  double theta, int n_f, float* __restrict__ table) {
   const int r = blockIdx.x, half = d_k / 2;
   for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    const double N = (double)(cu[r + 1] - cu[r]);
+    const double N = seq_len ? (double)seq_len[r] : (double)(cu[r + 1] - cu[r]);   // tokens seen so far
     const double w = pow(theta, -2.0 * (double)j / (double)d_k);
     double s0, c0, sm, cm;
     sincos((N - 1.0) * w, &s0, &c0);
@@ -199,7 +199,7 @@ int32_t launch_project_staged(const gvote_params* p, const __nv_bfloat16* X, con
 int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* h_last, int64_t h_last_ld,
                        const int32_t* h_last_rows_from_cu, const void* W_q, int64_t wq_ld, const float* b_q,
                        const int32_t* cu, int32_t batch, const WorkspaceMap& m, char* ws, __nv_bfloat16* Q,
-                       cudaStream_t st) {
+                       cudaStream_t st, const int32_t* seq_len) {
   const int d_h = p->d_h, S = p->S;
   __nv_bfloat16* X = reinterpret_cast<__nv_bfloat16*>(ws + m.x_bf16);
   float* table = reinterpret_cast<float*>(ws + m.rope);
@@ -216,7 +216,7 @@ int32_t launch_project(const gvote_params* p, const float* H_tilde, const void* 
   GVOTE_LAUNCH_CHECK("xstage_kernel");
   {
     LaunchScope scope_("rope_table_kernel", st);
-    rope_table_kernel<<<batch, 64, 0, st>>>(cu, p->d_k, p->rope_theta, p->n_f, table);
+    rope_table_kernel<<<batch, 64, 0, st>>>(cu, seq_len, p->d_k, p->rope_theta, p->n_f, table);
   }
   GVOTE_LAUNCH_CHECK("rope_table_kernel");
   return launch_project_staged(p, X, table, W_q, wq_ld, b_q, batch, m, ws, Q, st);

@@ -91,11 +91,12 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   const __grid_constant__ CUtensorMap tmQr, const int32_t* __restrict__ cu, int Hq, int G, int S1,
                   int d_k, int row_chunks, int stages, int n_out, float scale, int64_t n_tiles_total,
                   float* __restrict__ logits, uint16_t* __restrict__ keys16, uint32_t* __restrict__ rowmax,
-                  int32_t* __restrict__ status) {
+                  int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int r = blockIdx.z;
   const int kh = blockIdx.y / row_chunks, chunk = blockIdx.y % row_chunks;
-  const int start = cu[r], N = cu[r + 1] - start;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
   const int tiles = (N + kTileKeys - 1) / kTileKeys;
   const int kchunks = d_k / 64;
   const int S = S1 - 1;
@@ -262,7 +263,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         for (int i = 0; i < kRealCols; ++i) {
           if (i < G) {
             const float l = __uint_as_float(w[i]) * scale;
-            if (valid) Lreq[((int64_t)(kh * G + i) * S1) * N + n] = l;
+            if (valid) Lreq[((int64_t)(kh * G + i) * S1) * Ncap + n] = l;
             const uint32_t wmax = __reduce_max_sync(0xffffffffu, valid ? ordered_key(l) : 0u);
             if (lane == 0) atomicMax(&tail->rowmax[i], wmax);
           }
@@ -287,7 +288,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         for (int rr = e; rr < kRowChunk; rr += kEpiWarps) {
           const int grow = row0 + rr;
           if (grow >= G * S) break;
-          float* dst = Lreq + (int64_t)((kh * G + grow / S) * S1 + grow % S + 1) * N + (int64_t)t * kTileKeys;
+          float* dst = Lreq + (int64_t)((kh * G + grow / S) * S1 + grow % S + 1) * Ncap + (int64_t)t * kTileKeys;
           const uint8_t* srow = obuf + (size_t)rr * (kTileKeys * 4);
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -344,7 +345,7 @@ size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens) 
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                           bool all_f32, float* logits, uint16_t* keys16, uint32_t* rowmax, int32_t* status,
-                          cudaStream_t st) {
+                          const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
   const ScoreGeometry geo = score_geometry(p);
   const int row_chunks = geo.row_chunks;
@@ -390,7 +391,7 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
   {
     LaunchScope scope_("score_umma_kernel", st);
     kern<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, tmQr, cu, Hq, G, S1, d_k, row_chunks, stages, n_out, scale,
-                                           n_tiles_total, logits, keys16, rowmax, status);
+                                           n_tiles_total, logits, keys16, rowmax, status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_umma_kernel");
   return GVOTE_OK;

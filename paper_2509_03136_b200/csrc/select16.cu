@@ -381,11 +381,13 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
                    const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int RC, int row_chunks,
                    int64_t n_tiles_total, float scale, const int32_t* __restrict__ b_step, int64_t row_words,
-                   uint32_t* __restrict__ mask, int bitrow_bytes, int cand_per_thread) {
+                   uint32_t* __restrict__ mask, int bitrow_bytes, int cand_per_thread,
+                   const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint8_t dyn_smem[];   // [bit row | candidate lists]
   __shared__ Sel16Shared sh;
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
-  const int start = cu[r], N = cu[r + 1] - start;
+  const int start = cu[r];
+  const int N = valid_keys(kv_len, r, Hq / G, g / G, cu[r + 1] - start);
   if (N <= 0) return;
   const int k = b_step[r * Hq + g];
   if (k <= 0) return;
@@ -742,7 +744,8 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
 
 int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                       int64_t k_tok, int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens,
-                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, cudaStream_t st) {
+                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, const int32_t* kv_len,
+                      cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   const ScoreGeometry geo = score_geometry(p);
   dim3 grid(p->S, Hq, batch);
@@ -764,7 +767,7 @@ int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_
     LaunchScope scope_("topk16_rows_kernel", st);
     topk16_rows_kernel<<<grid, kThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
                                                      geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
-                                                     row_words, mask, bitrow_bytes, cand_per_thread);
+                                                     row_words, mask, bitrow_bytes, cand_per_thread, kv_len);
   }
   GVOTE_LAUNCH_CHECK("topk16_rows_kernel");
   return GVOTE_OK;

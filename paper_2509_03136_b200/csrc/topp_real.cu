@@ -118,7 +118,7 @@ __device__ __forceinline__ void block_scan_pair(uint32_t c, unsigned long long m
 __global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kThreads)
 real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
                  const uint32_t* __restrict__ rowmax, float p_nuc, int include_c0, int64_t row_words,
-                 uint32_t* __restrict__ mask, int32_t* __restrict__ b_step) {
+                 uint32_t* __restrict__ mask, int32_t* __restrict__ b_step, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint8_t dyn[];
   ClusterShared& cs = *reinterpret_cast<ClusterShared*>(dyn);
   // The generic radix search and the emission (rare routes of the first CTA) work in the space of the
@@ -129,13 +129,14 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
   const int crank = (int)cluster.block_rank();
   ClusterShared& lead = *cluster.map_shared_rank(&cs, 0);
   const int r = blockIdx.z, g = blockIdx.y;
-  const int start = cu[r], N = cu[r + 1] - start;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, g / G, Ncap);
   const int tid = threadIdx.x, lane = tid & 31;
   if (N <= 0) {                          // uniform over the cluster: nobody reaches a cluster barrier
     if (crank == 0 && tid == 0) b_step[r * Hq + g] = 0;
     return;
   }
-  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1) * N;
+  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1) * Ncap;
   const float mx = key_to_float(rowmax[r * Hq + g]);
   const float cut = tail_cut(N, p_nuc);
   const int per = (N + kClusterCtas - 1) / kClusterCtas;
@@ -394,7 +395,8 @@ size_t real_topp_scratch_bytes(const gvote_params* p, int32_t batch) {
 uint32_t* real_topp_rowmax(char* scratch) { return reinterpret_cast<uint32_t*>(scratch); }
 
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, cudaStream_t st) {
+                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, const int32_t* kv_len,
+                         cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads, S1 = p->S + 1;
   const uint32_t* rowmax = reinterpret_cast<const uint32_t*>(scratch);
   (void)max_N;
@@ -405,7 +407,7 @@ int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32
   {
     LaunchScope scope_("real_topp_kernel", st);
     real_topp_kernel<<<grid, kThreads, sizeof(ClusterShared), st>>>(logits, cu, Hq, G, S1, rowmax, p->p_nuc,
-                                                                    p->include_c0, row_words, mask, b_step);
+                                                                    p->include_c0, row_words, mask, b_step, kv_len);
   }
   GVOTE_LAUNCH_CHECK("real_topp_kernel");
   return GVOTE_OK;

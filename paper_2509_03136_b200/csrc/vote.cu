@@ -94,13 +94,14 @@ constexpr int kToppThreads = 1024;
 __global__ void __launch_bounds__(kToppThreads)
 topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
                  int rows_per_head, float p_nuc, int include_c0, int64_t row_words, uint32_t* __restrict__ mask,
-                 int32_t* __restrict__ b_step, int row_elems) {
+                 int32_t* __restrict__ b_step, int row_elems, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) float row_sm[];
   __shared__ SelShared sh;
   const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x;   // row < rows_per_head
-  const int start = cu[r], N = cu[r + 1] - start;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, g / G, Ncap);
   if (N <= 0) { if (row == 0 && threadIdx.x == 0) b_step[r * Hq + g] = 0; return; }
-  const float* Lg = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  const float* Lg = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * Ncap;
   const int tid = threadIdx.x, nthr = blockDim.x;
 
   // the row is staged in shared memory when it fits (eight loads in flight per thread), so the
@@ -160,15 +161,17 @@ topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
 // One CTA per synthetic row: the b_step[g] largest logits, ties to the lower index.
 __global__ void __launch_bounds__(kSelThreads)
 topk_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
-                 const int32_t* __restrict__ b_step, int64_t row_words, uint32_t* __restrict__ mask) {
+                 const int32_t* __restrict__ b_step, int64_t row_words, uint32_t* __restrict__ mask,
+                 const int32_t* __restrict__ kv_len) {
   __shared__ SelShared sh;
   const int r = blockIdx.z, g = blockIdx.y, row = blockIdx.x + 1;
-  const int start = cu[r], N = cu[r + 1] - start;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, g / G, Ncap);
   if (N <= 0) return;
   int k = b_step[r * Hq + g];
   if (k <= 0) return;
   if (k > N) k = N;
-  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * N;
+  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * Ncap;
   uint32_t t, above_cnt, eq_cnt;
   unsigned long long above_mass;
   radix_threshold<false>(L, N, 0.f, (unsigned long long)k, sh, t, above_cnt, above_mass, eq_cnt);
@@ -223,19 +226,21 @@ budget_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu,
 bool score_umma_supported(const gvote_params* p);
 int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                       int64_t k_tok, int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens,
-                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, cudaStream_t st);
+                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, const int32_t* kv_len,
+                      cudaStream_t st);
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                           bool all_f32, float* logits, uint16_t* keys16, uint32_t* rowmax, int32_t* status,
-                          cudaStream_t st);
+                          const int32_t* kv_len, cudaStream_t st);
 uint32_t* real_topp_rowmax(char* scratch);
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, cudaStream_t st);
+                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, const int32_t* kv_len,
+                         cudaStream_t st);
 
 int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                     uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs, const WorkspaceMap& m,
-                    char* ws, cudaStream_t st) {
+                    char* ws, cudaStream_t st, const int32_t* kv_len) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
   float* logits = reinterpret_cast<float*>(ws + m.logits);
   uint16_t* keys16 = reinterpret_cast<uint16_t*>(ws + m.keys16);
@@ -251,7 +256,7 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
     // row maxima and mass histograms of the current-query rows start from zero
     if (!all_f32) GVOTE_CUDA_CHECK(cudaMemsetAsync(ws + m.real_scratch, 0, m.real_scratch_bytes, st));
     const int32_t rc = launch_score_umma(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, all_f32, logits,
-                                         keys16, real_topp_rowmax(ws + m.real_scratch), status, st);
+                                         keys16, real_topp_rowmax(ws + m.real_scratch), status, kv_len, st);
     if (rc == GVOTE_OK) tensor_path = true;
     else if (rc != GVOTE_ERR_UNSUPPORTED_SHAPE) return rc;
   }
@@ -285,26 +290,26 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
   if (p->sel_mode == GVOTE_SEL_TOPK_C0) {
     if (tensor_path && !all_f32) {
       const int32_t rc = launch_real_topp(p, logits, cu, batch, max_N, ws + m.real_scratch, m.row_words, mask, b_step,
-                                          st);
+                                          kv_len, st);
       if (rc != GVOTE_OK) return rc;
     } else {
       dim3 g1(1, Hq, batch);
       {
         LaunchScope scope_("topp_rows_kernel", st);
         topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0,
-                                                              m.row_words, mask, b_step, topp_row_elems);
+                                                              m.row_words, mask, b_step, topp_row_elems, kv_len);
       }
       GVOTE_LAUNCH_CHECK("topp_rows_kernel");
     }
     dim3 g2(p->S, Hq, batch);
     if (tensor_path && !all_f32) {
       const int32_t rc = launch_topk16(p, keys16, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, b_step,
-                                       m.row_words, mask, st);
+                                       m.row_words, mask, kv_len, st);
       if (rc != GVOTE_OK) return rc;
     } else {
       {
         LaunchScope scope_("topk_rows_kernel", st);
-        topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask);
+        topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask, kv_len);
       }
       GVOTE_LAUNCH_CHECK("topk_rows_kernel");
     }
@@ -313,7 +318,7 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
     {
       LaunchScope scope_("topp_rows_kernel", st);
       topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0,
-                                                            m.row_words, mask, b_step, topp_row_elems);
+                                                            m.row_words, mask, b_step, topp_row_elems, kv_len);
     }
     GVOTE_LAUNCH_CHECK("topp_rows_kernel");
   }

@@ -23,7 +23,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
     "gvote_workspace_bytes", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
-    "gvote_compact", "gvote_pack", "gvote_overlap", "gvote_compress", "gvote_compress_moments", "gvote_compress_host", "gvote_host_arena_release",
+    "gvote_compact", "gvote_pack", "gvote_overlap", "gvote_compress", "gvote_compress_moments", "gvote_recompress", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
@@ -69,6 +69,9 @@ def load():
     lib.gvote_compress_moments.restype = i32
     lib.gvote_compress_moments.argtypes = [P, vp, vp, vp, vp, i64, vp, vp, vp, i64, i64, vp, i32, i64, i64, vp, vp, vp,
                                            vp, sz, vp]
+    lib.gvote_recompress.restype = i32
+    lib.gvote_recompress.argtypes = [P, vp, vp, vp, vp, i64, vp, vp, vp, i64, i64, vp, vp, vp, vp, i32, i64, i64, vp, vp,
+                                     vp, vp, sz, vp]
     lib.gvote_fit_static.restype = i32
     lib.gvote_fit_static.argtypes = [P, vp, i64, vp, i32, i64, vp, vp, vp]
     lib.gvote_sample.restype = i32
@@ -210,6 +213,26 @@ def gvote_compress_moments(p, mu, var, h_last, W_q, b_q, K, V, cu_seqlens, geom,
                                          _ptr(b_q), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(cu_seqlens),
                                          batch, total, max_N, _ptr(mask), _ptr(budget), _ptr(b_step), _ptr(ws),
                                          ws.numel(), _stream()), "gvote_compress_moments")
+
+
+def gvote_recompress(p, mu, var, h_last, W_q, b_q, K, V, cu_seqlens, kv_len, seq_len, token_pos, geom, mask, budget,
+                     b_step, ws) -> None:
+    """The pass on a cache pruned before: kv_len [batch, n_kv_heads] rows per head, seq_len [batch] tokens
+    seen, token_pos [n_kv_heads, total] slot -> position map (or None), compacted with the rows."""
+    batch, total, max_N = geom
+    _dev(mu, torch.float32, "mu"); _dev(var, torch.float32, "var")
+    _dev(h_last, torch.float32 if p.h_dtype == DTYPE_F32 else torch.bfloat16, "h_last")
+    _dev(W_q, torch.bfloat16, "W_q", dense=False); _dev(K, torch.bfloat16, "K", dense=False); _dev(V, torch.bfloat16, "V", dense=False)
+    _dev(mask, torch.int32, "mask"); _dev(budget, torch.int32, "budget"); _dev(b_step, torch.int32, "b_step")
+    _dev(kv_len, torch.int32, "kv_len"); _dev(seq_len, torch.int32, "seq_len")
+    if token_pos is not None:
+        _dev(token_pos, torch.int32, "token_pos")
+    if K.stride() != V.stride():
+        raise ValueError("K and V must share strides")
+    _check(load().gvote_recompress(ctypes.byref(p), _ptr(mu), _ptr(var), _ptr(h_last), _ptr(W_q), W_q.stride(0),
+                                   _ptr(b_q), _ptr(K), _ptr(V), K.stride(1), K.stride(0), _ptr(cu_seqlens),
+                                   _ptr(kv_len), _ptr(seq_len), _ptr(token_pos), batch, total, max_N, _ptr(mask),
+                                   _ptr(budget), _ptr(b_step), _ptr(ws), ws.numel(), _stream()), "gvote_recompress")
 
 
 FIT_STATIC_MAX_ENTRIES = 131072

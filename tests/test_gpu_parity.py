@@ -523,6 +523,144 @@ def test_compress_from_streamed_moments(gv, name):
     _check_compress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(name == "small2")), runner=_run_compress_moments)
 
 
+# ----------------------------------------------------------------------------- the pass applied again
+def _pruned_cache(cfg, li, rng, n_new, empty_head=None):
+    """A cache as an earlier pass and some decoding would leave it: per (request, KV head) a random
+    subset of the older tokens, in order, then the n_new latest tokens; the rest of each slab holds
+    rows that must be ignored (large values, so that a leak shows).  Returns slabs and the map."""
+    Hkv, T = cfg.n_kv_heads, cfg.total_tokens
+    K = np.full_like(li.K, 0x4700)            # bf16 32768.0 in every unused row
+    V = np.full_like(li.V, 0x4700)
+    kv_len = np.zeros((cfg.batch, Hkv), dtype=np.int32)
+    token_pos = np.full((Hkv, T), -1, dtype=np.int32)
+    kept = []
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        N = b - a
+        old = max(N - n_new, 0)
+        per_head = []
+        for h in range(Hkv):
+            if empty_head == (r, h):
+                idx = np.zeros(0, dtype=np.int64)
+            else:
+                frac = rng.uniform(0.3, 0.9)
+                idx = np.sort(rng.choice(old, size=max(1, int(frac * old)), replace=False)) if old > 0 else np.zeros(0, dtype=np.int64)
+                idx = np.concatenate([idx, np.arange(old, N)]).astype(np.int64)
+            n = idx.shape[0]
+            K[h, a:a + n] = li.K[h, a + idx]
+            V[h, a:a + n] = li.V[h, a + idx]
+            kv_len[r, h] = n
+            token_pos[h, a:a + n] = idx
+            per_head.append(idx)
+        kept.append(per_head)
+    return K, V, kv_len, token_pos, kept
+
+
+def _check_recompress(gv, cfg, li, sel_mode="topk", n_new=5, empty_head=None, seed=70):
+    rng = np.random.default_rng(seed)
+    Ks, Vs, kv_len, token_pos, kept = _pruned_cache(cfg, li, rng, n_new, empty_head)
+    p = gv.params_from_config(cfg, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    dK, dV = gv.bf16_from_bits(Ks), gv.bf16_from_bits(Vs)
+    mu = torch.empty(cfg.batch, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p, d["h"], d["cu"], geom, mu, var, ws)
+    cu = li.cu_seqlens
+    h_last = torch.from_numpy(np.stack([li.h[int(cu[r + 1]) - 1] for r in range(cfg.batch)])).cuda()
+    # tokens seen: more than the slab holds (the slabs of a pruned cache are shorter than its history)
+    seen = (np.diff(cu) + 37 * (np.arange(cfg.batch) + 1)).astype(np.int32)
+    seq_len = torch.from_numpy(seen).cuda()
+    d_len = torch.from_numpy(kv_len).cuda()
+    d_pos = torch.from_numpy(token_pos).cuda()
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_recompress(p, mu, var, h_last, d["W_q"], d["b_q"], dK, dV, d["cu"], d_len, seq_len, d_pos, geom, mask,
+                        budget, b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    mask, budget, b_step = mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy()
+    Kg, Vg, pos_g = gv.bits_from_bf16(dK), gv.bits_from_bf16(dV), d_pos.cpu().numpy()
+
+    W = o.bf16_bits_to_f64(li.W_q)
+    kw = pu.oracle_kwargs(cfg)
+    n_s = kw.pop("n_s")
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    for r in range(cfg.batch):
+        a, b = int(cu[r]), int(cu[r + 1])
+        N = b - a
+        m64, v64 = o.fit(li.h[a:b].astype(np.float64), n_s)
+        heads = [o.bf16_bits_to_f64(Ks[h, a:a + kv_len[r, h]]) for h in range(cfg.n_kv_heads)]
+        res = o.recompress_request(m64, v64, li.h[b - 1].astype(np.float64), W, li.b_q, heads, int(seen[r]), request_id=r,
+                                   sel_mode=sel_mode, token_pos=kept[r], **kw)
+        for h in range(cfg.n_kv_heads):
+            n = int(kv_len[r, h])
+            row = gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N)
+            assert not row[n:].any(), "a slot beyond the head's rows was kept"
+            gm = row[:n]
+            if n == 0:
+                assert budget[r, h] == 0 and not b_step[r, h * G:(h + 1) * G].any()
+                continue
+            pu.check_vote_against_oracle(res.Q[h * G:(h + 1) * G], heads[h][None], kw["p_nuc"], sel_mode, False,
+                                         gm[None], b_step[r, h * G:(h + 1) * G], mass_band=2e-2, logit_band=2e-2)
+            assert abs(int(budget[r, h]) - int(res.budget[h])) <= max(2, 0.005 * n)
+            keep = np.nonzero(gm)[0]
+            assert budget[r, h] == keep.shape[0]
+            # rows and map entries move together, bit for bit
+            assert np.array_equal(Kg[h, a:a + keep.shape[0]], Ks[h, a + keep])
+            assert np.array_equal(Vg[h, a:a + keep.shape[0]], Vs[h, a + keep])
+            assert np.array_equal(pos_g[h, a:a + keep.shape[0]], kept[r][h][keep])
+
+
+@pytest.mark.parametrize("idx", [2, 3])
+def test_recompress_small(gv, idx):
+    """The pass on a pruned, grown cache (heads of different lengths, positions from the tokens seen)
+    against the oracle's per-head restatement; same bands as the whole-pass checks."""
+    cfg = _small_cfgs()[idx]
+    _check_recompress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx == 3)))
+
+
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk")])
+def test_recompress_configs(gv, name, mode):
+    cfg = synth.make_config(name)
+    _check_recompress(gv, cfg, synth.make_layer(cfg, 0), mode, n_new=17)
+
+
+def test_recompress_head_without_rows(gv):
+    cfg = _small_cfgs()[2]
+    _check_recompress(gv, cfg, synth.make_layer(cfg, 0), empty_head=(1, 0), n_new=3)
+
+
+def test_recompress_of_a_full_cache_is_the_plain_pass(gv):
+    """kv_len = N for every head and seq_len = N: the same bits as gvote_compress_moments."""
+    cfg = synth.make_config("c1")
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    outs = []
+    for again in (False, True):
+        d = pu.upload_layer(li, gv, torch)
+        mu = torch.empty(cfg.batch, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+        gv.gvote_fit(p, d["h"], d["cu"], geom, mu, var, ws)
+        cu = li.cu_seqlens
+        h_last = torch.from_numpy(np.stack([li.h[int(cu[r + 1]) - 1] for r in range(cfg.batch)])).cuda()
+        mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+        budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+        b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+        if again:
+            lens = torch.from_numpy(np.diff(cu).astype(np.int32)).cuda()
+            kv_len = lens[:, None].expand(cfg.batch, cfg.n_kv_heads).contiguous()
+            gv.gvote_recompress(p, mu, var, h_last, d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], kv_len, lens, None,
+                                geom, mask, budget, b_step, ws)
+        else:
+            gv.gvote_compress_moments(p, mu, var, h_last, d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask,
+                                      budget, b_step, ws)
+        outs.append((mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"])))
+    for x, y in zip(*outs):
+        assert np.array_equal(x, y)
+
+
 def test_compress_with_an_empty_request(gv):
     """A request without cached tokens in the middle of a batch: nothing is read or written for it
     (budget 0, |C0| 0) and its neighbours are unaffected."""
