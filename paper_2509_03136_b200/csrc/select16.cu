@@ -459,55 +459,74 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
     uint32_t* bitrow = reinterpret_cast<uint32_t*>(dyn_smem);
     uint32_t* cand = reinterpret_cast<uint32_t*>(dyn_smem + bitrow_bytes);      // [cand_per_thread][kThreads]
     const __half2 tlo = pair_of(raw_of(lo)), thi = pair_of(raw_of(hi));
-    uint32_t a16 = 0;   // 16 per key above the bracket
-    int cnt = 0;        // bracket keys this thread has met
-    for (int base = 0; base < rv.nv8; base += kThreads * kLoads) {
+    uint8_t* bitbytes = reinterpret_cast<uint8_t*>(bitrow);     // byte v8 of the bit row = the 8 keys of vector v8
+    uint32_t above_cnt = 0;   // keys above the bracket this thread has met
+    int cnt = 0;              // bracket keys this thread has met
+    // one vector: mark the keys above the bracket, list the keys inside it
+    auto take = [&](const uint4& v, int v8) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t ge[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ge[j] = __hge2_mask(as_h2(w[j]), tlo);
+      uint32_t bits = 0;
+      if ((ge[0] | ge[1] | ge[2] | ge[3]) != 0u) {
+        // bit 2j of the low half and bit 2j+1 of the high half of word j mark its two keys
+        uint32_t gacc = 0, cacc = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t pick = (1u << (2 * j)) | (1u << (17 + 2 * j));
+          const uint32_t gt = __hgt2_mask(as_h2(w[j]), thi);
+          gacc |= gt & pick;
+          cacc |= (ge[j] & ~gt) & pick;
+        }
+        bits = (gacc | (gacc >> 16)) & 0xffu;
+        above_cnt += __popc(bits);
+        uint32_t cbits = (cacc | (cacc >> 16)) & 0xffu;
+        const uint32_t tag = (uint32_t)(v8 / kThreads) << 3;
+        while (cbits) {
+          const int j = __ffs(cbits) - 1;
+          cbits &= cbits - 1;
+          const uint32_t ww = (j < 4) ? ((j < 2) ? w[0] : w[1]) : ((j < 6) ? w[2] : w[3]);
+          const uint32_t key = (j & 1) ? (ww >> 16) : (ww & 0xffffu);
+          if (cnt < cand_per_thread) {
+            cand[cnt * kThreads + tid] = (key << 16) | tag | (uint32_t)j;
+            ++cnt;
+          } else {                                     // the rare key beyond the slice: shared spill list
+            const uint32_t slot = atomicAdd(&sh.novf, 1u);
+            if (slot < (uint32_t)kOvfCap) { sh.ovf_n[slot] = (uint32_t)(v8 * 8 + j); sh.ovf_key[slot] = (uint16_t)key; }
+          }
+        }
+      }
+      return bits;
+    };
+    // Vector v8 = base + u * kThreads + tid sits in tile (base / 16) + 8 u + tid / 16 at the thread's own
+    // chunk position (tid % 16) ^ swz: whole batches need no index arithmetic and no bounds checks.
+    const int full_end = ((N >> 3) / (kThreads * kLoads)) * (kThreads * kLoads);   // vectors in whole batches of whole vectors
+    const uint16_t* tp = rv.grow + (int64_t)(tid >> 4) * rv.tile_stride + ((((uint32_t)tid & 15u) ^ rv.swz) << 3);
+    const int64_t u_step = (int64_t)(kThreads / 16) * rv.tile_stride;
+    int base = 0;
+    for (; base < full_end; base += kThreads * kLoads, tp += kLoads * u_step) {
+      uint4 buf[kLoads];
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) buf[u] = *reinterpret_cast<const uint4*>(tp + u * u_step);
+#pragma unroll
+      for (int u = 0; u < kLoads; ++u) {
+        const int v8 = base + u * kThreads + tid;
+        bitbytes[v8] = (uint8_t)take(buf[u], v8);
+      }
+    }
+    for (; base < rv.nv8; base += kThreads * kLoads) {          // the ragged end: padded loads
       uint4 buf[kLoads];
 #pragma unroll
       for (int u = 0; u < kLoads; ++u) buf[u] = rv.load(base + u * kThreads + tid);
 #pragma unroll
       for (int u = 0; u < kLoads; ++u) {
         const int v8 = base + u * kThreads + tid;
-        const uint32_t w[4] = {buf[u].x, buf[u].y, buf[u].z, buf[u].w};
-        uint32_t ge[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) ge[j] = __hge2_mask(as_h2(w[j]), tlo);
-        uint32_t bits = 0;
-        if ((ge[0] | ge[1] | ge[2] | ge[3]) != 0u) {
-          // bit 2j of the low half and bit 2j+1 of the high half of word j mark its two keys
-          uint32_t gacc = 0, cacc = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t pick = (1u << (2 * j)) | (1u << (17 + 2 * j));
-            const uint32_t gt = __hgt2_mask(as_h2(w[j]), thi);
-            a16 += __popc(gt);
-            gacc |= gt & pick;
-            cacc |= (ge[j] & ~gt) & pick;
-          }
-          bits = (gacc | (gacc >> 16)) & 0xffu;
-          uint32_t cbits = (cacc | (cacc >> 16)) & 0xffu;
-          const uint32_t tag = (uint32_t)(v8 / kThreads) << 3;
-          while (cbits) {
-            const int j = __ffs(cbits) - 1;
-            cbits &= cbits - 1;
-            const uint32_t ww = (j < 4) ? ((j < 2) ? w[0] : w[1]) : ((j < 6) ? w[2] : w[3]);
-            const uint32_t key = (j & 1) ? (ww >> 16) : (ww & 0xffffu);
-            if (cnt < cand_per_thread) {
-              cand[cnt * kThreads + tid] = (key << 16) | tag | (uint32_t)j;
-              ++cnt;
-            } else {                                     // the rare key beyond the slice: shared spill list
-              const uint32_t slot = atomicAdd(&sh.novf, 1u);
-              if (slot < (uint32_t)kOvfCap) { sh.ovf_n[slot] = (uint32_t)(v8 * 8 + j); sh.ovf_key[slot] = (uint16_t)key; }
-            }
-          }
-        }
-        uint32_t word = bits << (8 * (lane & 3));
-        word |= __shfl_xor_sync(0xffffffffu, word, 1);
-        word |= __shfl_xor_sync(0xffffffffu, word, 2);
-        if ((lane & 3) == 0 && (v8 >> 2) < words) bitrow[v8 >> 2] = word;
+        const uint32_t bits = take(buf[u], v8);
+        if (v8 < words * 4) bitbytes[v8] = (uint8_t)bits;
       }
     }
-    const uint32_t A = block_sum(sh, a16 >> 4);
+    const uint32_t A = block_sum(sh, above_cnt);
     const uint32_t novf = sh.novf;
     const uint32_t C = block_sum(sh, (uint32_t)cnt) + novf;
     bool settled = novf <= (uint32_t)kOvfCap && A <= (uint32_t)k && A + C >= (uint32_t)k;
