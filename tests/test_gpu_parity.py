@@ -721,6 +721,12 @@ def test_compress_full_size_c4_layer(gv):
         _check_compress(gv, cfg, synth.make_layer(cfg, layer), layer_id=layer)
 
 
+def test_recompress_full_size_c2_layer(gv):
+    """The pass applied again at the 32K workload's shapes: heads of 10K to 30K rows each, 256 of them new."""
+    cfg = synth.make_config("c2")
+    _check_recompress(gv, cfg, synth.make_layer(cfg, 3), n_new=256, seed=71)
+
+
 def test_compress_host_variant_matches_device_variant(gv):
     cfg = synth.make_config("c0")
     li = synth.make_layer(cfg, 0)
