@@ -376,7 +376,11 @@ __device__ void window_find(Sel16Shared& sh, uint32_t need) {
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads, 8)
+// SWEEP_LOADS: 16-byte loads a thread keeps in flight in the one-sweep route.  Rows short enough for
+// seven or eight CTAs per SM hide the latency by occupancy (4); long rows, whose bit row and lists
+// leave room for two or three CTAs only, need it per thread (8, 16).
+template <int SWEEP_LOADS>
+__global__ void __launch_bounds__(kThreads, SWEEP_LOADS <= 4 ? 8 : (SWEEP_LOADS <= 8 ? 4 : 2))
 topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __restrict__ Q,
                    const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int RC, int row_chunks,
@@ -501,26 +505,26 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
     };
     // Vector v8 = base + u * kThreads + tid sits in tile (base / 16) + 8 u + tid / 16 at the thread's own
     // chunk position (tid % 16) ^ swz: whole batches need no index arithmetic and no bounds checks.
-    const int full_end = ((N >> 3) / (kThreads * kLoads)) * (kThreads * kLoads);   // vectors in whole batches of whole vectors
+    const int full_end = ((N >> 3) / (kThreads * SWEEP_LOADS)) * (kThreads * SWEEP_LOADS);   // vectors in whole batches of whole vectors
     const uint16_t* tp = rv.grow + (int64_t)(tid >> 4) * rv.tile_stride + ((((uint32_t)tid & 15u) ^ rv.swz) << 3);
     const int64_t u_step = (int64_t)(kThreads / 16) * rv.tile_stride;
     int base = 0;
-    for (; base < full_end; base += kThreads * kLoads, tp += kLoads * u_step) {
-      uint4 buf[kLoads];
+    for (; base < full_end; base += kThreads * SWEEP_LOADS, tp += SWEEP_LOADS * u_step) {
+      uint4 buf[SWEEP_LOADS];
 #pragma unroll
-      for (int u = 0; u < kLoads; ++u) buf[u] = *reinterpret_cast<const uint4*>(tp + u * u_step);
+      for (int u = 0; u < SWEEP_LOADS; ++u) buf[u] = *reinterpret_cast<const uint4*>(tp + u * u_step);
 #pragma unroll
-      for (int u = 0; u < kLoads; ++u) {
+      for (int u = 0; u < SWEEP_LOADS; ++u) {
         const int v8 = base + u * kThreads + tid;
         bitbytes[v8] = (uint8_t)take(buf[u], v8);
       }
     }
-    for (; base < rv.nv8; base += kThreads * kLoads) {          // the ragged end: padded loads
-      uint4 buf[kLoads];
+    for (; base < rv.nv8; base += kThreads * SWEEP_LOADS) {          // the ragged end: padded loads
+      uint4 buf[SWEEP_LOADS];
 #pragma unroll
-      for (int u = 0; u < kLoads; ++u) buf[u] = rv.load(base + u * kThreads + tid);
+      for (int u = 0; u < SWEEP_LOADS; ++u) buf[u] = rv.load(base + u * kThreads + tid);
 #pragma unroll
-      for (int u = 0; u < kLoads; ++u) {
+      for (int u = 0; u < SWEEP_LOADS; ++u) {
         const int v8 = base + u * kThreads + tid;
         const uint32_t bits = take(buf[u], v8);
         if (v8 < words * 4) bitbytes[v8] = (uint8_t)bits;
@@ -781,12 +785,15 @@ int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_
     cand_per_thread = (int)ceil(share + 1.7 * sqrt(share));
   }
   const size_t smem = (size_t)bitrow_bytes + (size_t)cand_per_thread * kThreads * sizeof(uint32_t);
-  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topk16_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  // CTAs an SM holds: dynamic + static shared memory + 1 KB reserved per CTA, of 228 KB
+  const int per_sm = (int)((228 * 1024) / (smem + sizeof(Sel16Shared) + 1024));
+  auto kern = per_sm >= 5 ? topk16_rows_kernel<4> : (per_sm >= 3 ? topk16_rows_kernel<8> : topk16_rows_kernel<16>);
+  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("topk16_rows_kernel", st);
-    topk16_rows_kernel<<<grid, kThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC,
-                                                     geo.row_chunks, (total_tokens >> 7) + batch, scale, b_step,
-                                                     row_words, mask, bitrow_bytes, cand_per_thread, kv_len);
+    kern<<<grid, kThreads, smem, st>>>(keys16, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, geo.RC, geo.row_chunks,
+                                       (total_tokens >> 7) + batch, scale, b_step, row_words, mask, bitrow_bytes,
+                                       cand_per_thread, kv_len);
   }
   GVOTE_LAUNCH_CHECK("topk16_rows_kernel");
   return GVOTE_OK;
