@@ -81,6 +81,35 @@ def test_fit_matches_oracle(gv, name, lens, d_h, n_s):
         assert np.abs(mu[r].cpu().numpy() - m).max() <= 1e-5 * np.sqrt(v).max() + 1e-6 * np.abs(m).max()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_fit_strided_rows_ragged_strips_and_long_chunks(gv, dtype):
+    """Hidden states that are a column window of a wider buffer (row stride > d_h), d_h that leaves a
+    partial 256-channel strip, one long request (many whole stages per chunk plus a ragged last one)
+    next to short ones; the mean sits far from zero relative to the spread."""
+    rng = np.random.default_rng(9)
+    lens, d_h, ld, n_s = (9001, 70, 333), 328, 344, 4
+    T = sum(lens)
+    wide = (rng.normal(size=(T, ld)) * rng.uniform(0.05, 2, size=ld) + rng.normal(size=ld) * 40).astype(np.float32)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    bf = dtype == "bf16"
+    buf = torch.from_numpy(wide).cuda()
+    if bf:
+        buf = buf.bfloat16()
+    h = buf[:, 8:8 + d_h]                                  # 16-byte aligned window, stride ld
+    href = h.double().cpu().numpy()
+    p = gv.make_params(d_h=d_h, n_q_heads=2, n_kv_heads=1, d_k=16, rope_theta=1e4, S=2, p_nuc=0.9, n_f=4, n_s=n_s,
+                       seed=0, h_dtype=gv.DTYPE_BF16 if bf else gv.DTYPE_F32)
+    geom = (len(lens), T, max(lens))
+    ws = gv.alloc_workspace(p, *geom)
+    mu = torch.empty(len(lens), d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p, h, torch.from_numpy(cu).cuda(), geom, mu, var, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    for r in range(len(lens)):
+        m, v = o.fit(href[cu[r]:cu[r + 1]], n_s)
+        assert np.allclose(var[r].cpu().numpy(), v, rtol=1e-5, atol=0)
+        assert np.abs(mu[r].cpu().numpy() - m).max() <= 1e-5 * np.sqrt(v).max() + 1e-6 * np.abs(m).max()
+
+
 def test_fit_bf16_hidden_states(gv):
     rng = np.random.default_rng(8)
     h = torch.from_numpy(rng.normal(size=(300, 128)).astype(np.float32)).bfloat16()
