@@ -62,6 +62,8 @@ struct Sel16Shared {
   int bin;
   uint32_t above;
   uint32_t inside;
+  int bin2;              // second search of a pair (sample_ranks)
+  uint32_t above2;
   uint32_t ntie;
   uint32_t novf;
   uint32_t ovf_n[kOvfCap];
@@ -79,46 +81,59 @@ __device__ __forceinline__ uint32_t block_sum(Sel16Shared& sh, uint32_t v) {
   return s;
 }
 
-// Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need).
+// Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need), found by
+// one warp: every lane returns the bin and the count in the bins above it.
+__device__ __forceinline__ void warp_find_bin256(const uint32_t* hist, uint32_t need, int lane, int& bin,
+                                                 uint32_t& above) {
+  uint32_t c = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) c += hist[lane * 8 + i];
+  uint32_t cs = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_down_sync(0xffffffffu, cs, o);
+    if (lane + o < 32) cs += t;
+  }
+  const uint32_t excl = cs - c;                          // count in the lanes above this one
+  const bool own = excl < need && excl + c >= need;
+  uint32_t a = excl;
+  int b = lane * 8 + 7;
+  if (own) {
+    for (; b > lane * 8; --b) {
+      if (a + hist[b] >= need) break;
+      a += hist[b];
+    }
+  }
+  const uint32_t who = __ballot_sync(0xffffffffu, own);
+  const int src = who ? __ffs(who) - 1 : 0;
+  bin = who ? __shfl_sync(0xffffffffu, b, src) : 0;
+  above = who ? __shfl_sync(0xffffffffu, a, src) : 0u;
+}
+
+// The same for the whole CTA on sh.hist: publishes sh.bin and sh.above.
 __device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
   if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    uint32_t c = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) c += sh.hist[lane * 8 + i];
-    uint32_t cs = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_down_sync(0xffffffffu, cs, o);
-      if (lane + o < 32) cs += t;
-    }
-    const uint32_t excl = cs - c;
-    if (lane == 0) { sh.bin = 0; sh.above = 0; }
-    __syncwarp();
-    if (excl < need && excl + c >= need) {
-      uint32_t a = excl;
-      int b = lane * 8 + 7;
-      for (; b > lane * 8; --b) {
-        if (a + sh.hist[b] >= need) break;
-        a += sh.hist[b];
-      }
-      sh.bin = b;
-      sh.above = a;
-    }
+    int bin;
+    uint32_t above;
+    warp_find_bin256(sh.hist, need, threadIdx.x, bin, above);
+    if (threadIdx.x == 0) { sh.bin = bin; sh.above = above; }
   }
   __syncthreads();
 }
 
 // The sample: vector i of `n_vecs` (at most four per thread).  A row of at most n_vecs vectors is
-// sampled completely (stride 0).  Otherwise thread t takes four consecutive vectors (64 bytes, one
-// DRAM access) from the middle of the t-th of kThreads equal stretches of the row: scattering single
-// 16-byte vectors instead costs four times the DRAM accesses for the same number of keys.
+// sampled completely (stride 0).  Otherwise the sample is kThreads runs of four consecutive vectors
+// (64 bytes, one DRAM access each; scattering single 16-byte vectors instead costs four times the
+// accesses for the same number of keys), run j taken from the middle of the j-th of kThreads equal
+// stretches of the row.  Four neighbouring lanes share a run, so a warp's load instruction asks for
+// eight 64-byte pieces instead of thirty-two 16-byte ones.
 struct Sample {
   int n_vecs, stride;
   __device__ __forceinline__ int vec(int i) const {
     if (stride == 0) return i;
     const int t = i % kThreads, u = i / kThreads;
-    return t * stride + ((stride >> 1) & ~3) + u;
+    const int run = (t >> 2) + (kThreads / 4) * u;
+    return run * stride + ((stride >> 1) & ~3) + (t & 3);
   }
 };
 
@@ -197,16 +212,30 @@ __device__ __forceinline__ SampleRegs sample_load(const RowView& rv, const Sampl
 // High byte of a key's code from the high byte hb of its half bits, and back.
 __device__ __forceinline__ uint32_t ord_hi(uint32_t hb) { return hb >= 0x80u ? 0xffu - hb : 0x80u + hb; }
 
-// Level 1: 256-bin histogram (left in sh.hist[0..256), indexed by the code's high byte) of the sampled
-// keys.  Every sampled key takes part and a few bins take most of them, so plain shared-memory
-// atomics would serialise on those addresses.  Counting goes into one 8-bit counter per (bin, lane)
-// instead, four bins to a word, word index (bin / 4) * 32 + lane: the lanes of a warp never meet, and
-// a counter takes at most (warps) * (sample keys per thread) = 4 * 32 increments, well below 256.
-// Bins are those of the raw half bits here (no per-key recoding); the fold puts them in code order.
-__device__ void sample_hist_hi(const SampleRegs& sr, Sel16Shared& sh) {
-  const int lane = threadIdx.x & 31;
+// Clears the counters sample_ranks starts from.  Called between issuing the sample's loads and
+// ranking it, so that the clearing and its barrier pass while the loads are in flight.
+__device__ __forceinline__ void sample_begin(Sel16Shared& sh) {
   for (int b = threadIdx.x; b < kWin; b += kThreads) sh.hist[b] = 0;
   __syncthreads();
+}
+
+// The sample's rank_a-th and rank_b-th largest codes (1 <= rank_a <= rank_b <= sampled keys; rank_a = 0
+// asks for the second one only).  For the second one also the number of sampled codes above it and
+// equal to it.  Every thread of the CTA calls it, after sample_begin.
+//
+// Two levels of 256 bins, both ranks at a time (warp 0 searches for rank_b, warp 1 for rank_a).
+// Level 1 bins the code's high byte.  Every sampled key takes part and a few bins take most of
+// them, so plain shared-memory atomics would serialise on those addresses: counting goes into one
+// 8-bit counter per (bin, lane) instead, four bins to a word, word index (bin / 4) * 32 + lane: the
+// lanes of a warp never meet, and a counter takes at most (warps) * (sample keys per thread) = 4 * 32
+// increments, well below 256.  Bins are those of the raw half bits here (no per-key recoding); the
+// fold puts them in code order, into the tie list's space (not in use yet).  Level 2 bins the low
+// byte of the keys whose high byte is the one found, for the two ranks side by side.
+__device__ void sample_ranks(const SampleRegs& sr, uint32_t rank_a, uint32_t rank_b, Sel16Shared& sh,
+                             uint32_t& code_a, uint32_t& code_b, uint32_t& above_b, uint32_t& equal_b) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t* bins = reinterpret_cast<uint32_t*>(sh.tie_val);
+  static_assert(kTieCap >= 256, "the folded bins borrow the tie list");
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     if (u >= sr.have) break;
@@ -222,80 +251,75 @@ __device__ void sample_hist_hi(const SampleRegs& sr, Sel16Shared& sh) {
   }
   __syncthreads();
   // fold the lanes: thread t < 64 sums word row t (raw bins 4t .. 4t+3), two bins per accumulator
-  uint32_t even = 0, odd = 0;
-  if (threadIdx.x < 64) {
-    const uint32_t* wrow = &sh.hist[threadIdx.x * 32];
+  if (tid < 64) {
+    uint32_t even = 0, odd = 0;
+    const uint32_t* wrow = &sh.hist[tid * 32];
 #pragma unroll 8
     for (int l = 0; l < 32; ++l) {
       const uint32_t w = wrow[(l + lane) & 31];           // rotated: conflict free
       even += w & 0x00ff00ffu;
       odd += (w >> 8) & 0x00ff00ffu;
     }
+    const uint32_t hb = 4u * tid;
+    bins[ord_hi(hb)] = even & 0xffffu;
+    bins[ord_hi(hb + 1)] = odd & 0xffffu;
+    bins[ord_hi(hb + 2)] = even >> 16;
+    bins[ord_hi(hb + 3)] = odd >> 16;
   }
   __syncthreads();
-  if (threadIdx.x < 64) {
-    const uint32_t hb = 4u * threadIdx.x;
-    sh.hist[ord_hi(hb)] = even & 0xffffu;
-    sh.hist[ord_hi(hb + 1)] = odd & 0xffffu;
-    sh.hist[ord_hi(hb + 2)] = even >> 16;
-    sh.hist[ord_hi(hb + 3)] = odd >> 16;
+  if (warp == 0) {
+    int bin;
+    uint32_t up;
+    warp_find_bin256(bins, rank_b, lane, bin, up);
+    if (lane == 0) { sh.bin = bin; sh.above = up; }
+  } else if (warp == 1 && rank_a) {
+    int bin;
+    uint32_t up;
+    warp_find_bin256(bins, rank_a, lane, bin, up);
+    if (lane == 0) { sh.bin2 = bin; sh.above2 = up; }
   }
+  for (int b = tid; b < 512; b += kThreads) sh.hist[b] = 0;      // level 2: [0, 256) for rank_b, [256, 512) for rank_a
   __syncthreads();
-}
-
-// Level 2: 256-bin histogram (sh.hist[0..256), indexed by the code's low byte) of the sampled keys
-// whose code has high byte `only`.
-__device__ void sample_hist_lo(const SampleRegs& sr, uint32_t only, Sel16Shared& sh) {
-  for (int b = threadIdx.x; b < 256; b += kThreads) sh.hist[b] = 0;
-  __syncthreads();
-  const bool neg = only < 0x80u;                          // codes below 0x8000 are negative numbers
-  const uint32_t raw_hb = neg ? 0xffu - only : only - 0x80u;
-  const uint32_t flip = neg ? 0xffu : 0u;
+  const uint32_t bin_b = (uint32_t)sh.bin, up_b = sh.above;
+  const uint32_t bin_a = rank_a ? (uint32_t)sh.bin2 : bin_b, up_a = rank_a ? sh.above2 : 0u;
+  const bool two = rank_a && bin_a != bin_b;
+  {
+    // codes below 0x8000 are negative numbers: their raw bits run the other way
+    const uint32_t raw_b = bin_b < 0x80u ? 0xffu - bin_b : bin_b - 0x80u, flip_b = bin_b < 0x80u ? 0xffu : 0u;
+    const uint32_t raw_a = bin_a < 0x80u ? 0xffu - bin_a : bin_a - 0x80u, flip_a = bin_a < 0x80u ? 0xffu : 0u;
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    if (u >= sr.have) break;
-    const uint32_t w[4] = {sr.v[u].x, sr.v[u].y, sr.v[u].z, sr.v[u].w};
+    for (int u = 0; u < 4; ++u) {
+      if (u >= sr.have) break;
+      const uint32_t w[4] = {sr.v[u].x, sr.v[u].y, sr.v[u].z, sr.v[u].w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t h0 = w[j] & 0xffffu, h1 = w[j] >> 16;
-      if (h0 == 0x8000u) h0 = 0u;
-      if (h1 == 0x8000u) h1 = 0u;
-      if ((h0 >> 8) == raw_hb) atomicAdd(&sh.hist[(h0 & 255u) ^ flip], 1u);
-      if ((h1 >> 8) == raw_hb) atomicAdd(&sh.hist[(h1 & 255u) ^ flip], 1u);
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          uint32_t h = e ? (w[j] >> 16) : (w[j] & 0xffffu);
+          if (h == 0x8000u) h = 0u;
+          if ((h >> 8) == raw_b) atomicAdd(&sh.hist[(h & 255u) ^ flip_b], 1u);
+          else if (two && (h >> 8) == raw_a) atomicAdd(&sh.hist[256u + ((h & 255u) ^ flip_a)], 1u);
+        }
+      }
     }
   }
   __syncthreads();
-}
-
-// The sample's rank_a-th and rank_b-th largest codes (1 <= rank_a <= rank_b <= sampled keys; rank_a = 0
-// asks for the second one only).  For the second one also the number of sampled codes above it and
-// equal to it.  Every thread of the CTA calls it.
-__device__ void sample_ranks(const SampleRegs& sr, uint32_t rank_a, uint32_t rank_b, Sel16Shared& sh,
-                             uint32_t& code_a, uint32_t& code_b, uint32_t& above_b, uint32_t& equal_b) {
-  sample_hist_hi(sr, sh);
-  uint32_t bin_a = 0, up_a = 0;
-  if (rank_a) {
-    find_bin256(sh, rank_a);
-    bin_a = (uint32_t)sh.bin;
-    up_a = sh.above;
-    __syncthreads();
+  if (warp == 0) {
+    int bin;
+    uint32_t up;
+    warp_find_bin256(sh.hist, rank_b - up_b, lane, bin, up);
+    if (lane == 0) { sh.bin = bin; sh.above = up; sh.inside = sh.hist[bin]; }
+  } else if (warp == 1 && rank_a) {
+    int bin;
+    uint32_t up;
+    warp_find_bin256(two ? sh.hist + 256 : sh.hist, rank_a - up_a, lane, bin, up);
+    if (lane == 0) sh.bin2 = bin;
   }
-  find_bin256(sh, rank_b);
-  const uint32_t bin_b = (uint32_t)sh.bin, up_b = sh.above;
   __syncthreads();
-  sample_hist_lo(sr, bin_b, sh);
-  find_bin256(sh, rank_b - up_b);
   code_b = (bin_b << 8) | (uint32_t)sh.bin;
   above_b = up_b + sh.above;
-  equal_b = sh.hist[sh.bin];
-  __syncthreads();
-  code_a = 0xffffu;
-  if (rank_a) {
-    if (bin_a != bin_b) sample_hist_lo(sr, bin_a, sh);
-    find_bin256(sh, rank_a - up_a);
-    code_a = (bin_a << 8) | (uint32_t)sh.bin;
-    __syncthreads();
-  }
+  equal_b = sh.inside;
+  code_a = rank_a ? ((bin_a << 8) | (uint32_t)sh.bin2) : 0xffffu;
 }
 
 // One sweep: A = number of keys with code > hi; hist[(c - lo) >> shift] = number of keys with code c
@@ -429,6 +453,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
     // the whole row is the sample: its k-th largest code is the threshold
     const Sample sm{rv.nv8, 0};
     const SampleRegs sr = sample_load(rv, sm);
+    sample_begin(sh);
     uint32_t unused;
     sample_ranks(sr, 0u, (uint32_t)k, sh, unused, T, above, eq);
     found = true;
@@ -448,6 +473,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
     const int r_hi = (int)floorf(rk - dlt);
     uint32_t a_s, e_s;
     const SampleRegs sr = sample_load(rv, sm);
+    sample_begin(sh);
     sample_ranks(sr, r_hi >= 1 ? (uint32_t)r_hi : 0u, (uint32_t)r_lo, sh, hi, lo, a_s, e_s);
     if (lo < kMinCode) lo = kMinCode;
     if (hi < lo) hi = lo;
