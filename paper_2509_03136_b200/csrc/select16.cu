@@ -59,6 +59,7 @@ struct Sel16Shared {
   int tie_idx[kTieCap];
   float tie_val[kTieCap];
   uint32_t red[kThreads / 32];
+  uint32_t red2[kThreads / 32];
   int bin;
   uint32_t above;
   uint32_t inside;
@@ -79,6 +80,19 @@ __device__ __forceinline__ uint32_t block_sum(Sel16Shared& sh, uint32_t v) {
 #pragma unroll
   for (int w = 0; w < kThreads / 32; ++w) s += sh.red[w];
   return s;
+}
+
+// Two sums over the CTA behind one pair of barriers.
+__device__ __forceinline__ void block_sum2(Sel16Shared& sh, uint32_t v0, uint32_t v1, uint32_t& s0, uint32_t& s1) {
+  v0 = (uint32_t)warp_sum_i((int)v0);
+  v1 = (uint32_t)warp_sum_i((int)v1);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) { sh.red[threadIdx.x >> 5] = v0; sh.red2[threadIdx.x >> 5] = v1; }
+  __syncthreads();
+  s0 = 0;
+  s1 = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) { s0 += sh.red[w]; s1 += sh.red2[w]; }
 }
 
 // Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need), found by
@@ -110,12 +124,12 @@ __device__ __forceinline__ void warp_find_bin256(const uint32_t* hist, uint32_t 
   above = who ? __shfl_sync(0xffffffffu, a, src) : 0u;
 }
 
-// The same for the whole CTA on sh.hist: publishes sh.bin and sh.above.
-__device__ void find_bin256(Sel16Shared& sh, uint32_t need) {
+// The same for the whole CTA on 256 bins in shared memory: publishes sh.bin and sh.above.
+__device__ void find_bin256(Sel16Shared& sh, const uint32_t* hist, uint32_t need) {
   if (threadIdx.x < 32) {
     int bin;
     uint32_t above;
-    warp_find_bin256(sh.hist, need, threadIdx.x, bin, above);
+    warp_find_bin256(hist, need, threadIdx.x, bin, above);
     if (threadIdx.x == 0) { sh.bin = bin; sh.above = above; }
   }
   __syncthreads();
@@ -556,39 +570,37 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
         if (v8 < words * 4) bitbytes[v8] = (uint8_t)bits;
       }
     }
-    const uint32_t A = block_sum(sh, above_cnt);
+    // the two histograms of the listed keys (high byte in [0, 256), low byte in [256, 512)) start from
+    // zero; the barriers of the sums also publish them, the bit row and the spill list
+    for (int b = tid; b < 512; b += kThreads) sh.hist[b] = 0;
+    uint32_t A, C;
+    block_sum2(sh, above_cnt, (uint32_t)cnt, A, C);
     const uint32_t novf = sh.novf;
-    const uint32_t C = block_sum(sh, (uint32_t)cnt) + novf;
+    C += novf;
     bool settled = novf <= (uint32_t)kOvfCap && A <= (uint32_t)k && A + C >= (uint32_t)k;
     if (settled && A < (uint32_t)k) {
       // the k - A largest of the listed keys: two-level histogram over the lists
       const uint32_t need = (uint32_t)k - A;
-      for (int b = tid; b < 256; b += kThreads) sh.hist[b] = 0;
-      __syncthreads();
       for (int i = 0; i < cnt; ++i) atomicAdd(&sh.hist[code_of(cand[i * kThreads + tid] >> 16) >> 8], 1u);
       for (int i = tid; i < (int)novf; i += kThreads) atomicAdd(&sh.hist[code_of(sh.ovf_key[i]) >> 8], 1u);
       __syncthreads();
-      find_bin256(sh, need);
+      find_bin256(sh, sh.hist, need);
       const uint32_t b_top = (uint32_t)sh.bin;
       uint32_t up = sh.above;
-      __syncthreads();
-      for (int b = tid; b < 256; b += kThreads) sh.hist[b] = 0;
-      __syncthreads();
       for (int i = 0; i < cnt; ++i) {
         const uint32_t c = code_of(cand[i * kThreads + tid] >> 16);
-        if ((c >> 8) == b_top) atomicAdd(&sh.hist[c & 255u], 1u);
+        if ((c >> 8) == b_top) atomicAdd(&sh.hist[256u + (c & 255u)], 1u);
       }
       for (int i = tid; i < (int)novf; i += kThreads) {
         const uint32_t c = code_of(sh.ovf_key[i]);
-        if ((c >> 8) == b_top) atomicAdd(&sh.hist[c & 255u], 1u);
+        if ((c >> 8) == b_top) atomicAdd(&sh.hist[256u + (c & 255u)], 1u);
       }
       __syncthreads();
-      find_bin256(sh, need - up);
+      find_bin256(sh, sh.hist + 256, need - up);
       T = (b_top << 8) | (uint32_t)sh.bin;
       up += sh.above;
-      eq = sh.hist[sh.bin];
+      eq = sh.hist[256 + sh.bin];
       const uint32_t ties = need - up;              // 1 <= ties <= eq
-      __syncthreads();
       if (ties < eq && eq > (uint32_t)kTieCap) {
         settled = false;                            // too many equal 16-bit keys for the list: exact route
       } else {
@@ -753,7 +765,7 @@ topk16_rows_kernel(const uint16_t* __restrict__ keys16, const __nv_bfloat16* __r
       }
     }
     __syncthreads();
-    find_bin256(sh, ties - acc);
+    find_bin256(sh, sh.hist, ties - acc);
     acc += sh.above;
     prefix |= (uint32_t)sh.bin << shift;
     known |= 255u << shift;
