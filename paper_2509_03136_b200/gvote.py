@@ -224,9 +224,9 @@ def gvote_recompress(p, mu, var, h_last, W_q, b_q, K, V, cu_seqlens, kv_len, seq
     _dev(h_last, torch.float32 if p.h_dtype == DTYPE_F32 else torch.bfloat16, "h_last")
     _dev(W_q, torch.bfloat16, "W_q", dense=False); _dev(K, torch.bfloat16, "K", dense=False); _dev(V, torch.bfloat16, "V", dense=False)
     _dev(mask, torch.int32, "mask"); _dev(budget, torch.int32, "budget"); _dev(b_step, torch.int32, "b_step")
-    _dev(kv_len, torch.int32, "kv_len"); _dev(seq_len, torch.int32, "seq_len")
-    if token_pos is not None:
-        _dev(token_pos, torch.int32, "token_pos")
+    for t, name in ((kv_len, "kv_len"), (seq_len, "seq_len"), (token_pos, "token_pos")):
+        if t is not None:                      # a missing kv_len or seq_len is the library's to refuse
+            _dev(t, torch.int32, name)
     if K.stride() != V.stride():
         raise ValueError("K and V must share strides")
     _check(load().gvote_recompress(ctypes.byref(p), _ptr(mu), _ptr(var), _ptr(h_last), _ptr(W_q), W_q.stride(0),

@@ -660,6 +660,45 @@ def test_recompress_head_without_rows(gv):
     _check_recompress(gv, cfg, synth.make_layer(cfg, 0), empty_head=(1, 0), n_new=3)
 
 
+def test_entry_points_refuse_bad_arguments_before_any_launch(gv):
+    """Host-side validation: a missing or misaligned pointer, a workspace that is too small, a shape the
+    kernels do not take: an error code comes back and nothing has been enqueued."""
+    cfg = _small_cfgs()[2]
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mu = torch.zeros(cfg.batch, cfg.d_h, device="cuda"); var = torch.ones_like(mu)
+    h_last = torch.zeros(cfg.batch, cfg.d_h, device="cuda")
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    kv_len = torch.zeros(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    seen = torch.ones(cfg.batch, dtype=torch.int32, device="cuda")
+    launches = gv.load().gvote_launch_count()
+
+    def status_of(fn):
+        with pytest.raises(gv.GVoteError) as e:
+            fn()
+        return e.value.status
+
+    # a pointer the re-application needs is missing
+    assert status_of(lambda: gv.gvote_recompress(p, mu, var, h_last, d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], None,
+                                                 seen, None, geom, mask, budget, b_step, ws)) == -1
+    # a workspace one byte short
+    assert status_of(lambda: gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask,
+                                               budget, b_step, ws[:-1])) == -3
+    # a misaligned output
+    odd = torch.empty(cfg.batch * cfg.n_kv_heads + 1, dtype=torch.int32, device="cuda")[1:].view(cfg.batch, cfg.n_kv_heads)
+    assert status_of(lambda: gv.gvote_recompress(p, mu, var, h_last, d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], kv_len,
+                                                 seen, None, geom, mask, odd, b_step, ws)) == -2
+    # the longest request must leave two rows for the fit after the sinks
+    short = (cfg.batch, cfg.total_tokens, cfg.n_s + 1)
+    assert status_of(lambda: gv.gvote_fit(p, d["h"], d["cu"], short, mu, var, ws)) == -1
+    assert gv.load().gvote_launch_count() == launches
+
+
 def test_recompress_of_a_full_cache_is_the_plain_pass(gv):
     """kv_len = N for every head and seq_len = N: the same bits as gvote_compress_moments."""
     cfg = synth.make_config("c1")
