@@ -154,8 +154,10 @@ int project_umma_splits(const gvote_params* p, int rows_total) {
   const int m_tiles = (int)ceil_div(F, kFeatTile);
   const int kchunks = (int)ceil_div(p->d_h, 64);
   const int rchunks = (int)ceil_div(rows_total, 240);
-  // about two CTAs per SM on a 148-SM part, every CTA with at least four 64-column steps
-  int splits = (int)ceil_div(296, (int64_t)m_tiles * rchunks);
+  // at most one CTA per SM of a 148-SM part (its ring is 100 KB, so the rest of the SM stays free for
+  // the kernels of other layers on other streams: fewer, longer CTAs take a little longer alone and
+  // less out of an overlapped pass), every CTA with at least four 64-column steps
+  int splits = (int)(148 / ((int64_t)m_tiles * rchunks));
   if (splits > kchunks / 4) splits = kchunks / 4;
   if (splits < 1) splits = 1;
   if (splits > 16) splits = 16;
@@ -189,7 +191,7 @@ int32_t launch_project_umma(const gvote_params* p, const __nv_bfloat16* X, const
     if (!encode_tensor_map_bf16(&tmX, X, 2, dims, strides, box)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   }
   const size_t stage_bytes = (size_t)kFeatTile * 128 + (size_t)NC * 128;
-  int stages = (int)((100 * 1024) / stage_bytes);        // two CTAs per SM when the rows are few
+  int stages = (int)((100 * 1024) / stage_bytes);
   if (stages > 8) stages = 8;
   if (stages < 3) stages = 3;
   if (stages > per) stages = per < 2 ? 2 : per;
