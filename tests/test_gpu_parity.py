@@ -641,12 +641,13 @@ def _check_recompress(gv, cfg, li, sel_mode="topk", n_new=5, empty_head=None, se
             assert np.array_equal(pos_g[h, a:a + keep.shape[0]], kept[r][h][keep])
 
 
-@pytest.mark.parametrize("idx", [2, 3])
-def test_recompress_small(gv, idx):
+@pytest.mark.parametrize("idx,mode", [(1, "topk"), (2, "topk"), (2, "topp"), (3, "topk")])
+def test_recompress_small(gv, idx, mode):
     """The pass on a pruned, grown cache (heads of different lengths, positions from the tokens seen)
-    against the oracle's per-head restatement; same bands as the whole-pass checks."""
+    against the oracle's per-head restatement; same bands as the whole-pass checks.  Case 1 has
+    d_k = 16 and so runs the kernels that stand in where the tensor-core ones do not apply."""
     cfg = _small_cfgs()[idx]
-    _check_recompress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx == 3)))
+    _check_recompress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx == 3)), mode)
 
 
 @pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk")])
