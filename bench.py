@@ -430,7 +430,7 @@ def main():
         up_ms = shard.max_over_ranks(up_ms, dist, dev) / args.steps
         upstream = {"value": shard.job_throughput(cfg.total_tokens, world, up_ms * 1e-3), "unit": UNIT,
                     "ms_per_step": up_ms,
-                    "note": "extra row: gvote_compress_moments, i.e. Algorithm 1 from line 5 on, with mu and var "
+                    "note": "extra row: gvote_compress_moments, i.e. Algorithm 1 from the sampling step on, with mu and var "
                             "fitted beforehand (the engine accumulates them during prefill); not the headline"}
 
     # ---- extra row (labelled, not the headline): the pass applied again to the cache it has just pruned,

@@ -8,7 +8,7 @@
  * averaged over n_f future positions (Step 3), score them against all cached keys, let each
  * synthetic query pick its keys (top-k with k = |C0|, where C0 is the top-p set of the
  * current query, Step 1), OR the picks into one keep-mask per KV head (Step 4) and prune K
- * and V to that set (Algorithm 1, line 11).
+ * and V to that set (the pruning step of Algorithm 1).
  *
  * Conventions, valid for every entry point unless it says otherwise
  *  - Every pointer named below is a DEVICE pointer unless its comment says "host".
@@ -77,9 +77,9 @@ typedef struct {
   float   p_nuc;        /* nucleus mass threshold in (0,1] (Section 3.5: 0.95 advised) */
   int32_t n_f;          /* future positions whose cos/sin are averaged (Step 3) */
   int32_t n_s;          /* leading sink tokens the fit ignores (Step 2) */
-  int32_t sel_mode;     /* GVOTE_SEL_TOPK_C0: Algorithm 1 line 9.  GVOTE_SEL_TOPP: the top-p rule
+  int32_t sel_mode;     /* GVOTE_SEL_TOPK_C0: the TopK step of Algorithm 1.  GVOTE_SEL_TOPP: the top-p rule
                            of Section 3.1 applied to every synthetic query instead. */
-  int32_t include_c0;   /* non-zero: the current query's set C0 joins the union (line 10 unions
+  int32_t include_c0;   /* non-zero: the current query's set C0 joins the union (Algorithm 1 unions
                            the synthetic sets only; default 0) */
   uint64_t seed;        /* Philox key */
   uint32_t layer_id;    /* Philox counter word: gives every layer its own stream */
@@ -99,7 +99,7 @@ static inline int64_t gvote_mask_word_offset(int64_t cu_seqlens_r, int32_t r) {
  * allocation (the library keeps it consistent afterwards).  Returns 0 on invalid params. */
 GVOTE_API size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
-/* Step 2 / Algorithm 1 line 4.  mu[r][c], var[r][c] = mean and unbiased variance over rows
+/* Step 2 of Section 3.2 (the Gaussian fit of Algorithm 1).  mu[r][c], var[r][c] = mean and unbiased variance over rows
  * cu_seqlens[r]+n_s .. cu_seqlens[r+1]-1 of h [total_tokens, d_h] (row stride h_row_stride
  * elements).  Every request needs N_r - n_s >= 2 (the result is NaN otherwise; the host cannot
  * check device-resident lengths, it checks max_N only).  mu, var: [batch, d_h] float. */
@@ -146,7 +146,7 @@ GVOTE_API int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_t
                          const int32_t* cu_seqlens, int32_t batch, int64_t max_N,
                          float* mu, float* var, void* stream);
 
-/* Step 3 / Algorithm 1 line 5.  H_tilde[r][s][c] = mu[r][c] + sqrt(var[r][c]) * z, z a standard
+/* Step 3 of Section 3.2 (the sampling step of Algorithm 1).  H_tilde[r][s][c] = mu[r][c] + sqrt(var[r][c]) * z, z a standard
  * normal drawn by Box-Muller from Philox4x32-10 with key = (seed low, seed high) and counter
  * = (c div 4, s, layer_id, r); word pairs (0,1) and (2,3) of a block give channels 4b..4b+3;
  * u = ((x >> 9) + 0.5) * 2^-23.  H_tilde: [batch, S, d_h] float.  raw_u32_or_null, when given,
@@ -154,7 +154,7 @@ GVOTE_API int32_t gvote_fit_static(const gvote_params* p, const void* h, int64_t
 GVOTE_API int32_t gvote_sample(const gvote_params* p, const float* mu, const float* var, int32_t batch,
                      float* H_tilde, uint32_t* raw_u32_or_null, void* stream);
 
-/* Algorithm 1 lines 1 (Q0), 6 and 7.  X = [h_last[r]; H_tilde[r]] is rounded to bf16, multiplied
+/* Algorithm 1: the current query Q0, AverageCosSin and the synthetic queries.  X = [h_last[r]; H_tilde[r]] is rounded to bf16, multiplied
  * by W_q (fp32 accumulation), b_q added when given ([n_q_heads*d_k] float), then rotated: row 0
  * exactly at position N_r-1, rows 1..S with the mean cos/sin of positions N_r..N_r+n_f-1.
  * Q: [batch, n_kv_heads, G*(S+1), d_k] bf16 with G = n_q_heads / n_kv_heads; the rows of a KV head
@@ -165,7 +165,7 @@ GVOTE_API int32_t gvote_project(const gvote_params* p, const float* H_tilde, con
                       const int32_t* cu_seqlens, int32_t batch,
                       void* Q, void* ws, size_t ws_bytes, void* stream);
 
-/* Algorithm 1 lines 1-3 and 8-10, given the rotated queries (layout as written by gvote_project).
+/* Algorithm 1, the current-query steps (A0, C0, B_step) and the vote (logits, TopK, union), given the rotated queries (layout as written by gvote_project).
  * Per query head g: logits of its
  * S+1 rows against the N_r keys of KV head g div G, scaled by 1/sqrt(d_k); row 0 -> softmax ->
  * top-p -> b_step[r][g] = |C0|; rows 1..S -> top-k(b_step) on logits (or top-p on their softmax
@@ -179,7 +179,7 @@ GVOTE_API int32_t gvote_vote(const gvote_params* p, const void* Q,
                    uint32_t* mask, int32_t* budget, int32_t* b_step,
                    float* dbg_probs_or_null, void* ws, size_t ws_bytes, void* stream);
 
-/* gvote_project followed by gvote_vote (Algorithm 1 lines 1-3 and 6-10); Q lives in ws. */
+/* gvote_project followed by gvote_vote (Algorithm 1 without the fit, the sampling and the pruning); Q lives in ws. */
 GVOTE_API int32_t gvote_select(const gvote_params* p, const float* H_tilde, const void* h_last,
                      const void* W_q, int64_t wq_ld, const float* b_q_or_null,
                      const void* K, int64_t k_tok_stride, int64_t k_head_stride,
@@ -187,7 +187,7 @@ GVOTE_API int32_t gvote_select(const gvote_params* p, const float* H_tilde, cons
                      uint32_t* mask, int32_t* budget, int32_t* b_step,
                      float* dbg_probs_or_null, void* ws, size_t ws_bytes, void* stream);
 
-/* Algorithm 1 line 11.  In place: for every request r and KV head h the kept rows of K and V
+/* Algorithm 1, the pruning step.  In place: for every request r and KV head h the kept rows of K and V
  * move, in ascending key order, to rows cu_seqlens[r] .. cu_seqlens[r]+budget[r][h]-1 of the
  * head's slab; rows behind them are left as they are.  budget [batch, n_kv_heads] is written
  * (popcount of the mask).  Rows are d_k bf16 values, moved in 16-byte pieces. */
@@ -231,7 +231,7 @@ GVOTE_API int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h
                        uint32_t* mask, int32_t* budget, int32_t* b_step,
                        void* ws, size_t ws_bytes, void* stream);
 
-/* Algorithm 1 from line 5 on, for a caller that already has the Gaussian (gvote_fit_finish): sample,
+/* Algorithm 1 from the sampling step on, for a caller that already has the Gaussian (gvote_fit_finish): sample,
  * project, vote, compact.  mu, var [batch, d_h] float; h_last [batch, d_h] of p->h_dtype is the current
  * query's hidden state.  Other arguments and outputs as in gvote_compress. */
 GVOTE_API int32_t gvote_compress_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
@@ -246,10 +246,10 @@ GVOTE_API int32_t gvote_compress_moments(const gvote_params* p, const float* mu,
  * no longer is a position, so the N of Algorithm 1 splits in two:
  *  - kv_len [batch, n_kv_heads] int32 (device): rows KV head h of request r holds (kept earlier plus
  *    appended since), at the front of its slab cu_seqlens[r] .. ; rows beyond are ignored.  Every query
- *    head votes over the rows of its own KV head only (lines 1-3, 8-10); kv_len may be 0 (budget 0).
+ *    head votes over the rows of its own KV head only (current-query steps and vote); kv_len may be 0 (budget 0).
  *  - seq_len [batch] int32 (device): tokens the request has seen.  The current query is rotated at
  *    position seq_len - 1, the synthetic queries with the mean over positions seq_len .. seq_len+n_f-1
- *    (lines 1 and 6); keys stay rotated where they were written.
+ *    (the current query and AverageCosSin); keys stay rotated where they were written.
  *  - cu_seqlens / total_tokens / max_N describe the slabs (capacity), as in gvote_compress.
  *  - token_pos_or_null [n_kv_heads, total_tokens] int32 (device, in/out): the original position of every
  *    slot; its kept entries move to the front of the slab with the rows (entries beyond the new budget

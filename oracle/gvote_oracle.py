@@ -13,7 +13,7 @@ places where the GPU data path rounds to bf16 (the projection's input rows and t
 queries) are mirrored as explicit rounding steps when `mirror_rounding=True`.
 
 Readings of the paper where it is silent (each is a parameter or stated where used):
-  * selection for synthetic queries: top-k with k = |C0| (Algorithm 1, line 9; Section 3.1
+  * selection for synthetic queries: top-k with k = |C0| (Algorithm 1, TopK step; Section 3.1
     last paragraph) is the default `sel_mode="topk"`; `sel_mode="topp"` applies the
     Section 3.1 top-p rule to every synthetic row instead;
   * Q0 is the query of the last cached token; one A0 row and one k per query head;
@@ -122,7 +122,7 @@ def box_muller(raw: np.ndarray) -> np.ndarray:
 
 # ----------------------------------------------------------------------------- Step 2: fit
 def fit(h: np.ndarray, n_s: int) -> Tuple[np.ndarray, np.ndarray]:
-    """Step 2 / Algorithm 1 line 4: per-channel mean and (unbiased) variance of the
+    """Step 2 of Section 3.2 (the Gaussian fit of Algorithm 1): per-channel mean and (unbiased) variance of the
     hidden states along the sequence axis, ignoring the first n_s (sink) tokens."""
     x = np.asarray(h, dtype=np.float64)[n_s:]
     T = x.shape[0]
@@ -178,7 +178,7 @@ def fit_finish(s: FitState) -> Tuple[np.ndarray, np.ndarray]:
 # ----------------------------------------------------------------------------- Step 3: sample
 def sample(mu: np.ndarray, var: np.ndarray, S: int, seed: int, layer_id: int,
            request_id: int) -> Tuple[np.ndarray, np.ndarray]:
-    """Step 3 / Algorithm 1 line 5: H~ in R^{S x d_h} drawn from N(mu, diag var).
+    """Step 3 of Section 3.2 (the sampling step of Algorithm 1): H~ in R^{S x d_h} drawn from N(mu, diag var).
     Returns (H~, raw u32 words)."""
     d_h = mu.shape[0]
     raw = gvote_philox_raw(S, d_h, seed, layer_id, request_id)
@@ -193,7 +193,7 @@ def rope_frequencies(d_k: int, theta: float) -> np.ndarray:
 
 
 def average_cos_sin(N: int, n_f: int, d_k: int, theta: float) -> Tuple[np.ndarray, np.ndarray]:
-    """Algorithm 1 line 6: mean of cos and of sin over the n_f future positions
+    """AverageCosSin of Algorithm 1: mean of cos and of sin over the n_f future positions
     N, N+1, ..., N+n_f-1, per RoPE frequency.  Direct summation."""
     w = rope_frequencies(d_k, theta)
     cbar = np.zeros_like(w)
@@ -220,7 +220,7 @@ def softmax_rows(L: np.ndarray) -> np.ndarray:
 
 
 def top_p_set(a: np.ndarray, p: float) -> np.ndarray:
-    """TopP (Algorithm 1 line 2; Section 3.1): the minimal set of keys whose weights reach
+    """TopP (the set C0 of Algorithm 1; Section 3.1): the minimal set of keys whose weights reach
     cumulative mass p.  Keys are taken by (weight desc, index asc); the key that crosses
     p is kept.  Returns the selected indices in that order."""
     order = np.argsort(-a, kind="stable")
@@ -231,7 +231,7 @@ def top_p_set(a: np.ndarray, p: float) -> np.ndarray:
 
 
 def top_k_set(l: np.ndarray, k: int) -> np.ndarray:
-    """TopK on logits (Algorithm 1 line 9); ties go to the lower index; k clamps to N."""
+    """TopK on logits (the TopK step of Algorithm 1); ties go to the lower index; k clamps to N."""
     k = max(0, min(int(k), l.shape[0]))
     return np.argsort(-l, kind="stable")[:k]
 
@@ -263,7 +263,7 @@ class RequestResult:
 def queries_for_request(H_tilde: np.ndarray, h_last: np.ndarray, W_q: np.ndarray,
                         b_q: Optional[np.ndarray], N: int, *, n_q_heads: int, d_k: int,
                         theta: float, n_f: int, mirror_rounding: bool = True) -> np.ndarray:
-    """Algorithm 1 lines 1 (Q0) and 6-7 (Q~): project [h_last; H~] through W_q; rotate row 0
+    """Algorithm 1, the current query Q0 and the synthetic queries Q~ (AverageCosSin, RoPE): project [h_last; H~] through W_q; rotate row 0
     exactly at position N-1 and rows 1..S with the averaged cos/sin of positions N..N+n_f-1.
     Returns [H_q, S+1, d_k]."""
     X = np.concatenate([np.asarray(h_last, dtype=np.float64)[None, :], H_tilde], axis=0)
@@ -283,7 +283,8 @@ def queries_for_request(H_tilde: np.ndarray, h_last: np.ndarray, W_q: np.ndarray
 
 def vote(Q: np.ndarray, K: np.ndarray, *, p_nuc: float, sel_mode: str = "topk",
          include_c0: bool = False, keep_rows: bool = False, keep_probs: bool = False):
-    """Algorithm 1 lines 1-3 and 8-10 for one request.
+    """Algorithm 1 for one request, from the queries on: the current-query steps (A0, C0, B_step) and the
+    vote (logits, TopK, union).
 
     Q [H_q, S+1, d_k] (row 0 of each head is the real query), K [H_kv, N, d_k].
     Returns (mask [H_kv, N] bool, budget [H_kv], b_step [H_q], row_sets, probs)."""
@@ -296,23 +297,23 @@ def vote(Q: np.ndarray, K: np.ndarray, *, p_nuc: float, sel_mode: str = "topk",
     probs = np.zeros((H_q, R1, N)) if keep_probs else None
     for g in range(H_q):
         kh = g // G
-        L = (Q[g] @ K[kh].T) / math.sqrt(d_k)            # line 8 (and the logits of line 1)
+        L = (Q[g] @ K[kh].T) / math.sqrt(d_k)            # the logits (synthetic rows and A0's row)
         A = softmax_rows(L)
         if keep_probs:
             probs[g] = A
-        C0 = top_p_set(A[0], p_nuc)                      # line 2
-        k = int(C0.shape[0])                             # line 3
+        C0 = top_p_set(A[0], p_nuc)                      # C0 = TopP(A0, p)
+        k = int(C0.shape[0])                             # B_step = |C0|
         b_step[g] = k
         sets = [C0]
         for s in range(1, R1):
             if sel_mode == "topk":
-                Cs = top_k_set(L[s], k)                  # line 9
+                Cs = top_k_set(L[s], k)                  # TopK step
             elif sel_mode == "topp":
                 Cs = top_p_set(A[s], p_nuc)              # Section 3.1 rule per synthetic query
             else:
                 raise ValueError(sel_mode)
             sets.append(Cs)
-            mask[kh, Cs] = True                          # line 10
+            mask[kh, Cs] = True                          # union
         if include_c0:
             mask[kh, C0] = True
         if keep_rows:
@@ -336,7 +337,7 @@ def attention_overlap(Q: np.ndarray, K: np.ndarray, mask: np.ndarray) -> np.ndar
 
 
 def compact(K: np.ndarray, V: np.ndarray, mask: np.ndarray):
-    """Algorithm 1 line 11: keep the rows of the keep-set, in ascending index order.
+    """Algorithm 1, the pruning step: keep the rows of the keep-set, in ascending index order.
     K, V [H_kv, N, d_k] (any dtype; moved, not computed on); returns lists per head."""
     Kc, Vc = [], []
     for kh in range(K.shape[0]):
@@ -375,18 +376,18 @@ def compress_request(h: np.ndarray, W_q: np.ndarray, b_q: Optional[np.ndarray], 
                      sel_mode: str = "topk", include_c0: bool = False,
                      mirror_rounding: bool = True, h_last: Optional[np.ndarray] = None,
                      keep_rows: bool = False, keep_probs: bool = False) -> RequestResult:
-    """Algorithm 1 for one request and one layer, lines 1-10 (pruning is `compact`).
+    """Algorithm 1 for one request and one layer, up to the union (pruning is `compact`).
 
     h [N, d_h] fp64 hidden states; W_q, K already widened to fp64 (exact bf16 values)."""
     N = K.shape[1]
-    mu, var = fit(h, n_s)                                               # line 4
-    H_tilde, _ = sample(mu, var, S, seed, layer_id, request_id)         # line 5
+    mu, var = fit(h, n_s)                                               # fit
+    H_tilde, _ = sample(mu, var, S, seed, layer_id, request_id)         # sample
     hl = h[-1] if h_last is None else h_last
     Q = queries_for_request(H_tilde, hl, W_q, b_q, N, n_q_heads=n_q_heads, d_k=d_k,
-                            theta=theta, n_f=n_f, mirror_rounding=mirror_rounding)  # 1, 6-7
+                            theta=theta, n_f=n_f, mirror_rounding=mirror_rounding)  # Q0, Q~
     mask, budget, b_step, rows, probs = vote(Q, K, p_nuc=p_nuc, sel_mode=sel_mode,
                                              include_c0=include_c0, keep_rows=keep_rows,
-                                             keep_probs=keep_probs)     # 1-3, 8-10
+                                             keep_probs=keep_probs)     # A0, C0, vote
     return RequestResult(mu=mu, var=var, H_tilde=H_tilde, Q=Q, b_step=b_step, mask=mask,
                          budget=budget, row_sets=rows, probs=probs)
 
@@ -412,17 +413,17 @@ def recompress_request(mu: np.ndarray, var: np.ndarray, h_last: np.ndarray, W_q:
     KV head kh now holds K_heads[kh] [len_kh, d_k]: the rows that survived plus the rows appended
     since, each still rotated at the position it was written at, so head lengths differ and a
     slot number no longer is a position.  What Algorithm 1 calls N splits in two: the keys a
-    query head sees are the len_kh rows of its own KV head (lines 1-3 and 8-10 run per head on
-    those), while the positions of lines 1 and 6 come from seq_len, the number of tokens the
+    query head sees are the len_kh rows of its own KV head (the current-query steps and the vote run
+    per head on those), while the positions of the current query and of AverageCosSin come from seq_len, the number of tokens the
     request has seen: the current query sits at seq_len - 1 and the synthetic queries average
-    positions seq_len .. seq_len + n_f - 1.  mu and var are the caller's running fit (line 4).
+    positions seq_len .. seq_len + n_f - 1.  mu and var are the caller's running fit.
     token_pos[kh] [len_kh] (optional) maps slots to original positions; the result carries the
     map of the slots that stay."""
     H_kv = len(K_heads)
     G = n_q_heads // H_kv
-    H_tilde, _ = sample(mu, var, S, seed, layer_id, request_id)                      # line 5
+    H_tilde, _ = sample(mu, var, S, seed, layer_id, request_id)                      # sample
     Q = queries_for_request(H_tilde, h_last, W_q, b_q, seq_len, n_q_heads=n_q_heads, d_k=d_k,
-                            theta=theta, n_f=n_f, mirror_rounding=mirror_rounding)   # 1, 6-7
+                            theta=theta, n_f=n_f, mirror_rounding=mirror_rounding)   # Q0, Q~
     masks: List[np.ndarray] = []
     b_step = np.zeros(n_q_heads, dtype=np.int64)
     budget = np.zeros(H_kv, dtype=np.int64)
@@ -432,13 +433,13 @@ def recompress_request(mu: np.ndarray, var: np.ndarray, h_last: np.ndarray, W_q:
             masks.append(np.zeros(0, dtype=bool))
             continue
         m, b, ks, _, _ = vote(Q[kh * G:(kh + 1) * G], Kh[None], p_nuc=p_nuc, sel_mode=sel_mode,
-                              include_c0=include_c0)                                  # 1-3, 8-10
+                              include_c0=include_c0)                                  # A0, C0, vote
         masks.append(m[0])
         budget[kh] = b[0]
         b_step[kh * G:(kh + 1) * G] = ks
     kept_pos = None
     if token_pos is not None:
-        kept_pos = [np.asarray(token_pos[kh])[masks[kh]] for kh in range(H_kv)]      # line 11, on the map
+        kept_pos = [np.asarray(token_pos[kh])[masks[kh]] for kh in range(H_kv)]      # pruning, on the map
     return RecompressResult(b_step=b_step, masks=masks, budget=budget, token_pos=kept_pos, Q=Q)
 
 
@@ -463,7 +464,7 @@ def compress_layer(h: np.ndarray, W_q_bits: np.ndarray, b_q: Optional[np.ndarray
                                sel_mode=sel_mode, include_c0=include_c0,
                                mirror_rounding=mirror_rounding, keep_rows=keep_rows,
                                keep_probs=keep_probs)
-        Kc, Vc = compact(K_bits[:, a:b], V_bits[:, a:b], res.mask)      # line 11
+        Kc, Vc = compact(K_bits[:, a:b], V_bits[:, a:b], res.mask)      # pruning
         results.append(res)
         Kc_all.append(Kc)
         Vc_all.append(Vc)

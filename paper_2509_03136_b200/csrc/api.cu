@@ -228,7 +228,7 @@ int32_t gvote_fit_finish(const gvote_params* p, const double* state, int32_t bat
 }
 
 namespace {
-// The pass from line 5 on, from fitted moments; kv_len / seq_len / token_pos are the extras of the
+// The pass from the sampling step of Algorithm 1 on, from fitted moments; kv_len / seq_len / token_pos are the extras of the
 // re-application (all null for a cache that has not been pruned before).
 int32_t compress_from_moments(const gvote_params* p, const float* mu, const float* var, const void* h_last,
                               const void* W_q, int64_t wq_ld, const float* b_q_or_null, void* K, void* V,

@@ -1,4 +1,4 @@
-// Algorithm 1 line 11: prune K and V to the keep-set, in place.
+// Algorithm 1, the pruning step: prune K and V to the keep-set, in place.
 //
 // Two kernels.  mask_scan_kernel turns each (request, KV head) bit row into an exclusive popcount
 // prefix per 32-key word and the head's budget.  compact_kernel then moves the kept rows of one

@@ -1,4 +1,4 @@
-// Step 2 of the GVote scheme (Algorithm 1, line 4): per-channel mean and unbiased variance of the
+// Step 2 of the GVote scheme (Section 3.2; the Gaussian fit of Algorithm 1): per-channel mean and unbiased variance of the
 // hidden states along the sequence axis, skipping the first n_s sink tokens of every request.
 //
 // The hidden-state matrix is the largest tensor the pass touches (16 KiB per token at d_h = 4096

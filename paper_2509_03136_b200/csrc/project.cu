@@ -1,4 +1,4 @@
-// Algorithm 1 lines 1 (the current query Q0), 6 (AverageCosSin) and 7 (Q~ = RoPE(H~ W_q, P)).
+// Algorithm 1: the current query Q0, AverageCosSin, and the synthetic queries Q~ = RoPE(H~ W_q, P).
 //
 // Per request the S+1 rows X = [h_last; H~] are rounded to bf16, multiplied by the stored weight
 // W_q [n_q_heads*d_k, d_h] with fp32 accumulation, the bias is added, and each head's d_k-vector

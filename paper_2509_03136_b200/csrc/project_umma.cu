@@ -1,4 +1,4 @@
-// Algorithm 1 lines 1 and 7, the matrix product: out[row][f] = sum_c X[row][c] * W_q[f][c] for the
+// Algorithm 1, the projections of the current query and of the synthetic queries: the matrix product out[row][f] = sum_c X[row][c] * W_q[f][c] for the
 // S+1 rows of every request (current query first, then the S synthetic hidden states), on the
 // fifth-generation tensor cores.
 //

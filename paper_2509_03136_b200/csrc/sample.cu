@@ -1,4 +1,4 @@
-// Step 3 of the GVote scheme (Algorithm 1, line 5): S synthetic hidden states per request drawn
+// Step 3 of the GVote scheme (Section 3.2; the sampling step of Algorithm 1): S synthetic hidden states per request drawn
 // from N(mu, diag(var)).  Randomness is counter based (Philox4x32-10, Salmon et al., SC'11) so
 // that any draw can be recomputed from (seed, layer, request, sample, channel) alone: key =
 // (seed low word, seed high word), counter = (channel div 4, sample, layer, request); the four

@@ -1,4 +1,4 @@
-// Algorithm 1 line 8 (and the logits of line 1) on the fifth-generation tensor cores:
+// The logits of Algorithm 1 (synthetic queries, and the current query's row A0) on the fifth-generation tensor cores:
 // L = Q K^T / sqrt(d_k) for all (S+1)*G query rows of a KV head against that head's cached keys.
 //
 // Shape of the contraction.  A KV head's G*S synthetic rows are cut into chunks of 128, and a chunk
@@ -20,7 +20,7 @@
 // half precision (all the top-k search needs to bracket its threshold), staged in shared memory as a
 // [row][128 keys] tile (16-byte chunks XOR-swizzled by the row so the stores do not collide) and
 // written with one bulk copy per tile into keys16[head][tile][chunk][row][128].  Only the rows of the
-// current query are written as fp32, because the softmax mass of line 2 needs them exactly; their
+// current query are written as fp32, because the top-p mass of the set C0 needs them exactly; their
 // running maxima go to `rowmax`.  In the all-fp32 mode (per-sample top-p, softmax dump) the
 // synthetic rows are staged as fp32 instead and written to the logits buffer row by row.
 //
@@ -252,7 +252,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
 
       // ---- current-query rows (chunk 0 only): thread = key, exact fp32 logits and their running
-      // maximum for the softmax of Algorithm 1 line 1
+      // maximum for the softmax row A0 of Algorithm 1
       if (with_real && half == 0) {
         uint32_t w[16];
         ptx::tmem_ld_32x16(tmem_base + (uint32_t)(kD2Col + a * 32) + ((uint32_t)(q * 32) << 16), w);

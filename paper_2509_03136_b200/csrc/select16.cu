@@ -1,6 +1,6 @@
-// Algorithm 1 line 9 for the synthetic queries: the k = |C0| largest logits of a row, found on the
+// Algorithm 1, the TopK step for the synthetic queries: the k = |C0| largest logits of a row, found on the
 // 16-bit keys the tensor-core score kernel leaves behind (each logit rounded to half precision), and
-// OR-ed into the head's keep mask (line 10).
+// OR-ed into the head's keep mask (the union step).
 //
 // One small CTA per synthetic row, many resident per SM.  Keys are compared as half-precision numbers,
 // two per instruction; for counting they are mapped to an order-preserving 16-bit code.

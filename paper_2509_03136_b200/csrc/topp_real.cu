@@ -1,4 +1,4 @@
-// Algorithm 1 lines 1-3 for the current query of every head: softmax of its logits over all cached
+// Algorithm 1, the current-query steps (A0, C0, B_step), for every head: softmax of its logits over all cached
 // keys, the smallest set C0 of keys whose weights reach the mass p, and its size B_step = |C0|.
 //
 // There are only n_q_heads such rows per request but each is N long, so a row is shared by a thread-

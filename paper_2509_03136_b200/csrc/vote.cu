@@ -1,4 +1,4 @@
-// Algorithm 1 lines 1-3 and 8-10: attention logits of the current query and of the S synthetic
+// Algorithm 1, the current-query steps and the vote: attention logits of the current query and of the S synthetic
 // queries against all cached keys, the current query's top-p set size |C0| (the step budget),
 // each synthetic query's selection (top-k with k = |C0|, or top-p in the alternative mode), and
 // the union of the selections as one keep bit-mask per KV head.

@@ -322,7 +322,8 @@ def test_vote_union_contains_every_voter_and_counts(mode):
 
 
 def test_vote_by_brute_force_tiny():
-    """All of lines 1-3, 8-10 re-derived with exhaustive subset search on N=10."""
+    """The current-query steps (A0, C0, B_step) and the vote (logits, TopK, union) of Algorithm 1 re-derived
+    with exhaustive subset search on N=10."""
     Q, K = _small_problem(12, H_q=2, H_kv=1, d_k=4, S=3, N=10)
     p = 0.7
     mask, budget, b_step, _, _ = o.vote(Q, K, p_nuc=p)
