@@ -521,7 +521,7 @@ def main():
         same = all(np.array_equal(hbud[l].numpy(), d_budget[l].cpu().numpy()) for l in range(L))
         e2e["budgets_match_device_run"] = bool(same)
 
-    # ---- the oracle on this machine's host cores, on a bounded sample (rank 0, one GPU only)
+    # ---- the oracle on the host cores, on a bounded sample (rank 0, one GPU only)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         t_or, res = time_oracle_layer(cfg, layers[0], 0)
