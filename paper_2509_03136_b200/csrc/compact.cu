@@ -47,10 +47,15 @@ mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ 
     }
   }
   __syncthreads();
-  for (int base = 0; base < words; base += kScanThreads) {
-    const int w = base + tid;
-    const int c = (w < words) ? __popc(m[w]) : 0;
-    int inc = c;
+  // four consecutive words per thread and step (1024 words = 32768 keys per step): the thread scans
+  // its own four, the CTA scans the threads' totals
+  for (int base = 0; base < words; base += 4 * kScanThreads) {
+    const int w0 = base + 4 * tid;
+    int c[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) c[j] = (w0 + j < words) ? __popc(m[w0 + j]) : 0;
+    const int mine = c[0] + c[1] + c[2] + c[3];
+    int inc = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, inc, o);
@@ -60,7 +65,12 @@ mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ 
     __syncthreads();
     int before = carry;
     for (int i = 0; i < warp; ++i) before += warp_tot[i];
-    if (w < words) pf[w] = before + inc - c;
+    int run = before + inc - mine;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (w0 + j < words) pf[w0 + j] = run;
+      run += c[j];
+    }
     __syncthreads();
     if (tid == kScanThreads - 1) carry = before + inc;
     __syncthreads();
