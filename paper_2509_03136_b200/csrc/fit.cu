@@ -24,7 +24,7 @@ namespace {
 
 constexpr int kFitTx = 64;                 // column threads (x4 channels each)
 constexpr int kFitTy = 2;                  // row lanes
-constexpr int kFitRows = 32;               // rows per stage (one lane of the producer warp per row in the tail)
+constexpr int kFitRows = 32;               // rows per stage of fp32 hidden states (bf16: twice as many, the same 32 KB)
 constexpr int kFitConsumers = kFitTx * kFitTy;
 constexpr int kFitThreads = kFitConsumers + 32;    // + the producer warp
 constexpr int kFitMaxStages = 8;
@@ -56,7 +56,7 @@ __device__ __forceinline__ void acc4(float4& s1, float4& s2, const float4& v, co
 }
 __device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
-// tmH describes h as [rows][d_h] with a [kFitRows x 256] box.  Its row extent may be an upper bound:
+// tmH describes h as [rows][d_h] with a [rows per stage x 256] box.  Its row extent may be an upper bound:
 // a stage that would reach past the chunk's last row is fetched row by row instead, so no load
 // touches a row the chunk does not own.
 template <typename T>
@@ -68,7 +68,7 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
   __shared__ uint64_t full[kFitMaxStages], empty[kFitMaxStages];
   __shared__ int abort_flag;
   __shared__ float4 sm1[kFitTy][kFitTx], sm2[kFitTy][kFitTx];
-  constexpr int R = kFitRows;
+  constexpr int R = kFitRows * (4 / (int)sizeof(T));       // 32 KB per stage whatever the element type
   constexpr uint32_t pitch = kFitStripCols * sizeof(T);
   constexpr uint32_t stage_bytes = R * pitch;
   const int r = blockIdx.z, c = blockIdx.y;
@@ -113,7 +113,8 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
         const uint32_t row_bytes = (uint32_t)width * sizeof(T);
         if (lane == 0) ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)rows_here * row_bytes);
         __syncwarp();
-        if (lane < rows_here) ptx::bulk_load(dst + (size_t)lane * pitch, h + (int64_t)(row + lane) * ld + col0, row_bytes, &full[s]);
+        for (int rr = lane; rr < rows_here; rr += 32)
+          ptx::bulk_load(dst + (size_t)rr * pitch, h + (int64_t)(row + rr) * ld + col0, row_bytes, &full[s]);
       }
       issued = it + 1;
     }
@@ -136,11 +137,15 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
       if (active) {
         if (it == 0) sh = lds4<T>(st + tx * 4);     // shift: the chunk's first row (same for all row lanes)
         if (rows_here == R) {
-          float4 v[R / kFitTy];
 #pragma unroll
-          for (int j = 0; j < R / kFitTy; ++j) v[j] = lds4<T>(st + (size_t)(ty + j * kFitTy) * kFitStripCols + tx * 4);
+          for (int sub = 0; sub < R; sub += kFitRows) {      // 16 loads in flight, then 16 updates
+            float4 v[kFitRows / kFitTy];
 #pragma unroll
-          for (int j = 0; j < R / kFitTy; ++j) acc4(s1, s2, v[j], sh);
+            for (int j = 0; j < kFitRows / kFitTy; ++j)
+              v[j] = lds4<T>(st + (size_t)(sub + ty + j * kFitTy) * kFitStripCols + tx * 4);
+#pragma unroll
+            for (int j = 0; j < kFitRows / kFitTy; ++j) acc4(s1, s2, v[j], sh);
+          }
         } else {
           for (int row = ty; row < rows_here; row += kFitTy)
             acc4(s1, s2, lds4<T>(st + (size_t)row * kFitStripCols + tx * 4), sh);
@@ -268,11 +273,11 @@ int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, con
   {
     const uint64_t dims[2] = {(uint64_t)p->d_h, (uint64_t)rows_bound};
     const uint64_t strides[1] = {(uint64_t)ld * elem};
-    const uint32_t box[2] = {(uint32_t)kFitStripCols, (uint32_t)kFitRows};
+    const uint32_t box[2] = {(uint32_t)kFitStripCols, (uint32_t)(kFitRows * (4 / elem))};
     if (!encode_tensor_map_plain(&tmH, h, elem, 2, dims, strides, box)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   }
   // 96 KB of stages per CTA: what keeps one CTA per SM at the HBM rate
-  const size_t stage_bytes = (size_t)kFitRows * kFitStripCols * elem;
+  const size_t stage_bytes = (size_t)kFitRows * (4 / elem) * kFitStripCols * elem;
   int stages = (int)((96 * 1024) / stage_bytes);
   if (stages > kFitMaxStages) stages = kFitMaxStages;
   const size_t smem = stages * stage_bytes;

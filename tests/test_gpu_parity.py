@@ -488,6 +488,30 @@ def test_compress_configs(gv, name, mode):
     _check_compress(gv, cfg, synth.make_layer(cfg, 0), mode)
 
 
+def _run_compress_bf16_h(gv, cfg, li, sel_mode="topk", layer_id=0):
+    p = gv.params_from_config(cfg, layer_id=layer_id, h_dtype=gv.DTYPE_BF16)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_compress(p, d["h"].bfloat16(), d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget, b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
+            gv.bits_from_bf16(d["V"]))
+
+
+@pytest.mark.parametrize("name", ["small2", "c1", "c3"])
+def test_compress_bf16_hidden_states(gv, name):
+    """The whole pass with the hidden states in bf16 (half the bytes of the fit): the oracle gets the same
+    bf16 values widened to fp64."""
+    cfg = _small_cfgs()[2] if name == "small2" else synth.make_config(name)
+    li = synth.make_layer(cfg, 0)
+    li.h = torch.from_numpy(li.h).bfloat16().float().numpy()      # the values bf16 can hold
+    _check_compress(gv, cfg, li, runner=_run_compress_bf16_h)
+
+
 # ----------------------------------------------------------------------------- streaming fit
 def _stream_fit(gv, p, cfg, li, n_blocks, rng):
     """Feed every request's rows after the sinks in n_blocks uneven blocks; returns (mu, var) tensors."""
