@@ -4,7 +4,7 @@
 // The hidden-state matrix is the largest tensor the pass touches (16 KiB per token at d_h = 4096
 // in fp32), so this is a pure HBM stream.  Each CTA owns a strip of 256 channels and a chunk of
 // rows and pulls them through a ring of shared-memory stages: one thread asks the TMA unit for a
-// [32 rows x 256 channels] box per stage (marked evict-first in L2: the data is read once), four
+// [32 rows x 256 channels] box per stage (marked evict-first in L2: the data is read once), eight
 // warps take the stages as they land and keep shifted first and second moments of four channels
 // per thread in registers.  Few threads and registers per SM stay busy that way, which leaves room
 // for the kernels of other layers that run beside the fit on other streams.  One (mean, M2) pair
@@ -23,7 +23,7 @@ namespace gvote {
 namespace {
 
 constexpr int kFitTx = 64;                 // column threads (x4 channels each)
-constexpr int kFitTy = 2;                  // row lanes
+constexpr int kFitTy = 4;                  // row lanes
 constexpr int kFitRows = 32;               // rows per stage of fp32 hidden states (bf16: twice as many, the same 32 KB)
 constexpr int kFitConsumers = kFitTx * kFitTy;
 constexpr int kFitThreads = kFitConsumers + 32;    // + the producer warp
@@ -153,7 +153,7 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&empty[s]);
-      if ((it + 1) % kFitFlushStages == 0) {        // short fp32 runs: the rounding error stays that of 64 terms
+      if ((it + 1) % kFitFlushStages == 0) {        // short fp32 runs: the rounding error stays that of a few dozen terms
         add4(t1, s1); add4(t2, s2);
         s1 = make_float4(0.f, 0.f, 0.f, 0.f); s2 = s1;
       }
