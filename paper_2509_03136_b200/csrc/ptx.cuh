@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the tensor-core kernels use: mbarriers, TMA
-// tiled loads (cp.async.bulk.tensor, no multicast), tensor memory (tcgen05.alloc/ld/dealloc) and
+// tiled loads (cp.async.bulk.tensor, every load into the issuing CTA only), tensor memory (tcgen05.alloc/ld/dealloc) and
 // the fifth-generation MMA (tcgen05.mma) with its shared-memory and instruction descriptors.
 #pragma once
 
