@@ -220,6 +220,70 @@ def test_round_to_bf16_matches_torch():
     assert np.array_equal(o.round_to_bf16(x), ref)
 
 
+def _torch_bf16(x):
+    """bf16 rounding by a routine other than the oracle's (torch's conversion), result in fp64."""
+    import torch
+    return torch.tensor(np.asarray(x), dtype=torch.float64).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_mirrored_roundings_sit_before_the_product_and_after_the_rotation():
+    """Where `mirror_rounding=True` rounds: the projection's input rows X = [h_last; H~] before the
+    product, the rotated queries after RoPE, and nowhere else.  Each claim is checked against a
+    statement that a rounding put elsewhere fails."""
+    rng = np.random.default_rng(21)
+    d_h, H, d_k, S, N, n_f, theta = 40, 3, 8, 5, 77, 6, 1e4
+    Ht, hl = rng.normal(size=(S, d_h)) * 3, rng.normal(size=d_h)
+    W = _torch_bf16(rng.normal(size=(H * d_k, d_h)) / math.sqrt(d_h))
+    b = rng.normal(size=H * d_k) * 0.1
+    kw = dict(n_q_heads=H, d_k=d_k, theta=theta, n_f=n_f)
+    Qm = o.queries_for_request(Ht, hl, W, b, N, mirror_rounding=True, **kw)
+    # (a) the last step is a rounding: every entry lies on the bf16 grid
+    assert np.array_equal(Qm, _torch_bf16(Qm))
+    # (b) exactly one rounding lies between the product of the rounded rows and the result: the error
+    # against the unrounded rotation of those rows is at most half a bf16 step of the result's binade
+    Xr = _torch_bf16(np.concatenate([hl[None], Ht]))
+    Qx = o.queries_for_request(Xr[1:], Xr[0], W, b, N, mirror_rounding=False, **kw)
+    half_step = 2.0 ** (np.floor(np.log2(np.abs(Qx))) - 8)
+    assert np.all(np.abs(Qm - Qx) <= half_step)
+    assert np.array_equal(Qm, _torch_bf16(Qx))
+    # a second rounding between the product and the rotation (the planted mistake) breaks (b) somewhere
+    w = o.rope_frequencies(d_k, theta)
+    q_pre = _torch_bf16(o.project_queries(Xr, W, b, H, d_k))
+    c0, s0 = np.cos((N - 1) * w), np.sin((N - 1) * w)
+    cb, sb = o.average_cos_sin(N, n_f, d_k, theta)
+    wrong = np.empty_like(q_pre)
+    wrong[:, 0] = o.rope_apply(q_pre[:, 0], c0, s0)
+    wrong[:, 1:] = o.rope_apply(q_pre[:, 1:], cb, sb)
+    assert np.any(np.abs(_torch_bf16(wrong) - Qx) > half_step)
+    # (c) against the unrounded pass the two roundings together stay within what two roundings allow:
+    # the input rounding moves a row by at most 2^-9 relative per entry, i.e. the product by at most
+    # 2^-9 * sum |x_c W_fc|, the rotation mixes two features with |cos|, |sin| <= 1, and the final
+    # rounding adds half a step of the result
+    Qi = o.queries_for_request(Ht, hl, W, b, N, mirror_rounding=False, **kw)
+    X = np.concatenate([hl[None], Ht])
+    prod = (np.abs(X) @ np.abs(W).T).reshape(S + 1, H, d_k).transpose(1, 0, 2) * 2.0 ** -9
+    mix = prod + np.concatenate([prod[..., d_k // 2:], prod[..., :d_k // 2]], axis=-1)
+    assert np.all(np.abs(Qm - Qi) <= mix + 2.0 ** -8 * np.abs(Qi) + 1e-12)
+    assert np.any(Qm != _torch_bf16(Qi))                       # and the input rounding is not a no-op
+
+
+def test_input_rows_are_rounded_before_the_product_not_after():
+    """A hand case where the place of the first rounding changes the bits.  One head, no rotation
+    (N = 1 puts the current query at position 0, where RoPE is the identity), a weight row that adds
+    two channels: x = (1 + 2^-8, 2^-8).  Rounded first, 1 + 2^-8 is a tie that goes to the even
+    neighbour 1, the sum is 1 + 2^-8 and the final rounding gives 1 again.  Summed first, the result
+    is 1 + 2^-7, which bf16 holds exactly."""
+    d_k = 2
+    W = np.zeros((d_k, 2))
+    W[0] = [1.0, 1.0]
+    hl = np.array([1.0 + 2.0 ** -8, 2.0 ** -8])
+    Ht = np.zeros((1, 2))
+    Q = o.queries_for_request(Ht, hl, W, None, 1, n_q_heads=1, d_k=d_k, theta=1e4, n_f=1, mirror_rounding=True)
+    assert Q[0, 0, 0] == 1.0
+    Qi = o.queries_for_request(Ht, hl, W, None, 1, n_q_heads=1, d_k=d_k, theta=1e4, n_f=1, mirror_rounding=False)
+    assert Qi[0, 0, 0] == 1.0 + 2.0 ** -7 and _torch_bf16(Qi)[0, 0, 0] == 1.0 + 2.0 ** -7
+
+
 def test_bf16_bits_widen_exactly():
     import torch
     bits = np.arange(0, 65536, 7, dtype=np.uint16)
