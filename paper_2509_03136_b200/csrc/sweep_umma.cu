@@ -1,0 +1,646 @@
+// Algorithm 1, the logits of the synthetic queries and their TopK, fused on the fifth-generation
+// tensor cores so that the S x N logits matrix (the memory hazard Section 4.4 names) never exists:
+// two passes over a KV head's keys, both D[128 rows x 128 keys] = Q_chunk (128 x d_k) * K_tile^T per
+// 128-key tile with the accumulators in tensor memory, a lane per query row, a column per key.
+//
+//   score_sample_kernel  first pass.  Streams every key tile once for the G current-query rows of the
+//       head (a thin second product D2[128 keys x 16] = K_tile * Qr^T on the same tile in shared
+//       memory): their exact fp32 logits and running maxima, the input of the current query's top-p
+//       (A0, C0, B_step).  On the tiles of the row sample (vote_geom.cuh) it also runs the full product
+//       and stores the synthetic rows' logits there as half-precision keys - a few thousand keys per
+//       row, from which bracket_kernel takes two order statistics [lo, hi] that enclose the row's k-th
+//       largest logit.
+//   score_sweep_kernel   second pass.  Every tile, every row chunk.  The read-out thread of a row holds
+//       64 consecutive logits of its row in registers and compares them with the row's own bracket:
+//       keys above hi are certainly among the k largest - their bits are OR-ed over the 32 rows of the
+//       warp and then into the head's tentative mask (the union step), and counted per row; keys
+//       inside [lo, hi] are appended, as (fp32 logit, index), to the row's short candidate list.
+//       Nothing else leaves the SM.  resolve_kernel later picks the k - #above largest candidates.
+//
+// A CTA holds the query rows of up to four 128-row chunks in shared memory and walks the key tiles
+// x, x+X, ... of one (request, KV head): a tile is fetched once (TMA, 128-byte swizzle) and multiplied
+// with every chunk.  warp 0: TMA producer; warp 1: tensor-memory allocation and tcgen05.mma issue;
+// warps 2-9: read-out, two warps per lane quadrant, each 64 of the tile's 128 keys.  Accumulators are
+// double buffered so that the MMAs of one product overlap the read-out of the one before.
+//
+// Every wait on an mbarrier is bounded.  When one runs out the CTA raises a shared abort flag and
+// records GVOTE_ERR_TIMEOUT in the workspace status word; the remaining waits then give up at once,
+// the warps run their loops to the end (all addresses stay in bounds whatever the data), bulk copies
+// are drained, tensor memory is freed and the CTA returns.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "vote_geom.cuh"
+
+namespace gvote {
+namespace {
+
+constexpr int kTileKeys = kVoteTileKeys;
+constexpr int kRowChunk = kVoteRowChunk;
+constexpr int kRealCols = 16;     // current-query rows per KV head the thin product holds (MMA N)
+constexpr int kEpiWarps = 8;
+constexpr int kSweepThreads = 64 + 32 * kEpiWarps;
+constexpr int kMaxStages = 6;
+constexpr int kTmemCols = 512;    // 2 x 128 (D1) + 2 x 32 (D2, 16 used)
+constexpr int kD2Col = 256;
+
+struct SweepTail {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t q_full;
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t real_full[2];
+  uint64_t real_empty[2];
+  uint32_t tmem_slot;
+  volatile int abort_flag;
+  uint32_t rowmax[kRealCols];         // running maximum (order-preserving image) of each current-query row
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ uint32_t key16x2_of(float lo, float hi) {
+  uint32_t p;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(p) : "f"(hi), "f"(lo));
+  return p;
+}
+
+// The key tiles a CTA walks: every tile x, x+X, ..., or only those of the row sample.
+struct TileWalk {
+  SampleGeom g;
+  int x, X, count;
+  bool sampled_only;
+  __device__ __forceinline__ void init(int N, int x_, int X_, bool sampled_only_) {
+    g = sample_geom(N);
+    x = x_; X = X_; sampled_only = sampled_only_;
+    const int n = sampled_only ? g.ns : g.n_tiles;
+    count = (N > 0 && x < n) ? (n - x + X - 1) / X : 0;
+  }
+  __device__ __forceinline__ int tile(int i) const {
+    const int j = x + i * X;
+    return sampled_only ? sample_tile(g, j) : j;
+  }
+  // position of tile(i) in the sample, or -1
+  __device__ __forceinline__ int slot(int i) const {
+    return sampled_only ? x + i * X : sample_slot_of_tile(g, x + i * X);
+  }
+};
+
+struct SweepSmem {
+  uint8_t* Qs;      // [chunks][kchunks][128 rows][128 bytes]
+  uint8_t* Qr;      // [kchunks][16 rows][128 bytes]
+  uint8_t* Ks;      // [stages][kchunks][128 keys][128 bytes]
+  uint8_t* Os;      // staging of half-precision key tiles (first pass)
+  SweepTail* tail;
+};
+
+__device__ __forceinline__ SweepSmem carve(uint8_t* smem_raw, int kchunks, int cg, int stages, bool with_real,
+                                           int n_out) {
+  SweepSmem s;
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t q_bytes = (uint32_t)cg * kchunks * kRowChunk * 128;
+  const uint32_t qr_bytes = with_real ? (((uint32_t)kchunks * kRealCols * 128 + 1023u) & ~1023u) : 0u;
+  const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
+  s.Qs = base;
+  s.Qr = s.Qs + q_bytes;
+  s.Ks = s.Qr + qr_bytes;
+  s.Os = s.Ks + (size_t)stages * stage_bytes;
+  s.tail = reinterpret_cast<SweepTail*>(s.Os + (size_t)n_out * kRowChunk * kTileKeys * 2);
+  return s;
+}
+
+__device__ __forceinline__ void setup(SweepTail* tail, int stages, const CUtensorMap* a, const CUtensorMap* b,
+                                      const CUtensorMap* c) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
+    ptx::mbar_init(&tail->q_full, 1);
+    for (int a2 = 0; a2 < 2; ++a2) {
+      ptx::mbar_init(&tail->acc_full[a2], 1);
+      ptx::mbar_init(&tail->acc_empty[a2], kEpiWarps);
+      ptx::mbar_init(&tail->real_full[a2], 1);
+      ptx::mbar_init(&tail->real_empty[a2], kEpiWarps / 2);
+    }
+    tail->abort_flag = 0;
+    for (int i = 0; i < kRealCols; ++i) tail->rowmax[i] = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(a);
+    ptx::prefetch_tensormap(b);
+    if (c) ptx::prefetch_tensormap(c);
+  }
+  if ((threadIdx.x >> 5) == 1) {
+    ptx::tmem_alloc(&tail->tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+}
+
+// One 128 x 128 x d_k product into accumulator `d`: rows = the query chunk at q_addr, columns = the keys at k_addr.
+__device__ __forceinline__ void issue_d1(uint32_t d, uint32_t q_addr, uint32_t k_addr, int d_k) {
+  const uint32_t idesc = ptx::instr_desc_bf16_f32(kRowChunk, kTileKeys);
+  const int ksteps = d_k / 16;
+  for (int k = 0; k < ksteps; ++k) {
+    const uint32_t koff = (uint32_t)(k >> 2), kin = (uint32_t)(k & 3) * 32u;
+    const uint64_t dq = ptx::smem_desc_k_sw128(q_addr + koff * (uint32_t)(kRowChunk * 128) + kin);
+    const uint64_t dk = ptx::smem_desc_k_sw128(k_addr + koff * (uint32_t)(kTileKeys * 128) + kin);
+    ptx::umma_bf16(d, dq, dk, idesc, k > 0 ? 1u : 0u);
+  }
+}
+
+// ------------------------------------------------------------------------------------ first pass
+__global__ void __launch_bounds__(kSweepThreads, 1)
+score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+                    const __grid_constant__ CUtensorMap tmQr, const int32_t* __restrict__ cu, int Hq, int G, int S,
+                    int d_k, int row_chunks, int cg, int X0, int X1, int stages, int n_out, float scale,
+                    float* __restrict__ real_logits, uint32_t* __restrict__ rowmax, uint16_t* __restrict__ sample,
+                    int64_t sample_slots, int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int groups = (row_chunks + cg - 1) / cg;
+  const int r = blockIdx.z;
+  const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
+  const bool do_real = grp == 0;
+  if ((int)blockIdx.x >= (do_real ? X0 : X1)) return;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
+  const int kchunks = d_k / 64;
+  const int c_first = grp * cg, c_cnt = min(cg, row_chunks - c_first);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  TileWalk walk;
+  walk.init(N, (int)blockIdx.x, do_real ? X0 : X1, !do_real);
+
+  const SweepSmem sm = carve(smem_raw, kchunks, cg, stages, true, n_out);
+  SweepTail* tail = sm.tail;
+  setup(tail, stages, &tmK, &tmQ, &tmQr);
+  const uint32_t tmem_base = tail->tmem_slot;
+  volatile int* abort_flag = &tail->abort_flag;
+  const uint32_t q_chunk_bytes = (uint32_t)kchunks * kRowChunk * 128;
+  const uint32_t qr_bytes = (uint32_t)kchunks * kRealCols * 128;
+  const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
+  const int R = G * (S + 1);                          // rows of the head group: G*S synthetic, then G current
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && walk.count > 0) {
+      const int group_row = (r * (Hq / G) + kh) * R;
+      ptx::mbar_arrive_expect_tx(&tail->q_full, (uint32_t)c_cnt * q_chunk_bytes + (do_real ? qr_bytes : 0u));
+      for (int cc = 0; cc < c_cnt; ++cc)
+        for (int c = 0; c < kchunks; ++c)
+          ptx::tma_load_2d(sm.Qs + ((size_t)cc * kchunks + c) * kRowChunk * 128, &tmQ, &tail->q_full, c * 64,
+                           group_row + (c_first + cc) * kRowChunk);
+      if (do_real)
+        for (int c = 0; c < kchunks; ++c)
+          ptx::tma_load_2d(sm.Qr + (size_t)c * kRealCols * 128, &tmQr, &tail->q_full, c * 64, group_row + G * S);
+      for (int it = 0; it < walk.count; ++it) {
+        const int s = it % stages;
+        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+        if (!wait_or_abort(&tail->empty[s], ph ^ 1u, abort_flag)) break;
+        ptx::mbar_arrive_expect_tx(&tail->full[s], stage_bytes);
+        uint8_t* dst = sm.Ks + (size_t)s * stage_bytes;
+        const int t = walk.tile(it);
+        for (int c = 0; c < kchunks; ++c)
+          ptx::tma_load_3d(dst + (size_t)c * kTileKeys * 128, &tmK, &tail->full[s], c * 64, start + t * kTileKeys, kh);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && walk.count > 0) {
+      const uint32_t idesc2 = ptx::instr_desc_bf16_f32(kTileKeys, kRealCols);   // keys x current rows
+      const uint32_t q_addr = ptx::smem_u32(sm.Qs), qr_addr = ptx::smem_u32(sm.Qr);
+      bool ok = wait_or_abort(&tail->q_full, 0, abort_flag);
+      int n1 = 0;                                      // full products issued so far
+      for (int it = 0; ok && it < walk.count; ++it) {
+        const int s = it % stages;
+        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+        if (!wait_or_abort(&tail->full[s], ph, abort_flag)) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t k_addr = ptx::smem_u32(sm.Ks + (size_t)s * stage_bytes);
+        if (do_real) {
+          const int ar = it & 1;
+          if (!wait_or_abort(&tail->real_empty[ar], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) break;
+          ptx::tc_fence_after_sync();
+          const uint32_t d2 = tmem_base + (uint32_t)(kD2Col + ar * 32);
+          const int ksteps = d_k / 16;
+          for (int k = 0; k < ksteps; ++k) {
+            const uint32_t koff = (uint32_t)(k >> 2), kin = (uint32_t)(k & 3) * 32u;
+            const uint64_t dk = ptx::smem_desc_k_sw128(k_addr + koff * (uint32_t)(kTileKeys * 128) + kin);
+            const uint64_t dq = ptx::smem_desc_k_sw128(qr_addr + koff * (uint32_t)(kRealCols * 128) + kin);
+            ptx::umma_bf16(d2, dk, dq, idesc2, k > 0 ? 1u : 0u);
+          }
+          ptx::umma_commit(&tail->real_full[ar]);
+        }
+        if (walk.slot(it) >= 0) {
+          for (int cc = 0; ok && cc < c_cnt; ++cc, ++n1) {
+            const int a = n1 & 1;
+            if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)n1 >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            issue_d1(tmem_base + (uint32_t)(a * kRowChunk), q_addr + (uint32_t)cc * q_chunk_bytes, k_addr, d_k);
+            ptx::umma_commit(&tail->acc_full[a]);
+          }
+        }
+        ptx::umma_commit(&tail->empty[s]);       // the ring slot is free once these MMAs have read it
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ read-out (8 warps)
+    const int e = warp - 2;                      // 0..7
+    const int q = warp & 3;                      // tensor-memory lane quadrant this warp may read
+    const int half = e >> 2;                     // which 64 keys of the tile this warp takes
+    const int row = q * 32 + lane;               // D1 lane = synthetic row of the chunk; D2 lane = key of the tile
+    const bool leader = (e == 0 && lane == 0);
+    float* Lreq = real_logits + (int64_t)Hq * start;
+    int n1 = 0;
+    for (int it = 0; it < walk.count; ++it) {
+      const int t = walk.tile(it);
+      // ---- current-query rows: thread = key, exact fp32 logits and their running maximum
+      if (do_real && half == 0) {
+        const int ar = it & 1;
+        const bool got = wait_or_abort(&tail->real_full[ar], ((uint32_t)it >> 1) & 1u, abort_flag);
+        ptx::tc_fence_after_sync();
+        uint32_t w[16];
+        ptx::tmem_ld_32x16(tmem_base + (uint32_t)(kD2Col + ar * 32) + ((uint32_t)(q * 32) << 16), w);
+        ptx::tmem_wait_ld();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tail->real_empty[ar]);
+        const int n = t * kTileKeys + row;
+        const bool valid = got && n < N;
+#pragma unroll
+        for (int i = 0; i < kRealCols; ++i) {
+          if (i < G) {
+            const float l = __uint_as_float(w[i]) * scale;
+            if (valid) Lreq[(int64_t)(kh * G + i) * Ncap + n] = l;
+            const uint32_t wmax = __reduce_max_sync(0xffffffffu, valid ? ordered_key(l) : 0u);
+            if (lane == 0 && wmax) atomicMax(&tail->rowmax[i], wmax);
+          }
+        }
+      }
+      // ---- sampled tile: the synthetic rows' logits as half-precision keys, one staged tile per chunk
+      const int js = walk.slot(it);
+      if (js < 0) continue;
+      const int valid_keys_in_tile = N - t * kTileKeys;          // >= 128 except on a ragged last tile
+      for (int cc = 0; cc < c_cnt; ++cc, ++n1) {
+        const int a = n1 & 1;
+        uint8_t* obuf = sm.Os + (size_t)(n1 % n_out) * (kRowChunk * kTileKeys * 2);
+        // the staging buffer about to be overwritten must have been read by its bulk copy
+        if (leader) { if (n_out == 2) ptx::bulk_wait_read<1>(); else ptx::bulk_wait_read<0>(); }
+        ptx::named_barrier_sync(1, kEpiWarps * 32);
+        wait_or_abort(&tail->acc_full[a], ((uint32_t)n1 >> 1) & 1u, abort_flag);
+        ptx::tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + (uint32_t)(a * kRowChunk) + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 64);
+        uint32_t v0[32], v1[32];
+        ptx::tmem_ld_32x32(taddr, v0);
+        ptx::tmem_ld_32x32(taddr + 32u, v1);
+        ptx::tmem_wait_ld();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tail->acc_empty[a]);
+        // 16-byte piece c of the row (keys 8c .. 8c+7) sits at piece position c ^ (row & 15): the stores of
+        // a warp then spread over the banks; the order inside a row's sample does not matter to its ranks
+        uint8_t* orow = obuf + (size_t)row * (kTileKeys * 2);
+        const uint32_t swz = (uint32_t)row & 15u;
+        const int col0 = half * 64;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t* v = c < 4 ? &v0[8 * c] : &v1[8 * (c - 4)];
+          uint32_t pk[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float l0 = __uint_as_float(v[2 * j]) * scale, l1 = __uint_as_float(v[2 * j + 1]) * scale;
+            if (col0 + 8 * c + 2 * j >= valid_keys_in_tile) l0 = -INFINITY;       // pad of a ragged last tile
+            if (col0 + 8 * c + 2 * j + 1 >= valid_keys_in_tile) l1 = -INFINITY;
+            pk[j] = key16x2_of(l0, l1);
+            if (l0 == -INFINITY) pk[j] = (pk[j] & 0xffff0000u) | 0xfc00u;         // satfinite clamps: put -inf back
+            if (l1 == -INFINITY) pk[j] = (pk[j] & 0x0000ffffu) | 0xfc000000u;
+          }
+          *reinterpret_cast<uint4*>(orow + ((((uint32_t)(half * 8 + c)) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        ptx::fence_proxy_async();                // staged tile visible to the bulk-copy engine
+        ptx::named_barrier_sync(2, kEpiWarps * 32);
+        if (leader) {
+          const int64_t slot = sample_slot_offset(start, r) + js;
+          uint16_t* gdst = sample + ((((int64_t)kh * sample_slots + slot) * row_chunks + (c_first + cc)) * kRowChunk) * kTileKeys;
+          ptx::bulk_store(gdst, obuf, (uint32_t)(kRowChunk * kTileKeys * 2));
+          ptx::bulk_commit();
+        }
+      }
+    }
+    if (leader) ptx::bulk_wait_all<0>();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (threadIdx.x == 0 && tail->abort_flag) {
+    atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
+    atomicExch(&status[1], 5);
+  }
+  if (do_real && (int)threadIdx.x < G && tail->rowmax[threadIdx.x] != 0)
+    atomicMax(&rowmax[r * Hq + kh * G + (int)threadIdx.x], tail->rowmax[threadIdx.x]);
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------ second pass
+template <int CG>
+__global__ void __launch_bounds__(kSweepThreads, 1)
+score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+                   const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int row_chunks, int stages,
+                   float scale, const RowBracket* __restrict__ bracket, uint32_t* __restrict__ above,
+                   uint32_t* __restrict__ ncand, uint2* __restrict__ cand, int cap, uint32_t* __restrict__ tmask,
+                   int64_t row_words, int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int groups = (row_chunks + CG - 1) / CG;
+  const int r = blockIdx.z;
+  const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
+  const int start = cu[r], Ncap = cu[r + 1] - start;
+  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
+  const int kchunks = d_k / 64;
+  const int c_first = grp * CG, c_cnt = min(CG, row_chunks - c_first);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  TileWalk walk;
+  walk.init(N, (int)blockIdx.x, (int)gridDim.x, false);
+
+  const SweepSmem sm = carve(smem_raw, kchunks, CG, stages, false, 0);
+  SweepTail* tail = sm.tail;
+  setup(tail, stages, &tmK, &tmQ, nullptr);
+  const uint32_t tmem_base = tail->tmem_slot;
+  volatile int* abort_flag = &tail->abort_flag;
+  const uint32_t q_chunk_bytes = (uint32_t)kchunks * kRowChunk * 128;
+  const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
+  const int R = G * (S + 1);
+
+  if (warp == 0) {
+    if (lane == 0 && walk.count > 0) {
+      const int group_row = (r * (Hq / G) + kh) * R;
+      ptx::mbar_arrive_expect_tx(&tail->q_full, (uint32_t)c_cnt * q_chunk_bytes);
+      for (int cc = 0; cc < c_cnt; ++cc)
+        for (int c = 0; c < kchunks; ++c)
+          ptx::tma_load_2d(sm.Qs + ((size_t)cc * kchunks + c) * kRowChunk * 128, &tmQ, &tail->q_full, c * 64,
+                           group_row + (c_first + cc) * kRowChunk);
+      for (int it = 0; it < walk.count; ++it) {
+        const int s = it % stages;
+        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+        if (!wait_or_abort(&tail->empty[s], ph ^ 1u, abort_flag)) break;
+        ptx::mbar_arrive_expect_tx(&tail->full[s], stage_bytes);
+        uint8_t* dst = sm.Ks + (size_t)s * stage_bytes;
+        const int t = walk.tile(it);
+        for (int c = 0; c < kchunks; ++c)
+          ptx::tma_load_3d(dst + (size_t)c * kTileKeys * 128, &tmK, &tail->full[s], c * 64, start + t * kTileKeys, kh);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && walk.count > 0) {
+      const uint32_t q_addr = ptx::smem_u32(sm.Qs);
+      bool ok = wait_or_abort(&tail->q_full, 0, abort_flag);
+      int n1 = 0;
+      for (int it = 0; ok && it < walk.count; ++it) {
+        const int s = it % stages;
+        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+        if (!wait_or_abort(&tail->full[s], ph, abort_flag)) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t k_addr = ptx::smem_u32(sm.Ks + (size_t)s * stage_bytes);
+        for (int cc = 0; cc < c_cnt; ++cc, ++n1) {
+          const int a = n1 & 1;
+          if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)n1 >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          issue_d1(tmem_base + (uint32_t)(a * kRowChunk), q_addr + (uint32_t)cc * q_chunk_bytes, k_addr, d_k);
+          ptx::umma_commit(&tail->acc_full[a]);
+        }
+        ptx::umma_commit(&tail->empty[s]);
+      }
+    }
+  } else {
+    const int e = warp - 2;
+    const int q = warp & 3;
+    const int half = e >> 2;
+    // this thread's row in each chunk of the group: its bracket, its list, its count of keys above
+    float lo[CG], hi[CG];
+    uint32_t abv[CG];
+    int rowid[CG];
+#pragma unroll
+    for (int cc = 0; cc < CG; ++cc) {
+      const int grow = (c_first + cc) * kRowChunk + q * 32 + lane;       // row within the head group
+      abv[cc] = 0;
+      rowid[cc] = -1;
+      lo[cc] = INFINITY;
+      hi[cc] = INFINITY;
+      if (cc < c_cnt && grow < G * S) {
+        rowid[cc] = (r * Hq + kh * G + grow / S) * S + grow % S;
+        const RowBracket b = bracket[rowid[cc]];
+        lo[cc] = b.lo;
+        hi[cc] = b.hi;
+      }
+    }
+    uint32_t* mrow = tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
+    int n1 = 0;
+    for (int it = 0; it < walk.count; ++it) {
+      const int t = walk.tile(it);
+      // keys of this half of the tile that exist (a ragged last tile reads whatever follows the row)
+      const int left = N - t * kTileKeys - half * 64;
+      const uint32_t vm0 = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
+      const uint32_t vm1 = left >= 64 ? 0xffffffffu : (left > 32 ? (1u << (left - 32)) - 1u : 0u);
+      const int n0 = t * kTileKeys + half * 64;
+#pragma unroll
+      for (int cc = 0; cc < CG; ++cc) {
+        if (cc >= c_cnt) break;
+        const int a = n1 & 1;
+        wait_or_abort(&tail->acc_full[a], ((uint32_t)n1 >> 1) & 1u, abort_flag);
+        ++n1;
+        ptx::tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + (uint32_t)(a * kRowChunk) + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 64);
+        uint32_t v0[32], v1[32];
+        ptx::tmem_ld_32x32(taddr, v0);
+        ptx::tmem_ld_32x32(taddr + 32u, v1);
+        ptx::tmem_wait_ld();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tail->acc_empty[a]);     // the values are in registers: free the accumulator
+
+        const float hi_r = hi[cc], lo_r = lo[cc];
+        uint32_t ab0 = 0, ab1 = 0, cb0 = 0, cb1 = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float l0 = __uint_as_float(v0[i]) * scale, l1 = __uint_as_float(v1[i]) * scale;
+          ab0 |= (l0 > hi_r ? 1u : 0u) << i;
+          cb0 |= (l0 >= lo_r ? 1u : 0u) << i;
+          ab1 |= (l1 > hi_r ? 1u : 0u) << i;
+          cb1 |= (l1 >= lo_r ? 1u : 0u) << i;
+        }
+        ab0 &= vm0; ab1 &= vm1;
+        cb0 &= vm0 & ~ab0; cb1 &= vm1 & ~ab1;
+        // union step: the warp's 32 rows OR their bits, one atomic per mask word
+        const uint32_t w0 = __reduce_or_sync(0xffffffffu, ab0), w1 = __reduce_or_sync(0xffffffffu, ab1);
+        if (lane == 0) {
+          if (w0) atomicOr(&mrow[(n0 >> 5)], w0);
+          if (w1) atomicOr(&mrow[(n0 >> 5) + 1], w1);
+        }
+        abv[cc] += __popc(ab0) + __popc(ab1);
+        const uint32_t cnt = __popc(cb0) + __popc(cb1);
+        if (cnt) {
+          uint32_t slot = atomicAdd(&ncand[rowid[cc]], cnt);
+          uint2* list = cand + (int64_t)rowid[cc] * cap;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if ((cb0 >> i) & 1u) {
+              if (slot < (uint32_t)cap) list[slot] = make_uint2(__float_as_uint(__uint_as_float(v0[i]) * scale), (uint32_t)(n0 + i));
+              ++slot;
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if ((cb1 >> i) & 1u) {
+              if (slot < (uint32_t)cap) list[slot] = make_uint2(__float_as_uint(__uint_as_float(v1[i]) * scale), (uint32_t)(n0 + 32 + i));
+              ++slot;
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int cc = 0; cc < CG; ++cc)
+      if (rowid[cc] >= 0 && abv[cc]) atomicAdd(&above[rowid[cc]], abv[cc]);
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (threadIdx.x == 0 && tail->abort_flag) {
+    atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
+    atomicExch(&status[1], 6);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+constexpr size_t kSmemLimit = 227 * 1024;
+
+// Largest chunk count (4, 2 or 1, at most row_chunks rounded up) whose query rows leave room for `min_stages`
+// key stages next to `extra` bytes; returns the stage count through `stages`.
+int pick_chunks(int row_chunks, int kchunks, size_t extra, int min_stages, int* stages) {
+  const size_t q_chunk = (size_t)kchunks * kRowChunk * 128, stage = (size_t)kchunks * kTileKeys * 128;
+  for (int cg = 4; cg >= 1; cg >>= 1) {
+    if (cg > 1 && cg / 2 >= row_chunks) continue;
+    const size_t fixed = 1024 + cg * q_chunk + extra + sizeof(SweepTail) + 64;
+    if (fixed + (size_t)min_stages * stage > kSmemLimit) continue;
+    int st = (int)((kSmemLimit - fixed) / stage);
+    if (st > kMaxStages) st = kMaxStages;
+    *stages = st;
+    return cg;
+  }
+  return 0;
+}
+
+bool encode_maps(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
+                 int32_t batch, int64_t total_tokens, CUtensorMap* tmK, CUtensorMap* tmQ, CUtensorMap* tmQr) {
+  const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, S1 = p->S + 1, d_k = p->d_k;
+  {
+    const uint64_t dims[3] = {(uint64_t)d_k, (uint64_t)total_tokens, (uint64_t)Hkv};
+    const uint64_t strides[2] = {(uint64_t)k_tok * 2, (uint64_t)k_head * 2};
+    const uint32_t box[3] = {64, (uint32_t)kTileKeys, 1};
+    if (k_head <= 0 || !encode_tensor_map_bf16(tmK, K, 3, dims, strides, box)) return false;
+  }
+  const uint64_t dims[2] = {(uint64_t)d_k, (uint64_t)batch * Hq * S1};
+  const uint64_t strides[1] = {(uint64_t)d_k * 2};
+  const uint32_t box[2] = {64, (uint32_t)kRowChunk};
+  const uint32_t boxr[2] = {64, (uint32_t)kRealCols};
+  if (!encode_tensor_map_bf16(tmQ, Q, 2, dims, strides, box)) return false;
+  if (tmQr && !encode_tensor_map_bf16(tmQr, Q, 2, dims, strides, boxr)) return false;
+  return true;
+}
+
+}  // namespace
+
+bool sweep_umma_supported(const gvote_params* p) {
+  return p->d_k % 64 == 0 && p->d_k <= 256 && p->n_q_heads / p->n_kv_heads <= kRealCols;
+}
+
+// First pass.  Returns GVOTE_ERR_UNSUPPORTED_SHAPE when the tensor maps cannot describe the operands (the
+// caller then takes the SIMT path).
+int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                            int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                            float* real_logits, uint32_t* rowmax, const VoteState& vs, int32_t* status,
+                            const int32_t* kv_len, cudaStream_t st) {
+  const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, d_k = p->d_k;
+  const int row_chunks = score_geometry(p).row_chunks;
+  CUtensorMap tmK, tmQ, tmQr;
+  if (!encode_maps(p, Q, K, k_tok, k_head, batch, total_tokens, &tmK, &tmQ, &tmQr)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  const int kchunks = d_k / 64;
+  const size_t out_bytes = (size_t)kRowChunk * kTileKeys * 2;
+  const size_t qr = align_up((size_t)kchunks * kRealCols * 128, 1024);
+  int stages = 0, n_out = 2;
+  int cg = pick_chunks(row_chunks > 2 ? 2 : row_chunks, kchunks, qr + 2 * out_bytes, 3, &stages);
+  if (cg == 0) { n_out = 1; cg = pick_chunks(row_chunks > 2 ? 2 : row_chunks, kchunks, qr + out_bytes, 2, &stages); }
+  if (cg == 0) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  const size_t smem = 1024 + (size_t)cg * kchunks * kRowChunk * 128 + qr + (size_t)stages * kchunks * kTileKeys * 128 +
+                      n_out * out_bytes + sizeof(SweepTail) + 64;
+  const int groups = (row_chunks + cg - 1) / cg;
+  // CTAs per (request, KV head): one per SM when the batch is uniform; a ragged batch gets four times as
+  // many, shorter CTAs so that the hardware scheduler can even out long and short requests.  The group that
+  // streams every tile takes most of them, the groups that visit only the sampled tiles the rest.
+  const int64_t max_tiles = ceil_div(max_N, kTileKeys);
+  int64_t budget = (batch == 1 ? 148 : 592) / ((int64_t)Hkv * batch);
+  if (budget < 1) budget = 1;
+  int64_t X1 = groups > 1 ? budget / (6 * (groups - 1)) : 0;
+  if (groups > 1 && X1 < 1) X1 = 1;
+  int64_t X0 = budget - (groups - 1) * X1;
+  if (X0 < 1) X0 = 1;
+  if (X0 > max_tiles) X0 = max_tiles;
+  dim3 grid((unsigned)(X0 > X1 ? X0 : X1), (unsigned)(Hkv * groups), (unsigned)batch);
+  const float scale = (float)(1.0 / sqrt((double)d_k));
+  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    LaunchScope scope_("score_sample_kernel", st);
+    score_sample_kernel<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, tmQr, cu, Hq, G, p->S, d_k, row_chunks, cg, (int)X0,
+                                                           (int)X1, stages, n_out, scale, real_logits, rowmax, vs.sample,
+                                                           vs.sample_slots, status, kv_len);
+  }
+  GVOTE_LAUNCH_CHECK("score_sample_kernel");
+  return GVOTE_OK;
+}
+
+// Second pass (after bracket_kernel).
+int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                           const VoteState& vs, int64_t row_words, int32_t* status, const int32_t* kv_len,
+                           cudaStream_t st) {
+  const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, d_k = p->d_k;
+  const int row_chunks = score_geometry(p).row_chunks;
+  CUtensorMap tmK, tmQ;
+  if (!encode_maps(p, Q, K, k_tok, k_head, batch, total_tokens, &tmK, &tmQ, nullptr)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  const int kchunks = d_k / 64;
+  int stages = 0;
+  const int cg = pick_chunks(row_chunks, kchunks, 0, 2, &stages);
+  if (cg == 0) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  const size_t smem = 1024 + (size_t)cg * kchunks * kRowChunk * 128 + (size_t)stages * kchunks * kTileKeys * 128 +
+                      sizeof(SweepTail) + 64;
+  const int groups = (row_chunks + cg - 1) / cg;
+  const int64_t max_tiles = ceil_div(max_N, kTileKeys);
+  int64_t X = (batch == 1 ? 148 : 592) / ((int64_t)Hkv * groups * batch);
+  if (X > max_tiles) X = max_tiles;
+  if (X < 1) X = 1;
+  dim3 grid((unsigned)X, (unsigned)(Hkv * groups), (unsigned)batch);
+  const float scale = (float)(1.0 / sqrt((double)d_k));
+  auto kern = cg == 4 ? score_sweep_kernel<4> : (cg == 2 ? score_sweep_kernel<2> : score_sweep_kernel<1>);
+  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    LaunchScope scope_("score_sweep_kernel", st);
+    kern<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, stages, scale, vs.bracket,
+                                            vs.above, vs.ncand, vs.cand, vs.cap, vs.tmask, row_words, status, kv_len);
+  }
+  GVOTE_LAUNCH_CHECK("score_sweep_kernel");
+  return GVOTE_OK;
+}
+
+}  // namespace gvote

@@ -1,0 +1,126 @@
+// Geometry shared by the kernels of the fused vote (Algorithm 1: logits, TopK, union without the S x N
+// logits ever reaching memory): which key tiles of a row form its sample, where a row's sampled keys,
+// its bracket, its counters and its candidate list live, and the exact fp32 logit of one key.
+//
+// A row is one synthetic query of one query head: global row id = (r * n_q_heads + g) * S + s.
+// Inside its KV head's group it is row gl * S + s (gl = g mod G) of the G * S synthetic rows, i.e. row
+// `crow` of 128-row chunk `chunk`.
+#pragma once
+
+#include "common.cuh"
+
+namespace gvote {
+
+constexpr int kVoteTileKeys = 128;   // keys per tile of the score contraction
+constexpr int kVoteRowChunk = 128;   // synthetic rows per accumulator (MMA M)
+
+// The sample of a row of N keys, in whole key tiles.  Rows of at most 32 tiles are sampled completely
+// (the bracket then is the threshold itself); longer rows take `ns` of their full tiles, one from each
+// stretch of `stride` tiles, at an offset that changes from stretch to stretch so that a periodic
+// pattern in the keys cannot line up with the sample.
+struct SampleGeom {
+  int n_tiles, ns, stride;
+  bool whole;
+};
+__host__ __device__ __forceinline__ SampleGeom sample_geom(int N) {
+  SampleGeom g;
+  g.n_tiles = (N + kVoteTileKeys - 1) / kVoteTileKeys;
+  if (g.n_tiles <= 32) {
+    g.ns = g.n_tiles;
+    g.stride = 1;
+    g.whole = true;
+  } else {
+    int want = g.n_tiles >> 3;
+    want = want < 32 ? 32 : (want > 128 ? 128 : want);
+    const int n_full = N / kVoteTileKeys;          // >= 32 here
+    g.ns = want;
+    g.stride = n_full / want;                      // >= 1
+    g.whole = false;
+  }
+  return g;
+}
+__host__ __device__ __forceinline__ int sample_tile(const SampleGeom& g, int j) {
+  if (g.stride == 1) return j;
+  const uint32_t hsh = ((uint32_t)j * 2654435761u) >> 15;
+  return j * g.stride + (int)(hsh % (uint32_t)g.stride);
+}
+// Position of tile t in the sample, or -1.
+__host__ __device__ __forceinline__ int sample_slot_of_tile(const SampleGeom& g, int t) {
+  const int j = t / g.stride;
+  return (j < g.ns && sample_tile(g, j) == t) ? j : -1;
+}
+// Keys in the sample (a completely sampled row counts its N keys; the pad of its last tile reads as -inf).
+__host__ __device__ __forceinline__ int sample_keys(const SampleGeom& g, int N) {
+  return g.whole ? N : g.ns * kVoteTileKeys;
+}
+// First sample-tile slot of request r in the sample buffer, and the slots a batch needs: a request of
+// N keys takes at most 32 + N / 1024 + 1 slots.
+__host__ __device__ __forceinline__ int64_t sample_slot_offset(int cu_r, int r) { return (int64_t)34 * r + (cu_r >> 10); }
+inline int64_t sample_slots_total(int32_t batch, int64_t total_tokens) { return (int64_t)34 * batch + (total_tokens >> 10) + 1; }
+
+// Entries a row's candidate list holds.  The bracket spans 2 * (4.5 sqrt(m f (1 - f)) + 6) of the m
+// sampled keys' ranks, at most 4.5 sqrt(m) + 12, i.e. that many times N / m keys of the row; a quarter
+// more covers the spread of the count.  A completely sampled row lists only the keys that share the
+// threshold's 16-bit value or its neighbours'.
+inline int candidate_cap(int64_t max_N) {
+  if (max_N <= 0) return 256;
+  const SampleGeom g = sample_geom((int)max_N);
+  double need = 512.0;
+  if (!g.whole) {
+    const double m = (double)g.ns * kVoteTileKeys;
+    need = 1.25 * (4.5 * sqrt(m) + 12.0) * ((double)max_N / m) + 256.0;
+  }
+  int cap = 1024;
+  while (cap < need) cap += 1024;
+  return cap;
+}
+
+struct RowBracket { float lo, hi; };    // keys above hi are taken, keys in [lo, hi] are listed
+
+// Where the fused vote keeps its state in the workspace.
+struct VoteState {
+  uint16_t* sample;        // fp16 keys [n_kv_heads][sample slots][row_chunks][128 rows][128 keys]
+  RowBracket* bracket;     // [rows]
+  uint32_t* above;         // [rows] keys above the bracket (counted by the sweep)
+  uint32_t* ncand;         // [rows] keys inside the bracket (listed by the sweep, up to `cap`)
+  uint2* cand;             // [rows][cap] (fp32 logit bits, key index)
+  uint32_t* tmask;         // [n_kv_heads][row_words] the union while it is tentative
+  uint32_t* head_bad;      // [batch][n_kv_heads] a bracket of the head missed: redo the head exactly
+  int cap;
+  int64_t sample_slots;
+};
+
+#ifdef __CUDACC__
+// Exact fp32 logit of key n for one query row (fixed summation order).
+struct DotCtx {
+  const __nv_bfloat16* qf;      // the row's query, d_k values (shared memory)
+  const __nv_bfloat16* krows;   // K + head offset + request start
+  int64_t k_tok;
+  int d_k;
+  float scale;
+  __device__ __forceinline__ void add8(float& acc, const uint4& v, int c) const {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h[j]);
+      const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qf + c * 8 + 2 * j));
+      acc = fmaf(q.x, f.x, acc);
+      acc = fmaf(q.y, f.y, acc);
+    }
+  }
+  __device__ __forceinline__ float operator()(int n) const {
+    const uint4* kp = reinterpret_cast<const uint4*>(krows + (int64_t)n * k_tok);
+    float acc = 0.f;
+    const int nc = d_k / 8;
+    int c = 0;
+    for (; c + 4 <= nc; c += 4) {                     // four loads in flight, summed in index order
+      const uint4 v0 = __ldg(kp + c), v1 = __ldg(kp + c + 1), v2 = __ldg(kp + c + 2), v3 = __ldg(kp + c + 3);
+      add8(acc, v0, c); add8(acc, v1, c + 1); add8(acc, v2, c + 2); add8(acc, v3, c + 3);
+    }
+    for (; c < nc; ++c) add8(acc, __ldg(kp + c), c);
+    return acc * scale;
+  }
+};
+#endif
+
+}  // namespace gvote

@@ -123,7 +123,8 @@ def make_config(name: str, **overrides) -> GVoteConfig:
     elif name == "c4":
         cfg = GVoteConfig(name="c4", d_h=3584, n_q_heads=28, n_kv_heads=4, d_k=128,
                           rope_theta=1.0e6, S=64, p_nuc=0.98, seq_lens=(131072,), seed=4,
-                          n_layers=28, h_mode="diag", heavy_frac=(0.001,), local_window=512)
+                          n_layers=28, h_mode="diag", heavy_frac=(0.001,), local_window=512,
+                          heavy_gain=4.0)
     else:
         raise ValueError(f"unknown config {name!r}")
     return replace(cfg, **overrides) if overrides else cfg

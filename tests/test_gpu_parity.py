@@ -229,6 +229,24 @@ def test_vote_configs(gv, name, mode):
     _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode)
 
 
+def test_vote_many_row_chunks_strict_band(gv):
+    """G = 7 query heads per KV head and S = 64 synthetic queries: 448 synthetic rows per KV head, i.e.
+    four 128-row chunks in the score contraction, on rows long enough for the sampled bracket (ragged
+    last tile).  Oracle's queries, default 1e-3 bands."""
+    cfg = synth.make_small(21, seq_lens=(9001,), S=64, d_h=128, n_q_heads=7, n_kv_heads=1, d_k=128, p_nuc=0.98,
+                           heavy_frac=(0.01,))
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
+
+
+@pytest.mark.parametrize("N", [33000, 50001])
+def test_vote_topp_long_rows_strict_band(gv, N):
+    """Per-sample top-p on rows of more than 32K keys (N = 50001 no longer fits the shared-memory
+    staging of a row).  Oracle's queries, default 1e-3 bands."""
+    cfg = synth.make_small(22, seq_lens=(N,), S=3, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=64, p_nuc=0.95,
+                           heavy_frac=(0.002,))
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topp", want_probs=False)
+
+
 def test_vote_degenerate_all_keys_equal(gv):
     """Every logit ties: top-p keeps ceil(p N) keys and top-k keeps exactly k, lowest indices first."""
     cfg = synth.make_small(5, seq_lens=(100,), S=3, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=32, p_nuc=0.5)
@@ -292,7 +310,9 @@ def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
 # ----------------------------------------------------------------------------- compact
 @pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
                                                   ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
-                                                  ((1000,), 1, 8, 1.0), ((1000,), 1, 16, 0.0)])
+                                                  ((1000,), 1, 8, 1.0), ((1000,), 1, 16, 0.0),
+                                                  ((131072,), 4, 128, 0.01), ((131072,), 4, 128, 0.3),
+                                                  ((131072,), 8, 128, 0.9), ((131072,), 4, 128, 0.7)])
 def test_compact_bit_exact(gv, lens, Hkv, d_k, density):
     rng = np.random.default_rng(12)
     T, B = sum(lens), len(lens)
@@ -301,7 +321,9 @@ def test_compact_bit_exact(gv, lens, Hkv, d_k, density):
     V = rng.integers(0, 65536, size=(Hkv, T, d_k)).astype(np.uint16)
     keep = rng.random((Hkv, T)) < density
     if density == 0.7:
-        keep[0, :1500] = True                                                 # long fully-kept prefix
+        keep[0, :T // 3 + 135] = True                                         # long fully-kept prefix
+        if Hkv > 1:
+            keep[1, :] = True                                                 # a head that keeps every key
     words = np.zeros((Hkv, gv.mask_row_words(T, B)), dtype=np.uint32)
     for r in range(B):
         for h in range(Hkv):
@@ -380,7 +402,8 @@ def test_overlap_matches_oracle(gv, idx):
 # ----------------------------------------------------------------------------- varlen packing
 @pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
                                                   ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
-                                                  ((1000,), 1, 8, 1.0), ((1000, 77), 2, 16, 0.0)])
+                                                  ((1000,), 1, 8, 1.0), ((1000, 77), 2, 16, 0.0),
+                                                  ((131072,), 4, 128, 0.01), ((131072,), 4, 128, 0.9)])
 def test_pack_varlen_bit_exact(gv, lens, Hkv, d_k, density):
     """gvote_pack against the oracle's packing, bit for bit, with K and V left untouched."""
     rng = np.random.default_rng(31)
@@ -812,6 +835,75 @@ def test_compress_full_size_c4_layer(gv):
     layers = _layers_to_check(1)
     for layer in (range(cfg.n_layers) if layers is None else layers):
         _check_compress(gv, cfg, synth.make_layer(cfg, layer), layer_id=layer)
+
+
+def _check_stages_strict(gv, cfg, li, layer_id):
+    """The stages one by one on a full-size layer, every stage fed what the stage before it produced on
+    the GPU and checked against the oracle's step on those same inputs, so that each is held to its own
+    stated tolerance at full size: fit 1e-5; normal draws 1e-5 on z; rotated queries within one bf16
+    step plus the rounding of an fp32 accumulation; the vote inside the 1e-3 bands."""
+    p = gv.params_from_config(cfg, layer_id=layer_id)
+    geom = _geom(cfg)
+    B, S, G = cfg.batch, cfg.S, cfg.G
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mu = torch.empty(B, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p, d["h"], d["cu"], geom, mu, var, ws)
+    Ht = torch.empty(B, S, cfg.d_h, device="cuda")
+    gv.gvote_sample(p, mu, var, B, Ht)
+    cu = li.cu_seqlens
+    h_last = torch.from_numpy(np.stack([li.h[int(cu[r + 1]) - 1] for r in range(B)])).cuda()
+    Q = torch.empty(B, cfg.n_kv_heads, G * (S + 1), cfg.d_k, dtype=torch.bfloat16, device="cuda")
+    gv.gvote_project(p, Ht, h_last, d["W_q"], d["b_q"], d["cu"], B, Q, ws)
+    mask = torch.full((cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, B)), -1, dtype=torch.int32, device="cuda")
+    budget = torch.empty(B, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(B, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_vote(p, Q, d["K"], d["cu"], geom, mask, budget, b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    mu_g, var_g = mu.cpu().numpy().astype(np.float64), var.cpu().numpy().astype(np.float64)
+    Ht_g = Ht.cpu().numpy().astype(np.float64)
+    Qg = Q.float().cpu().numpy().astype(np.float64)
+    mask, budget, b_step = mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy()
+    W = o.bf16_bits_to_f64(li.W_q)
+    kw = pu.oracle_kwargs(cfg, layer_id)
+    for r in range(B):
+        a, b = int(cu[r]), int(cu[r + 1])
+        N = b - a
+        h64 = li.h[a:b].astype(np.float64)
+        # fit
+        m64, v64 = o.fit(h64, cfg.n_s)
+        assert np.allclose(var_g[r], v64, rtol=1e-5, atol=0)
+        assert np.abs(mu_g[r] - m64).max() <= 1e-5 * np.sqrt(v64).max() + 1e-6 * np.abs(m64).max()
+        # sample, from the GPU's moments
+        Ho, _ = o.sample(mu_g[r], var_g[r], S, cfg.seed, layer_id, r)
+        sig = np.sqrt(var_g[r])
+        assert np.abs((Ht_g[r] - Ho) / sig).max() < 1e-5 + 2e-6 * np.abs(mu_g[r] / sig).max()
+        # projection and RoPE, from the GPU's samples
+        Qo = o.queries_for_request(Ht_g[r], h64[-1], W, li.b_q, N, n_q_heads=cfg.n_q_heads, d_k=cfg.d_k,
+                                   theta=cfg.rope_theta, n_f=cfg.n_f)
+        X = o.round_to_bf16(np.concatenate([h64[-1:], Ht_g[r]]))
+        mag = (np.abs(X) @ np.abs(W).T).reshape(S + 1, cfg.n_q_heads, cfg.d_k).transpose(1, 0, 2)
+        mag = mag + np.concatenate([mag[..., cfg.d_k // 2:], mag[..., :cfg.d_k // 2]], axis=-1)
+        Qr = pu.from_group_major(Qg[r], G)
+        diff = np.abs(Qr - Qo)
+        assert np.all(diff <= 2.0 ** -7 * np.abs(Qo) + 2.0 ** -21 * mag)  # one bf16 step + fp32 accumulation
+        assert (diff == 0).mean() > 0.98
+        # the vote, from the GPU's queries
+        Kr = o.bf16_bits_to_f64(li.K[:, a:b])
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N) for h in range(cfg.n_kv_heads)])
+        pu.check_vote_against_oracle(Qr, Kr, kw["p_nuc"], "topk", False, gm, b_step[r])      # 1e-3 bands
+        om, ob, _, _, _ = o.vote(Qr, Kr, p_nuc=kw["p_nuc"])
+        assert np.array_equal(budget[r], gm.sum(axis=1))
+        assert np.all(np.abs(budget[r] - ob) <= max(1, 0.005 * N))
+        assert (gm != om).sum() <= max(2, 0.005 * N * cfg.n_kv_heads)
+
+
+@pytest.mark.parametrize("name,layer", [("c2", 3), ("c4", 1), ("c3", 0)])
+def test_stages_full_size_strict_band(gv, name, layer):
+    """Full-size layers of the 32K, the 128K (G = 7, four row chunks) and the ragged workloads, stage by
+    stage, the vote inside the 1e-3 bands."""
+    cfg = synth.make_config(name)
+    _check_stages_strict(gv, cfg, synth.make_layer(cfg, layer), layer)
 
 
 def test_recompress_full_size_c2_layer(gv):
