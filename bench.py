@@ -141,7 +141,8 @@ def flops(cfg):
 
 STAGE_OF = {
     "fit_partial_kernel": "fit", "fit_finalize_kernel": "fit", "sample_kernel": "sample",
-    "prep_kernel": "sample", "real_topp_kernel": "vote", "topk16_rows_kernel": "vote",
+    "prep_kernel": "sample", "real_topp_kernel": "vote", "score_sample_kernel": "vote", "bracket_kernel": "vote",
+    "score_sweep_kernel": "vote", "resolve_kernel": "vote", "commit_kernel": "vote",
     "xstage_kernel": "project", "rope_table_kernel": "project", "project_simt_kernel": "project",
     "project_umma_kernel": "project", "project_finish_kernel": "project",
     "score_simt_kernel": "vote", "score_umma_kernel": "vote", "topp_rows_kernel": "vote",

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "vote_geom.cuh"
 
 namespace gvote {
 
@@ -72,7 +73,12 @@ static int32_t validate_batch(int32_t batch, int64_t total_tokens, int64_t max_N
   return GVOTE_OK;
 }
 
-WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N) {
+bool vote_needs_full_rows(const gvote_params* p) {
+  return p->sel_mode != GVOTE_SEL_TOPK_C0 || !sweep_umma_supported(p);
+}
+
+WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N,
+                           bool full_rows) {
   WorkspaceMap m;
   memset(&m, 0, sizeof(m));
   const int64_t S1 = p->S + 1, F = (int64_t)p->n_q_heads * p->d_k;
@@ -92,10 +98,26 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   m.q_f32 = take((size_t)m.proj_splits * batch * S1 * F * sizeof(float));
   m.q_bf16 = take((size_t)batch * S1 * F * sizeof(__nv_bfloat16));
   m.rope = take((size_t)batch * 4 * (p->d_k / 2) * sizeof(float));
-  m.logits = take((size_t)p->n_q_heads * S1 * (size_t)total_tokens * sizeof(float));
-  m.keys16 = take(keys16_elems(p, batch, total_tokens) * sizeof(uint16_t));
-  m.real_scratch_bytes = real_topp_scratch_bytes(p, batch);
-  m.real_scratch = take(m.real_scratch_bytes);
+  m.full_rows = full_rows;
+  m.logits = take((size_t)p->n_q_heads * (full_rows ? S1 : 1) * (size_t)total_tokens * sizeof(float));
+  if (!full_rows) {
+    const size_t rows = (size_t)batch * p->n_q_heads * p->S;
+    m.cand_strip = cand_layout(batch, total_tokens, max_N).strip;
+    m.sample_slots = sample_slots_total(batch, total_tokens, max_N);
+    m.vote_zero = off;
+    m.tmask = take((size_t)p->n_kv_heads * m.row_words * sizeof(uint32_t));
+    m.head_bad = take((size_t)batch * p->n_kv_heads * sizeof(uint32_t));
+    m.rowmax = take((size_t)batch * p->n_q_heads * sizeof(uint32_t));
+    m.vote_zero_bytes = off - m.vote_zero;
+    m.sample = take((size_t)p->n_kv_heads * m.sample_slots * score_geometry(p).row_chunks * kVoteRowChunk *
+                    kVoteTileKeys * sizeof(uint16_t));
+    m.bracket = take(rows * sizeof(RowBracket));
+    m.above = take(rows * sizeof(uint32_t));
+    m.ncand = take(rows * sizeof(uint32_t));
+    m.cand = take((size_t)p->n_q_heads * p->S * (size_t)m.cand_strip * sizeof(uint2));
+  }
+  m.remap_tmp = take((size_t)p->n_kv_heads * (size_t)total_tokens * sizeof(int32_t));
+  m.ov_partial = take((size_t)batch * p->n_q_heads * (size_t)ceil_div(max_N > 0 ? max_N : 1, kOverlapKeys) * 16);
   m.prefix = take((size_t)p->n_kv_heads * m.row_words * sizeof(int32_t));
   m.flags = take(((size_t)2 * p->n_kv_heads * m.n_tiles + (size_t)2 * p->n_kv_heads * 32) * sizeof(int32_t));
   m.total = off;
@@ -150,7 +172,7 @@ int32_t gvote_project(const gvote_params* p, const float* H_tilde, const void* h
   if (wq_ld < p->d_h || wq_ld % 8 != 0) return GVOTE_ERR_UNALIGNED;
   // the projection's scratch does not depend on the token counts
   const WorkspaceMap m = workspace_map(p, batch, 0, 0);
-  if (ws_bytes < m.logits) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < m.logits) return GVOTE_ERR_WORKSPACE_TOO_SMALL;      // the areas up to the vote's
   return launch_project(p, H_tilde, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m,
                         (char*)ws, (__nv_bfloat16*)Q, (cudaStream_t)stream);
 }
@@ -164,10 +186,11 @@ int32_t gvote_vote(const gvote_params* p, const void* Q, const void* K, int64_t 
   REQUIRE_PTR(Q); REQUIRE_PTR(K); REQUIRE_PTR(cu_seqlens); REQUIRE_PTR(mask); REQUIRE_PTR(budget);
   REQUIRE_PTR(b_step); OPTIONAL_PTR(dbg_probs_or_null); REQUIRE_PTR(ws);
   if (k_tok_stride < p->d_k || k_tok_stride % 8 != 0 || k_head_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
-  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
+  // the softmax dump needs the fp32 logits of every row: the workspace of the per-sample top-p mode
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N, vote_needs_full_rows(p) || dbg_probs_or_null);
   if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
   return launch_vote(p, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, k_tok_stride, k_head_stride, cu_seqlens,
-                     batch, total_tokens, max_N, mask, budget, b_step, dbg_probs_or_null, m, (char*)ws,
+                     batch, total_tokens, max_N, mask, budget, b_step, dbg_probs_or_null, (char*)ws, ws_bytes,
                      (cudaStream_t)stream);
 }
 
@@ -183,13 +206,13 @@ int32_t gvote_select(const gvote_params* p, const float* H_tilde, const void* h_
   OPTIONAL_PTR(dbg_probs_or_null); REQUIRE_PTR(ws);
   if (wq_ld < p->d_h || wq_ld % 8 != 0) return GVOTE_ERR_UNALIGNED;
   if (k_tok_stride < p->d_k || k_tok_stride % 8 != 0 || k_head_stride % 8 != 0) return GVOTE_ERR_UNALIGNED;
-  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N);
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N, vote_needs_full_rows(p) || dbg_probs_or_null);
   if (ws_bytes < m.total) return GVOTE_ERR_WORKSPACE_TOO_SMALL;
   __nv_bfloat16* Q = reinterpret_cast<__nv_bfloat16*>((char*)ws + m.q_bf16);
   PROPAGATE(launch_project(p, H_tilde, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m,
                            (char*)ws, Q, (cudaStream_t)stream));
   return launch_vote(p, Q, (const __nv_bfloat16*)K, k_tok_stride, k_head_stride, cu_seqlens, batch, total_tokens,
-                     max_N, mask, budget, b_step, dbg_probs_or_null, m, (char*)ws, (cudaStream_t)stream);
+                     max_N, mask, budget, b_step, dbg_probs_or_null, (char*)ws, ws_bytes, (cudaStream_t)stream);
 }
 
 int32_t gvote_compact(const gvote_params* p, void* K, void* V, int64_t tok_stride, int64_t head_stride,
@@ -253,7 +276,7 @@ int32_t compress_from_moments(const gvote_params* p, const float* mu, const floa
   PROPAGATE(launch_project(p, Ht, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q, st,
                            seq_len));
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, nullptr, b_step, nullptr, m, w, st, kv_len));
+                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st, kv_len));
   PROPAGATE(launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
                            total_tokens, max_N, budget, m, w, st));
   if (token_pos) PROPAGATE(launch_remap(p, token_pos, mask, cu_seqlens, batch, total_tokens, max_N, budget, m, w, st));
@@ -346,7 +369,7 @@ int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_strid
                           cu_seqlens, cu_seqlens, batch, mu, var, X, rope, st));
   PROPAGATE(launch_project_staged(p, X, rope, W_q, wq_ld, b_q_or_null, batch, m, w, Q, st));
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, nullptr, b_step, nullptr, m, w, st));   // budgets come from the scan below
+                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st));   // budgets come from the scan below
   return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
                         total_tokens, max_N, budget, m, w, st);
 }

@@ -54,6 +54,7 @@ int32_t validate_params(const gvote_params* p);
 constexpr size_t kStatusBytes = 256;
 constexpr int kCompactTile = 128;   // tokens per compaction tile
 constexpr int kFitStripCols = 256;  // channels per fit CTA (64 column threads x 4 channels)
+constexpr int kOverlapKeys = 1024;  // keys per CTA of the attention-overlap diagnostic
 
 struct WorkspaceMap {
   size_t status;        // int32[64]
@@ -64,10 +65,24 @@ struct WorkspaceMap {
   size_t q_f32;         // float [proj_splits][batch*(S+1)][Hq*d_k]
   size_t q_bf16;        // bf16 [batch][Hq][S+1][d_k]
   size_t rope;          // float [batch][4][d_k/2]  (cos0, sin0, cbar, sbar)
-  size_t logits;        // float [Hq*(S+1) * total_tokens], request-major
-  size_t keys16;        // uint16 [Hq*S * (padded tokens)]: 16-bit logit keys of the synthetic rows
-  size_t real_scratch;  // row maxima and mass histograms of the current-query rows (topp_real.cu)
-  size_t real_scratch_bytes;
+  // --- the vote.  full_rows: fp32 logits of every row, [Hq*(S+1) * total_tokens] request-major (the
+  // per-sample top-p mode, the softmax dump, shapes the tensor-core kernels do not take); otherwise only
+  // the current-query rows, [Hq * total_tokens], and the state of the fused top-k (vote_geom.cuh)
+  bool full_rows;
+  size_t logits;
+  size_t vote_zero;     // cleared at the start of every vote: [tmask | head_bad | rowmax]
+  size_t vote_zero_bytes;
+  size_t tmask;         // uint32 [Hkv][row_words]
+  size_t head_bad;      // uint32 [batch][Hkv]
+  size_t rowmax;        // uint32 [batch][Hq]  row maxima of the current-query rows (topp_real.cu)
+  size_t sample;        // uint16 [Hkv][sample_slots][row_chunks][128][128]
+  size_t bracket;       // RowBracket [batch*Hq*S]
+  size_t above, ncand;  // uint32 [batch*Hq*S] each
+  size_t cand;          // uint2 [Hq*S][cand_strip]
+  int64_t cand_strip;
+  int64_t sample_slots;
+  size_t remap_tmp;     // int32 [Hkv][total_tokens]  scratch of the slot -> position map's gather
+  size_t ov_partial;    // float4 [batch][Hq][ceil(max_N / kOverlapKeys)]  partial sums of gvote_overlap
   size_t prefix;        // int32 [Hkv][row_words]  exclusive popcount prefix per mask word
   size_t flags;         // int32 [2*Hkv*n_tiles] compaction "tile loaded" flags + [2*Hkv][32] ticket counters
   size_t total;
@@ -81,9 +96,14 @@ struct WorkspaceMap {
 // `row_chunks` chunks of RC = 128 rows (the current-query rows travel with chunk 0).
 struct ScoreGeometry { int RC; int row_chunks; };
 ScoreGeometry score_geometry(const gvote_params* p);
-size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens);
-size_t real_topp_scratch_bytes(const gvote_params* p, int32_t batch);
-WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
+bool sweep_umma_supported(const gvote_params* p);
+// Whether the vote of these parameters keeps fp32 logits of every row (see WorkspaceMap::full_rows).
+bool vote_needs_full_rows(const gvote_params* p);
+WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N,
+                           bool full_rows);
+inline WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N) {
+  return workspace_map(p, batch, total_tokens, max_N, vote_needs_full_rows(p));
+}
 
 // ---------------------------------------------------------------------------------- stage launchers
 // (each enqueues kernels on `st`; pointers are device pointers; see gvote.h for the layouts)
@@ -123,7 +143,7 @@ int32_t launch_remap(const gvote_params* p, int32_t* token_pos, const uint32_t* 
 int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                     uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs,
-                    const WorkspaceMap& m, char* ws, cudaStream_t st,
+                    char* ws, size_t ws_bytes, cudaStream_t st,
                     const int32_t* kv_len = nullptr);   // [batch][n_kv_heads] rows that count, or all
 int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
                        const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens,

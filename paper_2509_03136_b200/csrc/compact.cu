@@ -257,15 +257,14 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
   return GVOTE_OK;
 }
 
-// After launch_compact (which leaves the prefix in the workspace and the budgets with the caller).  The
-// gather's scratch is the logits area of the workspace, dead once the vote is over.
+// After launch_compact (which leaves the prefix in the workspace and the budgets with the caller).
 int32_t launch_remap(const gvote_params* p, int32_t* token_pos, const uint32_t* mask, const int32_t* cu, int32_t batch,
                      int64_t total_tokens, int64_t max_N, const int32_t* budget, const WorkspaceMap& m, char* ws,
                      cudaStream_t st) {
   if (max_N <= 0 || total_tokens <= 0) return GVOTE_OK;
   const int Hkv = p->n_kv_heads;
   const int32_t* prefix = reinterpret_cast<const int32_t*>(ws + m.prefix);
-  int32_t* tmp = reinterpret_cast<int32_t*>(ws + m.logits);
+  int32_t* tmp = reinterpret_cast<int32_t*>(ws + m.remap_tmp);
   dim3 grid((unsigned)ceil_div(max_N, 256), (unsigned)Hkv, (unsigned)batch);
   {
     LaunchScope scope_("remap_gather_kernel", st);

@@ -12,7 +12,7 @@ namespace gvote {
 namespace {
 
 constexpr int kOvThreads = 256;
-constexpr int kOvKeys = 1024;      // keys per CTA
+constexpr int kOvKeys = kOverlapKeys;      // keys per CTA
 
 __global__ void __launch_bounds__(kOvThreads)
 overlap_partial_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K, int64_t k_tok,
@@ -110,7 +110,7 @@ int32_t launch_overlap(const gvote_params* p, const __nv_bfloat16* Q, const __nv
                        float* overlap, const WorkspaceMap& m, char* ws, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   const int chunks = (int)ceil_div(max_N > 0 ? max_N : 1, kOvKeys);
-  float4* partial = reinterpret_cast<float4*>(ws + m.logits);       // the logits area is free outside gvote_vote
+  float4* partial = reinterpret_cast<float4*>(ws + m.ov_partial);
   const float scale = (float)(1.0 / sqrt((double)p->d_k));
   dim3 g1((unsigned)chunks, (unsigned)Hq, (unsigned)batch);
   {

@@ -158,30 +158,28 @@ struct CandKeys {
 
 __global__ void __launch_bounds__(kRowThreads)
 resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32_t* __restrict__ b_step,
-               const uint32_t* __restrict__ above, const uint32_t* __restrict__ ncand, uint2* __restrict__ cand, int cap,
-               int smem_keys, uint32_t* __restrict__ tmask, int64_t row_words, uint32_t* __restrict__ head_bad,
-               const int32_t* __restrict__ kv_len) {
+               const VoteState vs, int smem_keys, int64_t row_words, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint32_t keys_sm[];
   __shared__ uint32_t red[2 * (kRowThreads / 32)];
   __shared__ uint32_t s_min, s_max;
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int rowid = (r * Hq + g) * S + s;
-  const int start = cu[r];
+  const int start = cu[r], Ncap = cu[r + 1] - start;
   const int kh = g / G, Hkv = Hq / G;
-  const int N = valid_keys(kv_len, r, Hkv, kh, cu[r + 1] - start);
+  const int N = valid_keys(kv_len, r, Hkv, kh, Ncap);
   if (N <= 0) return;
   const int k = min(b_step[r * Hq + g], N);
   if (k <= 0) return;
   const int tid = threadIdx.x;
-  const uint32_t A = above[rowid], C = ncand[rowid];
-  if (A > (uint32_t)k || C > (uint32_t)cap || A + C < (uint32_t)k) {       // the bracket missed or the list overflowed
-    if (tid == 0) atomicExch(&head_bad[r * Hkv + kh], 1u);
+  const uint32_t A = vs.above[rowid], C = vs.ncand[rowid];
+  if (A > (uint32_t)k || C > (uint32_t)vs.lay.cap(Ncap) || A + C < (uint32_t)k) {   // the bracket missed or the list overflowed
+    if (tid == 0) atomicExch(&vs.head_bad[r * Hkv + kh], 1u);
     return;
   }
   const uint32_t need = (uint32_t)k - A;
   if (need == 0) return;
-  uint2* list = cand + (int64_t)rowid * cap;
-  uint32_t* mrow = tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
+  uint2* list = vs.list(g, s, S, start, r);
+  uint32_t* mrow = vs.tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
   if (need == C) {                                         // every listed key is taken
     for (int i = tid; i < (int)C; i += kRowThreads) {
       const uint32_t n = list[i].y;
@@ -308,19 +306,19 @@ int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, 
   return GVOTE_OK;
 }
 
-int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs,
-                       int64_t row_words, const int32_t* kv_len, cudaStream_t st) {
+int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, int64_t max_N, const int32_t* b_step,
+                       const VoteState& vs, int64_t row_words, const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   dim3 grid(p->S, Hq, batch);
   // the keys of a list live in shared memory when it leaves room for six CTAs per SM
-  const int smem_keys = vs.cap <= 8192 ? vs.cap : 8192;
+  const int64_t longest = vs.lay.uniform_cap > 0 ? vs.lay.uniform_cap : vs.lay.cap((int)max_N);
+  const int smem_keys = (int)(longest <= 8192 ? longest : 8192);
   const size_t smem = (size_t)smem_keys * sizeof(uint32_t);
   if (smem > 48 * 1024)
     GVOTE_CUDA_CHECK(cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("resolve_kernel", st);
-    resolve_kernel<<<grid, kRowThreads, smem, st>>>(cu, Hq, G, p->S, b_step, vs.above, vs.ncand, vs.cand, vs.cap,
-                                                    smem_keys, vs.tmask, row_words, vs.head_bad, kv_len);
+    resolve_kernel<<<grid, kRowThreads, smem, st>>>(cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
   }
   GVOTE_LAUNCH_CHECK("resolve_kernel");
   return GVOTE_OK;

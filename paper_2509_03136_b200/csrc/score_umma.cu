@@ -1,32 +1,26 @@
-// The logits of Algorithm 1 (synthetic queries, and the current query's row A0) on the fifth-generation tensor cores:
-// L = Q K^T / sqrt(d_k) for all (S+1)*G query rows of a KV head against that head's cached keys.
+// The logits of Algorithm 1 for every query row, as fp32 rows in memory, on the fifth-generation tensor
+// cores: L = Q K^T / sqrt(d_k) for all (S+1)*G query rows of a KV head against that head's cached keys.
+// This is the route of the per-sample top-p mode (Section 3.1's rule applied to every synthetic query,
+// which needs each row's softmax mass) and of the softmax dump; the default top-k mode never writes
+// these rows (sweep_umma.cu).
 //
 // Shape of the contraction.  A KV head's G*S synthetic rows are cut into chunks of 128, and a chunk
 // goes on the MMA's M axis: D1[128 rows x 128 keys] = Qs (128 x d_k) * Ktile^T per 128-key tile, so that
-// in tensor memory a lane is a query row and a column is a key.  The read-out thread of a row thus
-// holds consecutive keys of its own row, which is the order the keys are stored in: 16-byte stores,
-// no transposition.  The G current-query rows ride along in a second, thin product with the roles
-// swapped, D2[128 keys x 16] = Ktile * Qr^T, whose read-out thread is a key and writes coalesced fp32
-// rows.  Both products read the same K tile in shared memory (TMA, 128-byte swizzle, read once from
-// HBM); both accumulators are double buffered in tensor memory so that the MMAs of tile t+1 overlap
-// the read-out of tile t.
+// in tensor memory a lane is a query row and a column is a key.  The G current-query rows ride along in
+// a second, thin product with the roles swapped, D2[128 keys x 16] = Ktile * Qr^T, whose read-out thread
+// is a key and writes coalesced fp32 rows.  Both products read the same K tile in shared memory (TMA,
+// 128-byte swizzle, read once from HBM); both accumulators are double buffered in tensor memory so that
+// the MMAs of tile t+1 overlap the read-out of tile t.
 //
 // One persistent CTA walks the key tiles x, x+X, x+2X, ... of one (request, KV head, row chunk):
 //   warp 0   : TMA producer - the chunk's query rows once, then a ring of key tiles
 //   warp 1   : allocates tensor memory, issues tcgen05.mma, commits to the ring and to the read-out
-//   warps 2-9: read-out - two warps per lane quadrant, each takes 64 of the tile's 128 keys
-//
-// Read-out, default mode.  The S x N logits never reach HBM as fp32.  Every scaled logit is rounded to
-// half precision (all the top-k search needs to bracket its threshold), staged in shared memory as a
-// [row][128 keys] tile (16-byte chunks XOR-swizzled by the row so the stores do not collide) and
-// written with one bulk copy per tile into keys16[head][tile][chunk][row][128].  Only the rows of the
-// current query are written as fp32, because the top-p mass of the set C0 needs them exactly; their
-// running maxima go to `rowmax`.  In the all-fp32 mode (per-sample top-p, softmax dump) the
-// synthetic rows are staged as fp32 instead and written to the logits buffer row by row.
+//   warps 2-9: read-out - two warps per lane quadrant, each takes 64 of the tile's 128 keys; the rows are
+//              staged in shared memory (16-byte chunks XOR-swizzled by the row) and written out row by row
 //
 // Every wait on an mbarrier is bounded.  When one runs out the CTA raises a shared abort flag,
-// records GVOTE_ERR_TIMEOUT in the workspace status word, leaves its loops, waits for its bulk
-// copies, frees its tensor memory and returns.
+// records GVOTE_ERR_TIMEOUT in the workspace status word, leaves its loops, frees its tensor memory
+// and returns.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -51,7 +45,6 @@ struct ScoreSmemTail {
   uint32_t tmem_slot;
   volatile int abort_flag;
   volatile int epi_go;                // read-out warps continue (decided by their leader, read after a barrier)
-  uint32_t rowmax[kRealCols];         // running maximum (order-preserving image) of each current-query row
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -63,34 +56,15 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
-// Two fp32 logits -> two 16-bit keys: their half-precision roundings (monotone; 11 significant bits,
-// values beyond the half range saturate to the largest finite half).
-__device__ __forceinline__ uint32_t key16x2_of(float lo, float hi) {
-  uint32_t p;
-  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(p) : "f"(hi), "f"(lo));
-  return p;
-}
-
-// Eight accumulator values -> eight half-precision keys (one 16-byte chunk).
-__device__ __forceinline__ uint4 keys8(const uint32_t* v, float scale) {
-  uint4 pk;
-  pk.x = key16x2_of(__uint_as_float(v[0]) * scale, __uint_as_float(v[1]) * scale);
-  pk.y = key16x2_of(__uint_as_float(v[2]) * scale, __uint_as_float(v[3]) * scale);
-  pk.z = key16x2_of(__uint_as_float(v[4]) * scale, __uint_as_float(v[5]) * scale);
-  pk.w = key16x2_of(__uint_as_float(v[6]) * scale, __uint_as_float(v[7]) * scale);
-  return pk;
-}
 __device__ __forceinline__ float4 logits4(const uint32_t* v, float scale) {
   return make_float4(__uint_as_float(v[0]) * scale, __uint_as_float(v[1]) * scale, __uint_as_float(v[2]) * scale,
                      __uint_as_float(v[3]) * scale);
 }
 
-template <bool ALL_F32>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                   const __grid_constant__ CUtensorMap tmQr, const int32_t* __restrict__ cu, int Hq, int G, int S1,
-                  int d_k, int row_chunks, int stages, int n_out, float scale, int64_t n_tiles_total,
-                  float* __restrict__ logits, uint16_t* __restrict__ keys16, uint32_t* __restrict__ rowmax,
+                  int d_k, int row_chunks, int stages, float scale, float* __restrict__ logits,
                   int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int r = blockIdx.z;
@@ -110,19 +84,18 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   const uint32_t q_bytes = (uint32_t)kchunks * kRowChunk * 128;
   const uint32_t qr_bytes = (uint32_t)kchunks * kRealCols * 128;
   const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
-  const uint32_t out_bytes = ALL_F32 ? (uint32_t)kRowChunk * kTileKeys * 4 : (uint32_t)kRowChunk * kTileKeys * 2;
+  const uint32_t out_bytes = (uint32_t)kRowChunk * kTileKeys * 4;
   uint8_t* Qs = base;
   uint8_t* Qr = Qs + q_bytes;
   uint8_t* Ks = Qr + ((qr_bytes + 1023u) & ~1023u);
   uint8_t* Os = Ks + (size_t)stages * stage_bytes;
-  ScoreSmemTail* tail = reinterpret_cast<ScoreSmemTail*>(Os + (size_t)n_out * out_bytes);
+  ScoreSmemTail* tail = reinterpret_cast<ScoreSmemTail*>(Os + out_bytes);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
     ptx::mbar_init(&tail->q_full, 1);
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(&tail->tmem_full[a], 1); ptx::mbar_init(&tail->tmem_empty[a], kEpiWarps); }
     tail->abort_flag = 0;
-    for (int i = 0; i < kRealCols; ++i) tail->rowmax[i] = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmK);
     ptx::prefetch_tensormap(&tmQ);
@@ -205,21 +178,17 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const int row = q * 32 + lane;               // D1 lane = synthetic row of the chunk; D2 lane = key of the tile
     const bool leader = (e == 0 && lane == 0);
     float* Lreq = logits + (int64_t)Hq * S1 * start;
-    const int64_t tile_base = ((int64_t)kh * n_tiles_total + tile_offset(start, r)) * row_chunks + chunk;
     int it = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
       const int a = it & 1;
       const uint32_t aph = (uint32_t)(it >> 1) & 1u;
       wait_or_abort(&tail->tmem_full[a], aph, abort_flag);
       ptx::tc_fence_after_sync();
-      uint8_t* obuf = Os + (size_t)(it % n_out) * out_bytes;
+      uint8_t* obuf = Os;
       // All eight warps reach this barrier in every iteration, so the decision to stop is uniform.
-      // The staging buffer about to be overwritten must have been read: by its bulk copy, or, in the
-      // all-fp32 mode, by the row writer of the previous iteration (every warp is past it here).
-      if (leader) {
-        if (!ALL_F32) { if (n_out == 2) ptx::bulk_wait_read<1>(); else ptx::bulk_wait_read<0>(); }
-        tail->epi_go = *abort_flag ? 0 : 1;
-      }
+      // The staging buffer about to be overwritten has been read by the row writer of the previous
+      // iteration (every warp is past it here).
+      if (leader) tail->epi_go = *abort_flag ? 0 : 1;
       ptx::named_barrier_sync(1, kEpiWarps * 32);
       if (!tail->epi_go) break;
 
@@ -229,17 +198,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       ptx::tmem_ld_32x32(taddr, v0);
       ptx::tmem_ld_32x32(taddr + 32u, v1);
       ptx::tmem_wait_ld();
-      if (!ALL_F32) {
-        // 16-byte chunk c of row `row` (keys 8c .. 8c+7) sits at chunk position c ^ (row & 15)
-        uint8_t* orow = obuf + (size_t)row * (kTileKeys * 2);
-        const uint32_t swz = (uint32_t)row & 15u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-          *reinterpret_cast<uint4*>(orow + ((((uint32_t)(half * 8 + c)) ^ swz) << 4)) = keys8(&v0[8 * c], scale);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-          *reinterpret_cast<uint4*>(orow + ((((uint32_t)(half * 8 + 4 + c)) ^ swz) << 4)) = keys8(&v1[8 * c], scale);
-      } else {
+      {
         // fp32 staging: 16-byte chunk c of the row (keys 4c .. 4c+3) at chunk position c ^ (row & 31)
         uint8_t* orow = obuf + (size_t)row * (kTileKeys * 4);
         const uint32_t swz = (uint32_t)row & 31u;
@@ -251,8 +210,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
           *reinterpret_cast<float4*>(orow + ((((uint32_t)(half * 16 + 8 + c)) ^ swz) << 4)) = logits4(&v1[4 * c], scale);
       }
 
-      // ---- current-query rows (chunk 0 only): thread = key, exact fp32 logits and their running
-      // maximum for the softmax row A0 of Algorithm 1
+      // ---- current-query rows (chunk 0 only): thread = key, exact fp32 logits for the softmax row A0
       if (with_real && half == 0) {
         uint32_t w[16];
         ptx::tmem_ld_32x16(tmem_base + (uint32_t)(kD2Col + a * 32) + ((uint32_t)(q * 32) << 16), w);
@@ -264,8 +222,6 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
           if (i < G) {
             const float l = __uint_as_float(w[i]) * scale;
             if (valid) Lreq[((int64_t)(kh * G + i) * S1) * Ncap + n] = l;
-            const uint32_t wmax = __reduce_max_sync(0xffffffffu, valid ? ordered_key(l) : 0u);
-            if (lane == 0) atomicMax(&tail->rowmax[i], wmax);
           }
         }
       }
@@ -274,15 +230,7 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&tail->tmem_empty[a]);
-      if (!ALL_F32) {
-        ptx::fence_proxy_async();                // staged tile visible to the bulk-copy engine
-        ptx::named_barrier_sync(2, kEpiWarps * 32);
-        if (leader) {
-          uint16_t* gdst = keys16 + ((tile_base + (int64_t)t * row_chunks) * kRowChunk) * kTileKeys;
-          ptx::bulk_store(gdst, obuf, out_bytes);
-          ptx::bulk_commit();
-        }
-      } else {
+      {
         // write the staged fp32 rows out, one row per warp and step, 128 consecutive keys per row
         ptx::named_barrier_sync(2, kEpiWarps * 32);
         for (int rr = e; rr < kRowChunk; rr += kEpiWarps) {
@@ -300,7 +248,6 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
       }
     }
-    if (!ALL_F32 && leader) ptx::bulk_wait_all<0>();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -310,8 +257,6 @@ score_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
     atomicExch(&status[1], 2);
   }
-  if (with_real && rowmax != nullptr && (int)threadIdx.x < G && tail->rowmax[threadIdx.x] != 0)
-    atomicMax(&rowmax[r * Hq + kh * G + (int)threadIdx.x], tail->rowmax[threadIdx.x]);
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -333,19 +278,11 @@ ScoreGeometry score_geometry(const gvote_params* p) {
   return g;
 }
 
-size_t keys16_elems(const gvote_params* p, int32_t batch, int64_t total_tokens) {
-  if (!score_umma_supported(p)) return 0;
-  const ScoreGeometry g = score_geometry(p);
-  const int64_t n_tiles = (total_tokens >> 7) + batch;
-  return (size_t)p->n_kv_heads * n_tiles * g.row_chunks * g.RC * kTileKeys;
-}
-
 // Returns GVOTE_OK, or GVOTE_ERR_UNSUPPORTED_SHAPE when the tensor maps cannot describe the
 // operands (the caller then takes the SIMT path).
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                          bool all_f32, float* logits, uint16_t* keys16, uint32_t* rowmax, int32_t* status,
-                          const int32_t* kv_len, cudaStream_t st) {
+                          float* logits, int32_t* status, const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
   const ScoreGeometry geo = score_geometry(p);
   const int row_chunks = geo.row_chunks;
@@ -366,13 +303,12 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
     if (!encode_tensor_map_bf16(&tmQr, Q, 2, dims, strides, boxr)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   }
   const int kchunks = d_k / 64;
-  const size_t out_bytes = all_f32 ? (size_t)kRowChunk * kTileKeys * 4 : (size_t)kRowChunk * kTileKeys * 2;
+  const size_t out_bytes = (size_t)kRowChunk * kTileKeys * 4;
   const size_t fixed = 1024 + (size_t)kchunks * kRowChunk * 128 + align_up((size_t)kchunks * kRealCols * 128, 1024) +
                        sizeof(ScoreSmemTail) + 64;
   const size_t stage_bytes = (size_t)kchunks * kTileKeys * 128;
-  int stages = kMaxStages, n_out = all_f32 ? 1 : 2;
-  auto need = [&]() { return fixed + stages * stage_bytes + n_out * out_bytes; };
-  if (need() > 227 * 1024 && n_out == 2) n_out = 1;
+  int stages = kMaxStages;
+  auto need = [&]() { return fixed + stages * stage_bytes + out_bytes; };
   if (need() > 227 * 1024) stages = 2;
   if (need() > 227 * 1024) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   const size_t smem = need();
@@ -385,13 +321,11 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
   if (X < 1) X = 1;
   dim3 grid((unsigned)X, (unsigned)(Hkv * row_chunks), (unsigned)batch);
   const float scale = (float)(1.0 / sqrt((double)d_k));
-  const int64_t n_tiles_total = (total_tokens >> 7) + batch;
-  auto kern = all_f32 ? score_umma_kernel<true> : score_umma_kernel<false>;
-  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_umma_kernel", st);
-    kern<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, tmQr, cu, Hq, G, S1, d_k, row_chunks, stages, n_out, scale,
-                                           n_tiles_total, logits, keys16, rowmax, status, kv_len);
+    score_umma_kernel<<<grid, kUmmaThreads, smem, st>>>(tmK, tmQ, tmQr, cu, Hq, G, S1, d_k, row_chunks, stages, scale,
+                                                        logits, status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_umma_kernel");
   return GVOTE_OK;

@@ -112,9 +112,14 @@ __device__ void find_bin(SelShared& sh, int nbins, unsigned long long need) {
 // Outputs (same in every thread): t, number of keys above t, their mass (MASS only: mass above
 // in fixed point), number of keys equal to t.
 struct KeepAll { __device__ __forceinline__ bool operator()(float) const { return true; } };
+// A row of logits: anything that returns the logit of key n (stored values, or values computed on demand).
+struct StoredRow {
+  const float* p;
+  __device__ __forceinline__ float operator()(int n) const { return p[n]; }
+};
 
-template <bool MASS, typename Filter = KeepAll>
-__device__ void radix_threshold(const float* __restrict__ row, int N, float mx, unsigned long long need,
+template <bool MASS, typename Row, typename Filter = KeepAll>
+__device__ void radix_threshold(const Row& row, int N, float mx, unsigned long long need,
                                 SelShared& sh, uint32_t& t_out, uint32_t& above_cnt,
                                 unsigned long long& above_mass, uint32_t& eq_cnt, Filter keep = Filter()) {
   const int tid = threadIdx.x;
@@ -129,7 +134,7 @@ __device__ void radix_threshold(const float* __restrict__ row, int N, float mx, 
     for (int b = tid; b < nb; b += blockDim.x) { sh.cnt[b] = 0; if (MASS) sh.mass[b] = 0; }
     __syncthreads();
     for (int n = tid; n < N; n += blockDim.x) {
-      const float l = row[n];
+      const float l = row(n);
       const uint32_t key = ordered_key(l);
       if ((key & known_mask) == prefix && keep(l)) {
         const int b = (key >> shifts[pass]) & (nb - 1);
@@ -154,8 +159,9 @@ __device__ void radix_threshold(const float* __restrict__ row, int N, float mx, 
 }
 
 // OR the row's selection into the mask: keys above t, plus the first `ties` keys equal to t.
-__device__ inline void emit_row(const float* __restrict__ row, int N, uint32_t t, uint32_t ties, uint32_t eq_cnt,
-                         uint32_t* __restrict__ mask_row, SelShared& sh) {
+template <typename Row>
+__device__ inline void emit_row(const Row& row, int N, uint32_t t, uint32_t ties, uint32_t eq_cnt,
+                                uint32_t* __restrict__ mask_row, SelShared& sh) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool all_ties = ties >= eq_cnt;
   uint32_t taken = 0;   // ties taken so far (ordered path only)
@@ -163,7 +169,7 @@ __device__ inline void emit_row(const float* __restrict__ row, int N, uint32_t t
     const int n = base + tid;
     uint32_t key = 0;
     bool valid = n < N;
-    if (valid) key = ordered_key(row[n]);
+    if (valid) key = ordered_key(row(n));
     bool sel = valid && key > t;
     const bool tie = valid && key == t;
     if (all_ties) {

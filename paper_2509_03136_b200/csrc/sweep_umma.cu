@@ -356,9 +356,8 @@ template <int CG>
 __global__ void __launch_bounds__(kSweepThreads, 1)
 score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int row_chunks, int stages,
-                   float scale, const RowBracket* __restrict__ bracket, uint32_t* __restrict__ above,
-                   uint32_t* __restrict__ ncand, uint2* __restrict__ cand, int cap, uint32_t* __restrict__ tmask,
-                   int64_t row_words, int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
+                   float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
+                   const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int groups = (row_chunks + CG - 1) / CG;
   const int r = blockIdx.z;
@@ -428,21 +427,25 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     float lo[CG], hi[CG];
     uint32_t abv[CG];
     int rowid[CG];
+    uint2* list[CG];
+    const int cap = vs.lay.cap(Ncap);
 #pragma unroll
     for (int cc = 0; cc < CG; ++cc) {
       const int grow = (c_first + cc) * kRowChunk + q * 32 + lane;       // row within the head group
       abv[cc] = 0;
       rowid[cc] = -1;
+      list[cc] = nullptr;
       lo[cc] = INFINITY;
       hi[cc] = INFINITY;
       if (cc < c_cnt && grow < G * S) {
         rowid[cc] = (r * Hq + kh * G + grow / S) * S + grow % S;
-        const RowBracket b = bracket[rowid[cc]];
+        list[cc] = vs.list(kh * G + grow / S, grow % S, S, start, r);
+        const RowBracket b = vs.bracket[rowid[cc]];
         lo[cc] = b.lo;
         hi[cc] = b.hi;
       }
     }
-    uint32_t* mrow = tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
+    uint32_t* mrow = vs.tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
     int n1 = 0;
     for (int it = 0; it < walk.count; ++it) {
       const int t = walk.tile(it);
@@ -488,19 +491,19 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         abv[cc] += __popc(ab0) + __popc(ab1);
         const uint32_t cnt = __popc(cb0) + __popc(cb1);
         if (cnt) {
-          uint32_t slot = atomicAdd(&ncand[rowid[cc]], cnt);
-          uint2* list = cand + (int64_t)rowid[cc] * cap;
+          uint32_t slot = atomicAdd(&vs.ncand[rowid[cc]], cnt);
+          uint2* const lst = list[cc];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             if ((cb0 >> i) & 1u) {
-              if (slot < (uint32_t)cap) list[slot] = make_uint2(__float_as_uint(__uint_as_float(v0[i]) * scale), (uint32_t)(n0 + i));
+              if (slot < (uint32_t)cap) lst[slot] = make_uint2(__float_as_uint(__uint_as_float(v0[i]) * scale), (uint32_t)(n0 + i));
               ++slot;
             }
           }
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             if ((cb1 >> i) & 1u) {
-              if (slot < (uint32_t)cap) list[slot] = make_uint2(__float_as_uint(__uint_as_float(v1[i]) * scale), (uint32_t)(n0 + 32 + i));
+              if (slot < (uint32_t)cap) lst[slot] = make_uint2(__float_as_uint(__uint_as_float(v1[i]) * scale), (uint32_t)(n0 + 32 + i));
               ++slot;
             }
           }
@@ -509,7 +512,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     }
 #pragma unroll
     for (int cc = 0; cc < CG; ++cc)
-      if (rowid[cc] >= 0 && abv[cc]) atomicAdd(&above[rowid[cc]], abv[cc]);
+      if (rowid[cc] >= 0 && abv[cc]) atomicAdd(&vs.above[rowid[cc]], abv[cc]);
   }
 
   ptx::tc_fence_before_sync();
@@ -636,8 +639,8 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sweep_kernel", st);
-    kern<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, stages, scale, vs.bracket,
-                                            vs.above, vs.ncand, vs.cand, vs.cap, vs.tmask, row_words, status, kv_len);
+    kern<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, stages, scale, vs, row_words,
+                                            status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_sweep_kernel");
   return GVOTE_OK;

@@ -116,7 +116,7 @@ __device__ __forceinline__ void block_scan_pair(uint32_t c, unsigned long long m
 }
 
 __global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kThreads)
-real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G, int S1,
+real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G,
                  const uint32_t* __restrict__ rowmax, float p_nuc, int include_c0, int64_t row_words,
                  uint32_t* __restrict__ mask, int32_t* __restrict__ b_step, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint8_t dyn[];
@@ -136,7 +136,7 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
     if (crank == 0 && tid == 0) b_step[r * Hq + g] = 0;
     return;
   }
-  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1) * Ncap;
+  const float* L = logits + (int64_t)Hq * start + (int64_t)g * Ncap;       // [n_q_heads][N] per request
   const float mx = key_to_float(rowmax[r * Hq + g]);
   const float cut = tail_cut(N, p_nuc);
   const int per = (N + kClusterCtas - 1) / kClusterCtas;
@@ -368,7 +368,7 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
     uint32_t a_cnt;
     unsigned long long a_mass;
     InBin keep{mx, cut, bstar};
-    radix_threshold<true>(L, N, mx, lack, sh, t_key, a_cnt, a_mass, eq_cnt, keep);
+    radix_threshold<true>(StoredRow{L}, N, mx, lack, sh, t_key, a_cnt, a_mass, eq_cnt, keep);
     const unsigned long long e_t = mass_fix(key_to_float(t_key), mx);
     ties = eq_cnt;
     if (e_t > 0) {
@@ -381,24 +381,16 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
     if (!include_c0) return;
   }
   uint32_t* mrow = mask + (int64_t)(g / G) * row_words + mask_word_offset(start, r);
-  emit_row(L, N, t_key, ties, eq_cnt, mrow, sh);
+  emit_row(StoredRow{L}, N, t_key, ties, eq_cnt, mrow, sh);
 }
 
 }  // namespace
 
-size_t real_topp_scratch_bytes(const gvote_params* p, int32_t batch) {
-  return align_up((size_t)batch * p->n_q_heads * sizeof(uint32_t), 256);
-}
-
-// The row maxima live in `scratch` (real_topp_scratch_bytes), zeroed by the caller before the score
-// kernel runs (its read-out fills them with atomicMax).
-uint32_t* real_topp_rowmax(char* scratch) { return reinterpret_cast<uint32_t*>(scratch); }
-
+// `rowmax` [batch][n_q_heads]: the row maxima (order-preserving images) the first pass of the vote leaves.
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, const int32_t* kv_len,
-                         cudaStream_t st) {
-  const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads, S1 = p->S + 1;
-  const uint32_t* rowmax = reinterpret_cast<const uint32_t*>(scratch);
+                         const uint32_t* rowmax, int64_t row_words, uint32_t* mask, int32_t* b_step,
+                         const int32_t* kv_len, cudaStream_t st) {
+  const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   (void)max_N;
   static_assert(kBins == 2 * kThreads && kSubBins == kThreads && kRankCap == kThreads, "bins per thread");
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(real_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -406,7 +398,7 @@ int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32
   dim3 grid((unsigned)kClusterCtas, (unsigned)Hq, (unsigned)batch);
   {
     LaunchScope scope_("real_topp_kernel", st);
-    real_topp_kernel<<<grid, kThreads, sizeof(ClusterShared), st>>>(logits, cu, Hq, G, S1, rowmax, p->p_nuc,
+    real_topp_kernel<<<grid, kThreads, sizeof(ClusterShared), st>>>(logits, cu, Hq, G, rowmax, p->p_nuc,
                                                                     p->include_c0, row_words, mask, b_step, kv_len);
   }
   GVOTE_LAUNCH_CHECK("real_topp_kernel");

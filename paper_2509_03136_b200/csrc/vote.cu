@@ -11,6 +11,7 @@
 // warp ballot per 32 keys OR-ed into the mask word.
 #include "common.cuh"
 #include "select_common.cuh"
+#include "vote_geom.cuh"
 
 namespace gvote {
 namespace {
@@ -107,7 +108,7 @@ topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
   // the row is staged in shared memory when it fits (eight loads in flight per thread), so the
   // passes below do not wait on global memory; the running maximum is taken on the way in
   const bool fits = N <= row_elems;
-  const float* L = fits ? row_sm : Lg;
+  const StoredRow L{fits ? row_sm : Lg};
   float mx = -INFINITY;
   for (int base = 0; base < N; base += nthr * 8) {
     float v[8];
@@ -125,7 +126,7 @@ topp_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
   }
   mx = block_max(mx, sh.redf);      // (its barriers also publish the staged row)
   unsigned long long z = 0;
-  for (int n = tid; n < N; n += nthr) z += mass_fix(L[n], mx);
+  for (int n = tid; n < N; n += nthr) z += mass_fix(L(n), mx);
   z = block_sum_u64(z, sh.red64);
   // smallest integer mass that is >= p * Z
   unsigned long long need = (unsigned long long)ceil((double)p_nuc * (double)z);
@@ -171,7 +172,7 @@ topk_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
   int k = b_step[r * Hq + g];
   if (k <= 0) return;
   if (k > N) k = N;
-  const float* L = logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * Ncap;
+  const StoredRow L{logits + (int64_t)Hq * S1 * start + ((int64_t)g * S1 + row) * Ncap};
   uint32_t t, above_cnt, eq_cnt;
   unsigned long long above_mass;
   radix_threshold<false>(L, N, 0.f, (unsigned long long)k, sh, t, above_cnt, above_mass, eq_cnt);
@@ -224,39 +225,104 @@ budget_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu,
 }  // namespace
 
 bool score_umma_supported(const gvote_params* p);
-int32_t launch_topk16(const gvote_params* p, const uint16_t* keys16, const __nv_bfloat16* Q, const __nv_bfloat16* K,
-                      int64_t k_tok, int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens,
-                      int64_t max_N, const int32_t* b_step, int64_t row_words, uint32_t* mask, const int32_t* kv_len,
-                      cudaStream_t st);
 int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                          bool all_f32, float* logits, uint16_t* keys16, uint32_t* rowmax, int32_t* status,
-                          const int32_t* kv_len, cudaStream_t st);
-uint32_t* real_topp_rowmax(char* scratch);
+                          float* logits, int32_t* status, const int32_t* kv_len, cudaStream_t st);
+int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                            int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                            float* real_logits, uint32_t* rowmax, const VoteState& vs, int32_t* status,
+                            const int32_t* kv_len, cudaStream_t st);
+int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
+                           int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
+                           const VoteState& vs, int64_t row_words, int32_t* status, const int32_t* kv_len,
+                           cudaStream_t st);
+int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs,
+                       const int32_t* kv_len, cudaStream_t st);
+int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, int64_t max_N, const int32_t* b_step,
+                       const VoteState& vs, int64_t row_words, const int32_t* kv_len, cudaStream_t st);
+int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
+                      const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs, int64_t row_words,
+                      uint32_t* mask, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         char* scratch, int64_t row_words, uint32_t* mask, int32_t* b_step, const int32_t* kv_len,
-                         cudaStream_t st);
+                         const uint32_t* rowmax, int64_t row_words, uint32_t* mask, int32_t* b_step,
+                         const int32_t* kv_len, cudaStream_t st);
+
+namespace {
+
+int32_t launch_budget(const gvote_params* p, const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t row_words,
+                      int32_t* budget, cudaStream_t st) {
+  dim3 gb(p->n_kv_heads, batch);
+  {
+    LaunchScope scope_("budget_kernel", st);
+    budget_kernel<<<gb, 256, 0, st>>>(mask, cu, p->n_kv_heads, row_words, budget);
+  }
+  GVOTE_LAUNCH_CHECK("budget_kernel");
+  return GVOTE_OK;
+}
+
+// The default route: current-query top-p and the fused top-k of the synthetic queries on the tensor
+// cores; nothing of size S x N is written anywhere.  GVOTE_ERR_UNSUPPORTED_SHAPE (before anything has been
+// enqueued) when no tensor map describes the operands.
+int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
+                   const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N, uint32_t* mask,
+                   int32_t* b_step, const WorkspaceMap& m, char* ws, cudaStream_t st, const int32_t* kv_len) {
+  VoteState vs;
+  vs.sample = reinterpret_cast<uint16_t*>(ws + m.sample);
+  vs.bracket = reinterpret_cast<RowBracket*>(ws + m.bracket);
+  vs.above = reinterpret_cast<uint32_t*>(ws + m.above);
+  vs.ncand = reinterpret_cast<uint32_t*>(ws + m.ncand);
+  vs.cand = reinterpret_cast<uint2*>(ws + m.cand);
+  vs.tmask = reinterpret_cast<uint32_t*>(ws + m.tmask);
+  vs.head_bad = reinterpret_cast<uint32_t*>(ws + m.head_bad);
+  vs.lay = cand_layout(batch, total_tokens, max_N);
+  vs.sample_slots = m.sample_slots;
+  float* real_logits = reinterpret_cast<float*>(ws + m.logits);
+  uint32_t* rowmax = reinterpret_cast<uint32_t*>(ws + m.rowmax);
+  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
+  // tentative mask, per-head flags and row maxima start from zero
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(ws + m.vote_zero, 0, m.vote_zero_bytes, st));
+  const int32_t rc = launch_score_sample(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, real_logits, rowmax, vs,
+                                         status, kv_len, st);
+  if (rc != GVOTE_OK) return rc;
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(mask, 0, (size_t)p->n_kv_heads * m.row_words * sizeof(uint32_t), st));
+#define GVOTE_STEP(expr) do { const int32_t rc__ = (expr); if (rc__ != GVOTE_OK) return rc__; } while (0)
+  GVOTE_STEP(launch_real_topp(p, real_logits, cu, batch, max_N, rowmax, m.row_words, mask, b_step, kv_len, st));
+  GVOTE_STEP(launch_bracket(p, cu, batch, b_step, vs, kv_len, st));
+  GVOTE_STEP(launch_score_sweep(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, vs, m.row_words, status, kv_len,
+                                st));
+  GVOTE_STEP(launch_resolve(p, cu, batch, max_N, b_step, vs, m.row_words, kv_len, st));
+  GVOTE_STEP(launch_commit(p, Q, K, k_tok, k_head, cu, batch, b_step, vs, m.row_words, mask, kv_len, st));
+#undef GVOTE_STEP
+  return GVOTE_OK;
+}
+
+}  // namespace
 
 int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                    uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs, const WorkspaceMap& m,
-                    char* ws, cudaStream_t st, const int32_t* kv_len) {
+                    uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs, char* ws, size_t ws_bytes,
+                    cudaStream_t st, const int32_t* kv_len) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
-  float* logits = reinterpret_cast<float*>(ws + m.logits);
-  uint16_t* keys16 = reinterpret_cast<uint16_t*>(ws + m.keys16);
-  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
   const float scale = (float)(1.0 / sqrt((double)d_k));
-  GVOTE_CUDA_CHECK(cudaMemsetAsync(mask, 0, (size_t)Hkv * m.row_words * sizeof(uint32_t), st));
 
-  // fp32 rows for every query are needed by the per-sample top-p mode and by the softmax dump;
-  // the default mode keeps fp32 only for the current query's rows and 16-bit keys for the rest
-  const bool all_f32 = (p->sel_mode != GVOTE_SEL_TOPK_C0) || dbg_probs != nullptr;
+  if (!vote_needs_full_rows(p) && dbg_probs == nullptr && max_N > 0) {
+    const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N, false);
+    const int32_t rc = vote_fused(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, mask, b_step, m, ws, st, kv_len);
+    if (rc == GVOTE_OK) return budget ? launch_budget(p, mask, cu, batch, m.row_words, budget, st) : GVOTE_OK;
+    if (rc != GVOTE_ERR_UNSUPPORTED_SHAPE) return rc;
+    // operands no tensor map describes: the route below, if the workspace has room for its fp32 rows
+  }
+
+  // fp32 logits of every row: the per-sample top-p mode, the softmax dump, shapes the tensor-core kernels
+  // do not take.  On the tensor cores when possible, else SIMT.
+  const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N, true);
+  if (ws_bytes < m.total) return vote_needs_full_rows(p) || dbg_probs ? GVOTE_ERR_WORKSPACE_TOO_SMALL : GVOTE_ERR_UNSUPPORTED_SHAPE;
+  float* logits = reinterpret_cast<float*>(ws + m.logits);
+  int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(mask, 0, (size_t)Hkv * m.row_words * sizeof(uint32_t), st));
   bool tensor_path = false;
   if (score_umma_supported(p) && max_N > 0) {
-    // row maxima and mass histograms of the current-query rows start from zero
-    if (!all_f32) GVOTE_CUDA_CHECK(cudaMemsetAsync(ws + m.real_scratch, 0, m.real_scratch_bytes, st));
-    const int32_t rc = launch_score_umma(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, all_f32, logits,
-                                         keys16, real_topp_rowmax(ws + m.real_scratch), status, kv_len, st);
+    const int32_t rc = launch_score_umma(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, logits, status, kv_len, st);
     if (rc == GVOTE_OK) tensor_path = true;
     else if (rc != GVOTE_ERR_UNSUPPORTED_SHAPE) return rc;
   }
@@ -287,50 +353,23 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
   const size_t topp_smem = (size_t)topp_row_elems * sizeof(float);
   if (topp_smem > 16 * 1024)
     GVOTE_CUDA_CHECK(cudaFuncSetAttribute(topp_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topp_smem));
-  if (p->sel_mode == GVOTE_SEL_TOPK_C0) {
-    if (tensor_path && !all_f32) {
-      const int32_t rc = launch_real_topp(p, logits, cu, batch, max_N, ws + m.real_scratch, m.row_words, mask, b_step,
-                                          kv_len, st);
-      if (rc != GVOTE_OK) return rc;
-    } else {
-      dim3 g1(1, Hq, batch);
-      {
-        LaunchScope scope_("topp_rows_kernel", st);
-        topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, 1, p->p_nuc, p->include_c0,
-                                                              m.row_words, mask, b_step, topp_row_elems, kv_len);
-      }
-      GVOTE_LAUNCH_CHECK("topp_rows_kernel");
-    }
+  const bool topk = p->sel_mode == GVOTE_SEL_TOPK_C0;
+  dim3 g1(topk ? 1 : S1, Hq, batch);
+  {
+    LaunchScope scope_("topp_rows_kernel", st);
+    topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, topk ? 1 : S1, p->p_nuc, p->include_c0,
+                                                          m.row_words, mask, b_step, topp_row_elems, kv_len);
+  }
+  GVOTE_LAUNCH_CHECK("topp_rows_kernel");
+  if (topk) {
     dim3 g2(p->S, Hq, batch);
-    if (tensor_path && !all_f32) {
-      const int32_t rc = launch_topk16(p, keys16, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, b_step,
-                                       m.row_words, mask, kv_len, st);
-      if (rc != GVOTE_OK) return rc;
-    } else {
-      {
-        LaunchScope scope_("topk_rows_kernel", st);
-        topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask, kv_len);
-      }
-      GVOTE_LAUNCH_CHECK("topk_rows_kernel");
-    }
-  } else {
-    dim3 g1(S1, Hq, batch);
     {
-      LaunchScope scope_("topp_rows_kernel", st);
-      topp_rows_kernel<<<g1, kToppThreads, topp_smem, st>>>(logits, cu, Hq, G, S1, S1, p->p_nuc, p->include_c0,
-                                                            m.row_words, mask, b_step, topp_row_elems, kv_len);
+      LaunchScope scope_("topk_rows_kernel", st);
+      topk_rows_kernel<<<g2, kSelThreads, 0, st>>>(logits, cu, Hq, G, S1, b_step, m.row_words, mask, kv_len);
     }
-    GVOTE_LAUNCH_CHECK("topp_rows_kernel");
+    GVOTE_LAUNCH_CHECK("topk_rows_kernel");
   }
-  if (budget) {
-    dim3 gb(Hkv, batch);
-    {
-      LaunchScope scope_("budget_kernel", st);
-      budget_kernel<<<gb, 256, 0, st>>>(mask, cu, Hkv, m.row_words, budget);
-    }
-    GVOTE_LAUNCH_CHECK("budget_kernel");
-  }
-  return GVOTE_OK;
+  return budget ? launch_budget(p, mask, cu, batch, m.row_words, budget, st) : GVOTE_OK;
 }
 
 }  // namespace gvote

@@ -54,25 +54,50 @@ __host__ __device__ __forceinline__ int sample_keys(const SampleGeom& g, int N) 
   return g.whole ? N : g.ns * kVoteTileKeys;
 }
 // First sample-tile slot of request r in the sample buffer, and the slots a batch needs: a request of
-// N keys takes at most 32 + N / 1024 + 1 slots.
+// N keys takes at most 32 + N / 1024 + 1 slots (closed forms: no kernel has to add up the requests before
+// its own).  A single request takes exactly its own.
 __host__ __device__ __forceinline__ int64_t sample_slot_offset(int cu_r, int r) { return (int64_t)34 * r + (cu_r >> 10); }
-inline int64_t sample_slots_total(int32_t batch, int64_t total_tokens) { return (int64_t)34 * batch + (total_tokens >> 10) + 1; }
+inline int64_t sample_slots_total(int32_t batch, int64_t total_tokens, int64_t max_N) {
+  if (batch == 1) return sample_geom((int)max_N).ns > 0 ? sample_geom((int)max_N).ns : 1;
+  return (int64_t)34 * batch + (total_tokens >> 10) + 1;
+}
 
-// Entries a row's candidate list holds.  The bracket spans 2 * (4.5 sqrt(m f (1 - f)) + 6) of the m
+// Entries a row's candidate list needs.  The bracket spans 2 * (4.5 sqrt(m f (1 - f)) + 6) of the m
 // sampled keys' ranks, at most 4.5 sqrt(m) + 12, i.e. that many times N / m keys of the row; a quarter
 // more covers the spread of the count.  A completely sampled row lists only the keys that share the
 // threshold's 16-bit value or its neighbours'.
-inline int candidate_cap(int64_t max_N) {
-  if (max_N <= 0) return 256;
-  const SampleGeom g = sample_geom((int)max_N);
+inline int candidate_need(int64_t N) {
+  if (N <= 0) return 256;
+  const SampleGeom g = sample_geom((int)N);
   double need = 512.0;
   if (!g.whole) {
     const double m = (double)g.ns * kVoteTileKeys;
-    need = 1.25 * (4.5 * sqrt(m) + 12.0) * ((double)max_N / m) + 256.0;
+    need = 1.25 * (4.5 * sqrt(m) + 12.0) * ((double)N / m) + 256.0;
   }
-  int cap = 1024;
-  while (cap < need) cap += 1024;
-  return cap;
+  return ((int)need + 255) & ~255;
+}
+// Where the lists live: row (g, s) of the batch owns a strip of `strip` entries, request r's list starts
+// at entry cand_offset(r) of the strip and holds cand_cap(N_r) entries.  A single request gets exactly
+// candidate_need(N); in a batch the capacity is the line 512 + 3 N / 32, which lies above candidate_need
+// for every N and has a closed-form running sum over the requests.
+struct CandLayout {
+  int uniform_cap;       // > 0: one request, this capacity
+  int64_t strip;
+  __host__ __device__ __forceinline__ int cap(int N) const { return uniform_cap > 0 ? uniform_cap : 512 + (int)((3 * (int64_t)N) >> 5); }
+  __host__ __device__ __forceinline__ int64_t offset(int cu_r, int r) const {
+    return uniform_cap > 0 ? 0 : (int64_t)576 * r + ((3 * (int64_t)cu_r) >> 5);
+  }
+};
+inline CandLayout cand_layout(int32_t batch, int64_t total_tokens, int64_t max_N) {
+  CandLayout c;
+  if (batch == 1) {
+    c.uniform_cap = candidate_need(max_N);
+    c.strip = c.uniform_cap;
+  } else {
+    c.uniform_cap = 0;
+    c.strip = (int64_t)576 * batch + ((3 * total_tokens) >> 5) + 1;
+  }
+  return c;
 }
 
 struct RowBracket { float lo, hi; };    // keys above hi are taken, keys in [lo, hi] are listed
@@ -83,11 +108,15 @@ struct VoteState {
   RowBracket* bracket;     // [rows]
   uint32_t* above;         // [rows] keys above the bracket (counted by the sweep)
   uint32_t* ncand;         // [rows] keys inside the bracket (listed by the sweep, up to `cap`)
-  uint2* cand;             // [rows][cap] (fp32 logit bits, key index)
+  uint2* cand;             // [n_q_heads * S][strip] (fp32 logit bits, key index), see CandLayout
+  CandLayout lay;
   uint32_t* tmask;         // [n_kv_heads][row_words] the union while it is tentative
   uint32_t* head_bad;      // [batch][n_kv_heads] a bracket of the head missed: redo the head exactly
-  int cap;
   int64_t sample_slots;
+  // the list of row (g, s) of request r
+  __host__ __device__ __forceinline__ uint2* list(int g, int s, int S, int cu_r, int r) const {
+    return cand + (int64_t)(g * S + s) * lay.strip + lay.offset(cu_r, r);
+  }
 };
 
 #ifdef __CUDACC__

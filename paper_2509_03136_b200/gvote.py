@@ -169,7 +169,15 @@ def gvote_workspace_bytes(p: GVoteParams, batch: int, total_tokens: int, max_N: 
     return int(load().gvote_workspace_bytes(ctypes.byref(p), batch, total_tokens, max_N))
 
 
-def alloc_workspace(p: GVoteParams, batch: int, total_tokens: int, max_N: int, device="cuda") -> torch.Tensor:
+def alloc_workspace(p: GVoteParams, batch: int, total_tokens: int, max_N: int, device="cuda",
+                    softmax_dump: bool = False) -> torch.Tensor:
+    """A zero-filled workspace for these parameters.  softmax_dump=True sizes it for calls that ask
+    gvote_vote / gvote_select for the softmax rows (dbg_probs): those keep the fp32 logits of every row,
+    like the per-sample top-p mode, so the size is that mode's."""
+    if softmax_dump and p.sel_mode != SEL_TOPP:
+        q = GVoteParams.from_buffer_copy(p)
+        q.sel_mode = SEL_TOPP
+        p = q
     n = gvote_workspace_bytes(p, batch, total_tokens, max_N)
     if n == 0:
         raise GVoteError(-1, "gvote_workspace_bytes")

@@ -56,6 +56,26 @@ def test_workspace_bytes(gv):
     assert gv.gvote_workspace_bytes(_params(gv, d_k=36), 1, 512, 512) == 0
 
 
+def test_workspace_of_the_default_mode_holds_no_logits_matrix(gv):
+    """Section 4.4 names the S x N logits matrix as what runs out of memory beyond 128K.  The default
+    (top-k) mode keeps none: its workspace stays far below S x N fp32 values at the long-context
+    shapes, and below the per-sample top-p mode's, which does keep fp32 rows."""
+    shapes = {"c2": dict(d_h=4096, n_q_heads=32, n_kv_heads=8, d_k=128, S=32, N=32768),
+              "c4": dict(d_h=3584, n_q_heads=28, n_kv_heads=4, d_k=128, S=64, N=131072)}
+    for name, sh in shapes.items():
+        N = sh.pop("N")
+        kw = dict(rope_theta=1e6, p_nuc=0.95, n_f=128, n_s=4, seed=0)
+        topk = gv.gvote_workspace_bytes(gv.make_params(sel_mode=gv.SEL_TOPK_C0, **sh, **kw), 1, N, N)
+        topp = gv.gvote_workspace_bytes(gv.make_params(sel_mode=gv.SEL_TOPP, **sh, **kw), 1, N, N)
+        matrix = sh["n_q_heads"] * sh["S"] * N * 4
+        assert topp > matrix                    # every row as fp32
+        assert topk < matrix / 2.5 and topk < topp / 2.5, (name, topk, topp, matrix)
+    # doubling S doubles the per-row state, not an S x N area: the growth stays a small part of S x N x 4
+    a = gv.gvote_workspace_bytes(gv.make_params(sel_mode=0, d_h=4096, n_q_heads=32, n_kv_heads=8, d_k=128, S=32, **kw), 1, 32768, 32768)
+    b = gv.gvote_workspace_bytes(gv.make_params(sel_mode=0, d_h=4096, n_q_heads=32, n_kv_heads=8, d_k=128, S=64, **kw), 1, 32768, 32768)
+    assert (b - a) < 0.35 * (32 * 32 * 32768 * 4)
+
+
 def test_mask_geometry_never_overlaps(gv):
     import numpy as np
     rng = np.random.default_rng(0)

@@ -154,7 +154,7 @@ def _run_vote(gv, cfg, li, Q_or, sel_mode, include_c0, want_probs):
     p = gv.params_from_config(cfg, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0,
                               include_c0=include_c0)
     geom = _geom(cfg)
-    ws = gv.alloc_workspace(p, *geom)
+    ws = gv.alloc_workspace(p, *geom, softmax_dump=want_probs)
     K = gv.bf16_from_bits(li.K)
     cu = torch.from_numpy(li.cu_seqlens).cuda()
     Qgm = np.ascontiguousarray(np.stack([pu.to_group_major(q, cfg.G) for q in Q_or]))
@@ -211,22 +211,26 @@ def _check_vote(gv, cfg, li, sel_mode, include_c0=False, want_probs=True):
             assert np.all(last >> np.uint32(N % 32) == 0)
 
 
+# "topk" asks for the softmax rows too, which takes the route that keeps fp32 logits of every row;
+# "topk-fused" is the default route (no S x N logits anywhere), as the whole pass runs it
 @pytest.mark.parametrize("idx", range(4))
-@pytest.mark.parametrize("mode", ["topk", "topp"])
+@pytest.mark.parametrize("mode", ["topk", "topk-fused", "topp"])
 def test_vote_small(gv, idx, mode):
     cfg = _small_cfgs()[idx]
-    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode.split("-")[0], want_probs=not mode.endswith("fused"))
 
 
-def test_vote_include_c0(gv):
+@pytest.mark.parametrize("probs", [True, False])
+def test_vote_include_c0(gv, probs):
     cfg = _small_cfgs()[2]
-    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", include_c0=True)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", include_c0=True, want_probs=probs)
 
 
-@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c1", "topp")])
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topk-fused"), ("c0", "topp"), ("c1", "topk"),
+                                       ("c1", "topk-fused"), ("c1", "topp"), ("c3", "topk-fused")])
 def test_vote_configs(gv, name, mode):
     cfg = synth.make_config(name)
-    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), mode.split("-")[0], want_probs=not mode.endswith("fused"))
 
 
 def test_vote_many_row_chunks_strict_band(gv):
