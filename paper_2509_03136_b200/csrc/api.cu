@@ -102,7 +102,8 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
   m.logits = take((size_t)p->n_q_heads * (full_rows ? S1 : 1) * (size_t)total_tokens * sizeof(float));
   if (!full_rows) {
     const size_t rows = (size_t)batch * p->n_q_heads * p->S;
-    m.cand_strip = cand_layout(batch, total_tokens, max_N).strip;
+    m.cand_segs = 4 * sweep_geometry(p, batch, max_N).X;
+    m.cand_strip = cand_layout(m.cand_segs, batch, total_tokens, max_N).strip;
     m.sample_slots = sample_slots_total(batch, total_tokens, max_N);
     m.vote_zero = off;
     m.tmask = take((size_t)p->n_kv_heads * m.row_words * sizeof(uint32_t));
@@ -112,8 +113,7 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
     m.sample = take((size_t)p->n_kv_heads * m.sample_slots * score_geometry(p).row_chunks * kVoteRowChunk *
                     kVoteTileKeys * sizeof(uint16_t));
     m.bracket = take(rows * sizeof(RowBracket));
-    m.above = take(rows * sizeof(uint32_t));
-    m.ncand = take(rows * sizeof(uint32_t));
+    m.segstat = take(rows * (size_t)m.cand_segs * sizeof(uint2));
     m.cand = take((size_t)p->n_q_heads * p->S * (size_t)m.cand_strip * sizeof(uint2));
   }
   m.remap_tmp = take((size_t)p->n_kv_heads * (size_t)total_tokens * sizeof(int32_t));

@@ -77,9 +77,10 @@ struct WorkspaceMap {
   size_t rowmax;        // uint32 [batch][Hq]  row maxima of the current-query rows (topp_real.cu)
   size_t sample;        // uint16 [Hkv][sample_slots][row_chunks][128][128]
   size_t bracket;       // RowBracket [batch*Hq*S]
-  size_t above, ncand;  // uint32 [batch*Hq*S] each
+  size_t segstat;       // uint2 [batch*Hq*S][cand_segs]
   size_t cand;          // uint2 [Hq*S][cand_strip]
   int64_t cand_strip;
+  int cand_segs;
   int64_t sample_slots;
   size_t remap_tmp;     // int32 [Hkv][total_tokens]  scratch of the slot -> position map's gather
   size_t ov_partial;    // float4 [batch][Hq][ceil(max_N / kOverlapKeys)]  partial sums of gvote_overlap

@@ -25,72 +25,76 @@ namespace {
 
 using namespace sel;
 
-constexpr int kRowThreads = 256;
-
 // Half bits <-> 16-bit code whose unsigned order is the numeric order.
 __device__ __forceinline__ uint32_t raw_of_code(uint32_t c) { return (c & 0x8000u) ? (c & 0x7fffu) : (~c & 0xffffu); }
 __device__ __forceinline__ float float_of_code(uint32_t c) {
   return __half2float(__ushort_as_half((unsigned short)raw_of_code(c)));
 }
 
-// Sum of one value per thread over the CTA.  `red` holds two rows of one slot per warp, used alternately,
-// so that consecutive sums need one barrier each.
-struct BlockSum {
-  uint32_t* red;    // [2][kRowThreads / 32]
-  int flip;
-  __device__ __forceinline__ uint32_t operator()(uint32_t v) {
-    v = (uint32_t)warp_sum_i((int)v);
-    uint32_t* row = red + flip * (kRowThreads / 32);
-    flip ^= 1;
-    if ((threadIdx.x & 31) == 0) row[threadIdx.x >> 5] = v;
-    __syncthreads();
-    uint32_t s = 0;
-#pragma unroll
-    for (int w = 0; w < kRowThreads / 32; ++w) s += row[w];
-    return s;
-  }
-  __device__ __forceinline__ void sum2(uint32_t a, uint32_t b, uint32_t& sa, uint32_t& sb) {
-    a = (uint32_t)warp_sum_i((int)a);
-    b = (uint32_t)warp_sum_i((int)b);
-    uint32_t* row = red + flip * (kRowThreads / 32);
-    flip ^= 1;
-    if ((threadIdx.x & 31) == 0) row[threadIdx.x >> 5] = (a << 16) | b;      // both counts are below 2^16
-    __syncthreads();
-    sa = 0;
-    sb = 0;
-#pragma unroll
-    for (int w = 0; w < kRowThreads / 32; ++w) { sa += row[w] >> 16; sb += row[w] & 0xffffu; }
-  }
-};
-
-// ------------------------------------------------------------------------------------ bracket
-constexpr int kBrVecs = 8;      // 16-byte vectors of sampled keys per thread: 256 * 8 * 8 = 16384 keys at most
-
-__device__ __forceinline__ uint32_t count_ge(const uint4 (&v)[kBrVecs], uint32_t raw) {
-  const uint32_t p = raw | (raw << 16);
-  const __half2 th = *reinterpret_cast<const __half2*>(&p);
+// Largest bin b of hist[0..256) whose suffix count reaches `need` (need >= 1, total >= need), found by
+// one warp: every lane returns the bin and the count in the bins above it.
+__device__ __forceinline__ void warp_find_bin256(const uint32_t* hist, uint32_t need, int lane, int& bin,
+                                                 uint32_t& above) {
   uint32_t c = 0;
 #pragma unroll
-  for (int u = 0; u < kBrVecs; ++u) {
-    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+  for (int i = 0; i < 8; ++i) c += hist[lane * 8 + i];
+  uint32_t cs = c;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) c += __popc(__hge2_mask(*reinterpret_cast<const __half2*>(&w[j]), th));
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_down_sync(0xffffffffu, cs, o);
+    if (lane + o < 32) cs += t;
   }
-  return c >> 4;
+  const uint32_t excl = cs - c;                          // count in the lanes above this one
+  const bool own = excl < need && excl + c >= need;
+  uint32_t a = excl;
+  int b = lane * 8 + 7;
+  if (own) {
+    for (; b > lane * 8; --b) {
+      if (a + hist[b] >= need) break;
+      a += hist[b];
+    }
+  }
+  const uint32_t who = __ballot_sync(0xffffffffu, own);
+  const int src = who ? __ffs(who) - 1 : 0;
+  bin = who ? __shfl_sync(0xffffffffu, b, src) : 0;
+  above = who ? __shfl_sync(0xffffffffu, a, src) : 0u;
 }
 
-__global__ void __launch_bounds__(kRowThreads)
+// ------------------------------------------------------------------------------------ bracket
+// Two order statistics of a row's sampled keys (at most 16384 half-precision values, held in registers)
+// by a two-level radix search over their 16-bit order-preserving codes, both ranks at a time.
+// Level 1 bins the high byte.  Every sampled key takes part and a few bins take most of them, so plain
+// shared-memory atomics would queue on those addresses: counting goes into one 16-bit counter per (bin,
+// lane) instead, two bins to a word, word (bin / 2) * 32 + lane - the lanes of a warp never meet, and a
+// counter takes at most (4 warps) x (128 keys per thread) increments.  Bins are those of the raw half bits
+// (no recoding per key); the fold over the lanes puts them in code order.  Level 2 bins the low byte of
+// the keys whose high byte is the one found, for the two ranks side by side.  Integer counts only: the
+// same bits on every run.
+constexpr int kBrThreads = 128;
+constexpr int kBrVecs = 16;     // 16-byte vectors of sampled keys per thread: 128 * 16 * 8 = 16384 keys at most
+
+// High byte of a key's code from the high byte hb of its half bits.
+__device__ __forceinline__ uint32_t ord_hi(uint32_t hb) { return hb >= 0x80u ? 0xffu - hb : 0x80u + hb; }
+
+struct BracketShared {
+  uint32_t lanes[128 * 32];     // level 1: 16-bit counters per (raw high byte, lane)
+  uint32_t bins[256];           // level 1 folded, in code order
+  uint32_t low[512];            // level 2: [0, 256) for the lower rank's bin, [256, 512) for the upper one's
+  int bin[2];
+  uint32_t above[2];
+};
+
+__global__ void __launch_bounds__(kBrThreads)
 bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const int32_t* __restrict__ cu, int Hq,
                int G, int S, int row_chunks, const int32_t* __restrict__ b_step, RowBracket* __restrict__ bracket,
-               uint32_t* __restrict__ above, uint32_t* __restrict__ ncand, const int32_t* __restrict__ kv_len) {
-  __shared__ uint32_t red[2 * (kRowThreads / 32)];
+               const int32_t* __restrict__ kv_len) {
+  __shared__ BracketShared sh;
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int rowid = (r * Hq + g) * S + s;
   const int start = cu[r];
   const int kh = g / G;
   const int N = valid_keys(kv_len, r, Hq / G, kh, cu[r + 1] - start);
-  const int tid = threadIdx.x;
-  if (tid == 0) { above[rowid] = 0; ncand[rowid] = 0; }
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = N > 0 ? b_step[r * Hq + g] : 0;
   if (N <= 0 || k <= 0) {                                  // nothing to select
     if (tid == 0) bracket[rowid] = RowBracket{INFINITY, INFINITY};
@@ -108,13 +112,16 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
                                    kVoteRowChunk + crow) * kVoteTileKeys;
   uint4 v[kBrVecs];
   const int n_vecs = geo.ns * 16;
+  const int have = (n_vecs + kBrThreads - 1) / kBrThreads;   // the same for every thread of the CTA
 #pragma unroll
   for (int u = 0; u < kBrVecs; ++u) {
-    const int i = u * kRowThreads + tid;
-    v[u] = make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u);     // -inf: never counted
-    if (i < n_vecs) v[u] = *reinterpret_cast<const uint4*>(base + (int64_t)(i >> 4) * slot_stride + (i & 15) * 8);
+    const int i = u * kBrThreads + tid;
+    v[u] = make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u);     // -inf: below every rank asked for
+    if (u < have && i < n_vecs) v[u] = *reinterpret_cast<const uint4*>(base + (int64_t)(i >> 4) * slot_stride + (i & 15) * 8);
   }
-  // ranks (1-based, among the m sampled keys) whose keys become the bounds
+  for (int i = tid; i < 128 * 32; i += kBrThreads) sh.lanes[i] = 0;     // (while the loads are in flight)
+  for (int i = tid; i < 512; i += kBrThreads) sh.low[i] = 0;
+  // ranks (1-based, among the sampled keys; the pad counts as -inf keys) whose keys become the bounds
   const int m = sample_keys(geo, N);
   uint32_t rank_hi, rank_lo;                               // rank_hi <= rank_lo; 0 = no bound on that side
   if (geo.whole) {
@@ -128,17 +135,76 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
     rank_lo = r_lo > m ? 0u : (uint32_t)r_lo;
     rank_hi = r_hi >= 1 ? (uint32_t)r_hi : 0u;
   }
-  // both order statistics at once, bit by bit from the top: largest code c with #(key >= c) >= rank
-  BlockSum sum{red, 0};
-  uint32_t code_hi = 0, code_lo = 0;
-  for (int bit = 15; bit >= 0; --bit) {
-    const uint32_t t_hi = code_hi | (1u << bit), t_lo = code_lo | (1u << bit);
-    uint32_t c_hi, c_lo;
-    sum.sum2(rank_hi ? count_ge(v, raw_of_code(t_hi)) : 0u, rank_lo ? count_ge(v, raw_of_code(t_lo)) : 0u, c_hi, c_lo);
-    if (rank_hi && c_hi >= rank_hi) code_hi = t_hi;
-    if (rank_lo && c_lo >= rank_lo) code_lo = t_lo;
+  __syncthreads();
+  // ---- level 1
+#pragma unroll
+  for (int u = 0; u < kBrVecs; ++u) {
+    if (u >= have) break;
+    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t h0 = w[j] & 0xffffu, h1 = w[j] >> 16;
+      if (h0 == 0x8000u) h0 = 0u;                          // -0 counts as +0
+      if (h1 == 0x8000u) h1 = 0u;
+      atomicAdd(&sh.lanes[(h0 >> 9) * 32 + lane], 1u << ((h0 >> 4) & 16u));
+      atomicAdd(&sh.lanes[(h1 >> 9) * 32 + lane], 1u << ((h1 >> 4) & 16u));
+    }
   }
+  __syncthreads();
+  {
+    // thread t sums word row t (raw high bytes 2t, 2t+1) over the lanes, starting at its own lane: no conflicts
+    uint32_t acc = 0;
+    const uint32_t* wrow = &sh.lanes[tid * 32];
+#pragma unroll 8
+    for (int l = 0; l < 32; ++l) acc += wrow[(l + lane) & 31];
+    sh.bins[ord_hi(2u * tid)] = acc & 0xffffu;
+    sh.bins[ord_hi(2u * tid + 1u)] = acc >> 16;
+  }
+  __syncthreads();
+  if (warp < 2) {                                          // warp 0: the lower bound's rank, warp 1: the upper one's
+    const uint32_t rank = warp == 0 ? rank_lo : rank_hi;
+    int bin = 0;
+    uint32_t up = 0;
+    if (rank) warp_find_bin256(sh.bins, rank, lane, bin, up);
+    if (lane == 0) { sh.bin[warp] = bin; sh.above[warp] = up; }
+  }
+  __syncthreads();
+  // ---- level 2
+  const uint32_t bin_lo = (uint32_t)sh.bin[0], bin_hi = rank_hi ? (uint32_t)sh.bin[1] : bin_lo;
+  const uint32_t up_lo = sh.above[0], up_hi = sh.above[1];
+  const bool two = bin_hi != bin_lo;
+  {
+    // codes below 0x8000 are negative numbers: their raw bits run the other way
+    const uint32_t raw_lo = bin_lo < 0x80u ? 0xffu - bin_lo : bin_lo - 0x80u, flip_lo = bin_lo < 0x80u ? 0xffu : 0u;
+    const uint32_t raw_hi = bin_hi < 0x80u ? 0xffu - bin_hi : bin_hi - 0x80u, flip_hi = bin_hi < 0x80u ? 0xffu : 0u;
+#pragma unroll
+    for (int u = 0; u < kBrVecs; ++u) {
+      if (u >= have) break;
+      const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int e2 = 0; e2 < 2; ++e2) {
+          uint32_t h = e2 ? (w[j] >> 16) : (w[j] & 0xffffu);
+          if (h == 0x8000u) h = 0u;
+          if ((h >> 8) == raw_lo) atomicAdd(&sh.low[(h & 255u) ^ flip_lo], 1u);
+          else if (two && (h >> 8) == raw_hi) atomicAdd(&sh.low[256u + ((h & 255u) ^ flip_hi)], 1u);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (warp < 2) {
+    const uint32_t rank = warp == 0 ? rank_lo : rank_hi;
+    const uint32_t up = warp == 0 ? up_lo : up_hi;
+    int bin = 0;
+    uint32_t dummy = 0;
+    if (rank) warp_find_bin256(warp == 1 && two ? sh.low + 256 : sh.low, rank - up, lane, bin, dummy);
+    if (lane == 0) sh.bin[warp] = bin;
+  }
+  __syncthreads();
   if (tid == 0) {
+    const uint32_t code_lo = (bin_lo << 8) | (uint32_t)sh.bin[0], code_hi = (bin_hi << 8) | (uint32_t)sh.bin[1];
     // two codes of slack either side: the sweep compares fp32 logits, the sample held their roundings
     RowBracket b;
     b.lo = (rank_lo && code_lo >= 0x0402u) ? float_of_code(code_lo - 2u) : -INFINITY;
@@ -148,20 +214,28 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
 }
 
 // ------------------------------------------------------------------------------------ resolve
-// Candidate keys as order-preserving integers, in shared memory when the list fits there, else read
-// from the list in global memory.
-struct CandKeys {
-  const uint32_t* p;
-  int stride;
-  __device__ __forceinline__ uint32_t operator[](int i) const { return p[(int64_t)i * stride]; }
+constexpr int kRowThreads = 256;
+
+struct ResolveShared {
+  uint32_t hist[256];
+  uint32_t red[2][kRowThreads / 32];
+  uint32_t seg_off[kRowThreads / 32];   // scan scratch
+  uint32_t total_above, total_cand, overflow;
+  uint32_t kmin, kmax;
+  int bin;
+  uint32_t above;
 };
 
+// After the sweep: the row's k - #above largest listed candidates, by (fp32 logit descending, key index
+// ascending), into the tentative mask.  The candidates of a row sit in `segs` segments (one per writer of
+// the sweep); their order-preserving 32-bit images are gathered into shared memory and the threshold is
+// found by a most-significant-digit radix search over them (256 bins per pass, starting at the first bit
+// in which the images differ); integer counts only, so two runs give the same bits.
 __global__ void __launch_bounds__(kRowThreads)
 resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32_t* __restrict__ b_step,
                const VoteState vs, int smem_keys, int64_t row_words, const int32_t* __restrict__ kv_len) {
-  extern __shared__ __align__(16) uint32_t keys_sm[];
-  __shared__ uint32_t red[2 * (kRowThreads / 32)];
-  __shared__ uint32_t s_min, s_max;
+  extern __shared__ __align__(16) uint32_t dyn[];         // [seg offsets: segs + 1][keys: smem_keys]
+  __shared__ ResolveShared sh;
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int rowid = (r * Hq + g) * S + s;
   const int start = cu[r], Ncap = cu[r + 1] - start;
@@ -170,78 +244,175 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
   if (N <= 0) return;
   const int k = min(b_step[r * Hq + g], N);
   if (k <= 0) return;
-  const int tid = threadIdx.x;
-  const uint32_t A = vs.above[rowid], C = vs.ncand[rowid];
-  if (A > (uint32_t)k || C > (uint32_t)vs.lay.cap(Ncap) || A + C < (uint32_t)k) {   // the bracket missed or the list overflowed
-    if (tid == 0) atomicExch(&vs.head_bad[r * Hkv + kh], 1u);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int segs = vs.lay.segs, seg_cap = vs.lay.seg_cap(Ncap);
+  uint32_t* seg_off = dyn;                                 // exclusive prefix of the segments' counts
+  uint32_t* keys = dyn + segs + 1;
+  if (tid == 0) { sh.total_above = 0; sh.overflow = 0; sh.kmin = 0xffffffffu; sh.kmax = 0u; }
+  __syncthreads();
+  // what the sweep's writers met: totals, overflow of any segment, and where each segment's keys go
+  {
+    const uint2* st = vs.segstat + (int64_t)rowid * segs;
+    uint32_t run = 0;                                      // candidates in the segments before this round
+    for (int base = 0; base < segs; base += kRowThreads) {
+      const int i = base + tid;
+      const uint2 v = i < segs ? st[i] : make_uint2(0u, 0u);
+      if (v.y > (uint32_t)seg_cap) sh.overflow = 1u;
+      const uint32_t a = __reduce_add_sync(0xffffffffu, v.x);
+      if (lane == 0 && a) atomicAdd(&sh.total_above, a);
+      uint32_t inc = v.y;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+      }
+      if (lane == 31) sh.seg_off[warp] = inc;
+      __syncthreads();
+      uint32_t before = run, all = 0;
+#pragma unroll
+      for (int w = 0; w < kRowThreads / 32; ++w) { if (w < warp) before += sh.seg_off[w]; all += sh.seg_off[w]; }
+      if (i < segs) seg_off[i] = before + inc - v.y;
+      run += all;
+      __syncthreads();
+    }
+    if (tid == 0) { seg_off[segs] = run; sh.total_cand = run; }
+    __syncthreads();
+  }
+  const uint32_t A = sh.total_above, C = sh.total_cand;
+  if (sh.overflow || A > (uint32_t)k || A + C < (uint32_t)k || ((uint32_t)k > A && C > (uint32_t)smem_keys)) {
+    if (tid == 0) atomicExch(&vs.head_bad[r * Hkv + kh], 1u);   // the bracket missed or a list overflowed
     return;
   }
   const uint32_t need = (uint32_t)k - A;
   if (need == 0) return;
-  uint2* list = vs.list(g, s, S, start, r);
+  const uint2* list = vs.list(g, s, S, start, r);
   uint32_t* mrow = vs.tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
+  // one warp per segment, a lane per entry
   if (need == C) {                                         // every listed key is taken
-    for (int i = tid; i < (int)C; i += kRowThreads) {
-      const uint32_t n = list[i].y;
-      atomicOr(&mrow[n >> 5], 1u << (n & 31));
+    for (int sg = warp; sg < segs; sg += kRowThreads / 32) {
+      const uint32_t cnt = seg_off[sg + 1] - seg_off[sg];
+      for (uint32_t i = lane; i < cnt; i += 32) {
+        const uint32_t n = list[(int64_t)sg * seg_cap + i].y;
+        atomicOr(&mrow[n >> 5], 1u << (n & 31));
+      }
     }
     return;
   }
-  // order-preserving images of the listed logits
-  CandKeys keys;
-  if ((int)C <= smem_keys) {
-    for (int i = tid; i < (int)C; i += kRowThreads) keys_sm[i] = ordered_key(__uint_as_float(list[i].x));
-    keys.p = keys_sm;
-    keys.stride = 1;
-  } else {
-    for (int i = tid; i < (int)C; i += kRowThreads) list[i].x = ordered_key(__uint_as_float(list[i].x));
-    keys.p = reinterpret_cast<const uint32_t*>(list);
-    keys.stride = 2;
-  }
-  if (tid == 0) { s_min = 0xffffffffu; s_max = 0u; }
-  __syncthreads();
+  // Entry e of the row's candidates in list order: segment sg holds entries seg_off[sg] .. seg_off[sg+1]-1.
+  // A thread finds the segment of its entry by bisection over the offsets, so that the loads of all its
+  // entries are independent and in flight together.
+  auto entry_of = [&](uint32_t e) -> const uint2* {
+    int a = 0, b = segs;                                   // seg_off[a] <= e < seg_off[b]
+    while (b - a > 1) {
+      const int mid = (a + b) >> 1;
+      if (seg_off[mid] <= e) a = mid; else b = mid;
+    }
+    return list + (int64_t)a * seg_cap + (e - seg_off[a]);
+  };
+  // gather the order-preserving images of the listed logits
   {
     uint32_t mn = 0xffffffffu, mx = 0u;
-    for (int i = tid; i < (int)C; i += kRowThreads) { const uint32_t x = keys[i]; mn = min(mn, x); mx = max(mx, x); }
+    for (uint32_t base = 0; base < C; base += 4 * kRowThreads) {
+      uint32_t x[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t e = base + u * kRowThreads + tid;
+        x[u] = e < C ? entry_of(e)->x : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t e = base + u * kRowThreads + tid;
+        if (e < C) {
+          const uint32_t kx = ordered_key(__uint_as_float(x[u]));
+          keys[e] = kx;
+          mn = min(mn, kx);
+          mx = max(mx, kx);
+        }
+      }
+    }
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
-    if ((tid & 31) == 0) { atomicMin(&s_min, mn); atomicMax(&s_max, mx); }
+    if (lane == 0) { atomicMin(&sh.kmin, mn); atomicMax(&sh.kmax, mx); }
   }
   __syncthreads();
-  // the need-th largest key: the bits above the first one in which the extremes differ are common to all
-  BlockSum sum{red, 0};
-  const uint32_t diff = s_min ^ s_max;
-  uint32_t T = s_max;
-  if (diff) {
-    const int top = 31 - __clz(diff);
-    T = top == 31 ? 0u : (s_max & ~((2u << top) - 1u));
-    for (int bit = top; bit >= 0; --bit) {
-      const uint32_t trial = T | (1u << bit);
-      uint32_t c = 0;
-      for (int i = tid; i < (int)C; i += kRowThreads) c += keys[i] >= trial ? 1u : 0u;
-      if (sum(c) >= need) T = trial;
+  // radix search for the need-th largest image, from the first bit in which the extremes differ
+  uint32_t prefix = 0, known = 0, acc = 0;                 // acc: keys above the prefix found so far
+  uint32_t eq = 0;
+  bool whole_bin = false;                                  // every key of the last bin found is taken
+  {
+    const uint32_t diff = sh.kmin ^ sh.kmax;
+    int top = diff ? 31 - __clz(diff) : -1;
+    if (top < 31) { known = top < 0 ? 0xffffffffu : ~((2u << top) - 1u); prefix = sh.kmax & known; }
+    if (top < 0) { eq = C; }
+    while (top >= 0) {
+      const int lo_bit = top >= 7 ? top - 7 : 0;
+      const uint32_t digit_mask = (top - lo_bit == 31) ? 0xffffffffu : (((2u << (top - lo_bit)) - 1u));
+      sh.hist[tid] = 0;
+      __syncthreads();
+      for (uint32_t i = tid; i < C; i += kRowThreads) {
+        const uint32_t x = keys[i];
+        if ((x & known) == prefix) atomicAdd(&sh.hist[(x >> lo_bit) & digit_mask], 1u);
+      }
+      __syncthreads();
+      if (warp == 0) {
+        int bin;
+        uint32_t up;
+        warp_find_bin256(sh.hist, need - acc, lane, bin, up);
+        if (lane == 0) { sh.bin = bin; sh.above = up; }
+      }
+      __syncthreads();
+      const uint32_t bin = (uint32_t)sh.bin;
+      acc += sh.above;
+      eq = sh.hist[bin];
+      prefix |= bin << lo_bit;
+      known |= digit_mask << lo_bit;
+      __syncthreads();
+      if (eq == need - acc) { whole_bin = true; break; }   // the bin is taken whole: no finer digit needed
+      top = lo_bit - 1;
     }
   }
-  uint32_t gt = 0, eq = 0;
-  for (int i = tid; i < (int)C; i += kRowThreads) { const uint32_t x = keys[i]; gt += x > T ? 1u : 0u; eq += x == T ? 1u : 0u; }
-  gt = sum(gt);
-  eq = sum(eq);
-  const uint32_t ties = need - gt;                         // 1 <= ties <= eq
-  // equal logits go to the lower key index: the ties-th smallest index among them bounds the ones taken
+  // keys above the bin found are taken; of the bin's keys either all (whole_bin, or all equal images needed)
+  // or, when its keys are equal images and more than needed, the `ties` lowest key indices
+  const uint32_t ties = need - acc;                        // 1 <= ties <= eq
   uint32_t idx_max = 0xffffffffu;
-  if (ties < eq) {
-    uint32_t vlim = 0;                                     // largest v with #(equal, index < v) < ties
+  if (!whole_bin && ties < eq) {
+    // largest v with #(equal image, index < v) < ties, bit by bit: the ties-th lowest index among them
+    uint32_t vlim = 0;
     for (int bit = 31 - __clz(max(N - 1, 1)); bit >= 0; --bit) {
       const uint32_t trial = vlim | (1u << bit);
       uint32_t c = 0;
-      for (int i = tid; i < (int)C; i += kRowThreads) c += (keys[i] == T && list[i].y < trial) ? 1u : 0u;
-      if (sum(c) < ties) vlim = trial;
+      for (int sg = warp; sg < segs; sg += kRowThreads / 32) {
+        const uint32_t o = seg_off[sg], cnt = seg_off[sg + 1] - o;
+        for (uint32_t i = lane; i < cnt; i += 32)
+          c += (keys[o + i] == prefix && list[(int64_t)sg * seg_cap + i].y < trial) ? 1u : 0u;
+      }
+      c = __reduce_add_sync(0xffffffffu, c);
+      uint32_t* row = sh.red[bit & 1];
+      if (lane == 0) row[warp] = c;
+      __syncthreads();
+      uint32_t tot = 0;
+#pragma unroll
+      for (int w = 0; w < kRowThreads / 32; ++w) tot += row[w];
+      if (tot < ties) vlim = trial;
     }
     idx_max = vlim;
   }
-  for (int i = tid; i < (int)C; i += kRowThreads) {
-    const uint32_t x = keys[i], n = list[i].y;
-    if (x > T || (x == T && n <= idx_max)) atomicOr(&mrow[n >> 5], 1u << (n & 31));
+  const bool all_of_bin = whole_bin || ties >= eq;
+  for (uint32_t base = 0; base < C; base += 4 * kRowThreads) {
+    uint32_t n[4];
+    bool want[4], tie[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t e = base + u * kRowThreads + tid;
+      const uint32_t x = e < C ? keys[e] : 0u;
+      const bool in_bin = e < C && (x & known) == prefix;
+      want[u] = e < C && (x > (prefix | ~known) || (in_bin && all_of_bin));
+      tie[u] = in_bin && !all_of_bin;
+      n[u] = (want[u] || tie[u]) ? entry_of(e)->y : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (want[u] || (tie[u] && n[u] <= idx_max)) atomicOr(&mrow[n[u] >> 5], 1u << (n[u] & 31));
   }
 }
 
@@ -299,8 +470,8 @@ int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, 
   dim3 grid(p->S, Hq, batch);
   {
     LaunchScope scope_("bracket_kernel", st);
-    bracket_kernel<<<grid, kRowThreads, 0, st>>>(vs.sample, vs.sample_slots, cu, Hq, G, p->S, score_geometry(p).row_chunks,
-                                                 b_step, vs.bracket, vs.above, vs.ncand, kv_len);
+    bracket_kernel<<<grid, kBrThreads, 0, st>>>(vs.sample, vs.sample_slots, cu, Hq, G, p->S, score_geometry(p).row_chunks,
+                                                b_step, vs.bracket, kv_len);
   }
   GVOTE_LAUNCH_CHECK("bracket_kernel");
   return GVOTE_OK;
@@ -310,10 +481,13 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
                        const VoteState& vs, int64_t row_words, const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   dim3 grid(p->S, Hq, batch);
-  // the keys of a list live in shared memory when it leaves room for six CTAs per SM
-  const int64_t longest = vs.lay.uniform_cap > 0 ? vs.lay.uniform_cap : vs.lay.cap((int)max_N);
-  const int smem_keys = (int)(longest <= 8192 ? longest : 8192);
-  const size_t smem = (size_t)smem_keys * sizeof(uint32_t);
+  // shared memory: the segments' offsets and the images of the listed keys.  Room for twice the keys a
+  // row is expected to list at most, within 64 KB; a row that lists more goes the exact way.
+  (void)max_N;
+  int64_t cap_all = (int64_t)vs.lay.segs * (vs.lay.uniform_seg_cap > 0 ? vs.lay.uniform_seg_cap : vs.lay.seg_cap((int)max_N));
+  if (cap_all > 16000) cap_all = 16000;
+  const int smem_keys = (int)cap_all;
+  const size_t smem = ((size_t)vs.lay.segs + 1 + (size_t)smem_keys) * sizeof(uint32_t);
   if (smem > 48 * 1024)
     GVOTE_CUDA_CHECK(cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {

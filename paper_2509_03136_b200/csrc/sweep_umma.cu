@@ -73,25 +73,25 @@ __device__ __forceinline__ uint32_t key16x2_of(float lo, float hi) {
   return p;
 }
 
-// The key tiles a CTA walks: every tile x, x+X, ..., or only those of the row sample.
+// The key tiles a CTA walks.  Second pass: every tile x, x+X, ...  First pass: first the CTA's share of the
+// row sample (slots x, x+X, ... of the sample, whatever CTA streams those tiles: every CTA gets the same
+// number of full products), then, in the CTAs that stream the keys for the current-query rows, the tiles
+// x, x+X, ...
 struct TileWalk {
   SampleGeom g;
-  int x, X, count;
-  bool sampled_only;
-  __device__ __forceinline__ void init(int N, int x_, int X_, bool sampled_only_) {
+  int x, X, n_samp, count;
+  __device__ __forceinline__ void init(int N, int x_, int X_, bool sample, bool stream) {
     g = sample_geom(N);
-    x = x_; X = X_; sampled_only = sampled_only_;
-    const int n = sampled_only ? g.ns : g.n_tiles;
-    count = (N > 0 && x < n) ? (n - x + X - 1) / X : 0;
+    x = x_; X = X_;
+    n_samp = (sample && N > 0 && x < g.ns) ? (g.ns - x + X - 1) / X : 0;
+    const int n_stream = (stream && N > 0 && x < g.n_tiles) ? (g.n_tiles - x + X - 1) / X : 0;
+    count = n_samp + n_stream;
   }
   __device__ __forceinline__ int tile(int i) const {
-    const int j = x + i * X;
-    return sampled_only ? sample_tile(g, j) : j;
+    return i < n_samp ? sample_tile(g, x + i * X) : x + (i - n_samp) * X;
   }
-  // position of tile(i) in the sample, or -1
-  __device__ __forceinline__ int slot(int i) const {
-    return sampled_only ? x + i * X : sample_slot_of_tile(g, x + i * X);
-  }
+  // position of item i in the sample, or -1 for a streamed tile
+  __device__ __forceinline__ int slot(int i) const { return i < n_samp ? x + i * X : -1; }
 };
 
 struct SweepSmem {
@@ -103,7 +103,7 @@ struct SweepSmem {
 };
 
 __device__ __forceinline__ SweepSmem carve(uint8_t* smem_raw, int kchunks, int cg, int stages, bool with_real,
-                                           int n_out) {
+                                           uint32_t staging_bytes) {
   SweepSmem s;
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t q_bytes = (uint32_t)cg * kchunks * kRowChunk * 128;
@@ -113,7 +113,7 @@ __device__ __forceinline__ SweepSmem carve(uint8_t* smem_raw, int kchunks, int c
   s.Qr = s.Qs + q_bytes;
   s.Ks = s.Qr + qr_bytes;
   s.Os = s.Ks + (size_t)stages * stage_bytes;
-  s.tail = reinterpret_cast<SweepTail*>(s.Os + (size_t)n_out * kRowChunk * kTileKeys * 2);
+  s.tail = reinterpret_cast<SweepTail*>(s.Os + staging_bytes);
   return s;
 }
 
@@ -175,9 +175,9 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int c_first = grp * cg, c_cnt = min(cg, row_chunks - c_first);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   TileWalk walk;
-  walk.init(N, (int)blockIdx.x, do_real ? X0 : X1, !do_real);
+  walk.init(N, (int)blockIdx.x, do_real ? X0 : X1, true, do_real);
 
-  const SweepSmem sm = carve(smem_raw, kchunks, cg, stages, true, n_out);
+  const SweepSmem sm = carve(smem_raw, kchunks, cg, stages, true, (uint32_t)n_out * kRowChunk * kTileKeys * 2);
   SweepTail* tail = sm.tail;
   setup(tail, stages, &tmK, &tmQ, &tmQr);
   const uint32_t tmem_base = tail->tmem_slot;
@@ -223,9 +223,10 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (!wait_or_abort(&tail->full[s], ph, abort_flag)) break;
         ptx::tc_fence_after_sync();
         const uint32_t k_addr = ptx::smem_u32(sm.Ks + (size_t)s * stage_bytes);
-        if (do_real) {
-          const int ar = it & 1;
-          if (!wait_or_abort(&tail->real_empty[ar], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag)) break;
+        if (it >= walk.n_samp) {
+          const int is = it - walk.n_samp;                 // streamed tiles so far
+          const int ar = is & 1;
+          if (!wait_or_abort(&tail->real_empty[ar], (((uint32_t)is >> 1) & 1u) ^ 1u, abort_flag)) break;
           ptx::tc_fence_after_sync();
           const uint32_t d2 = tmem_base + (uint32_t)(kD2Col + ar * 32);
           const int ksteps = d_k / 16;
@@ -236,8 +237,7 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             ptx::umma_bf16(d2, dk, dq, idesc2, k > 0 ? 1u : 0u);
           }
           ptx::umma_commit(&tail->real_full[ar]);
-        }
-        if (walk.slot(it) >= 0) {
+        } else {
           for (int cc = 0; ok && cc < c_cnt; ++cc, ++n1) {
             const int a = n1 & 1;
             if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)n1 >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -261,9 +261,10 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     for (int it = 0; it < walk.count; ++it) {
       const int t = walk.tile(it);
       // ---- current-query rows: thread = key, exact fp32 logits and their running maximum
-      if (do_real && half == 0) {
-        const int ar = it & 1;
-        const bool got = wait_or_abort(&tail->real_full[ar], ((uint32_t)it >> 1) & 1u, abort_flag);
+      if (it >= walk.n_samp && half == 0) {
+        const int is = it - walk.n_samp;
+        const int ar = is & 1;
+        const bool got = wait_or_abort(&tail->real_full[ar], ((uint32_t)is >> 1) & 1u, abort_flag);
         ptx::tc_fence_after_sync();
         uint32_t w[16];
         ptx::tmem_ld_32x16(tmem_base + (uint32_t)(kD2Col + ar * 32) + ((uint32_t)(q * 32) << 16), w);
@@ -352,8 +353,14 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------ second pass
-template <int CG>
-__global__ void __launch_bounds__(kSweepThreads, 1)
+// Sixteen read-out warps: four per lane quadrant, each 32 of the tile's 128 keys, so that a thread holds 32
+// consecutive logits of its row.  Four warps per scheduler hide the latencies of the chain (accumulator
+// ready, tensor-memory load, compares, list writes) that two could not.
+constexpr int kSweepEpiWarps = 16;
+constexpr int kSweepBThreads = 64 + 32 * kSweepEpiWarps;
+
+template <int CG, int STG>      // STG: logits a thread stages at a time (16, or 8 when shared memory is short)
+__global__ void __launch_bounds__(kSweepBThreads, 1)
 score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int row_chunks, int stages,
                    float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
@@ -368,11 +375,27 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const int c_first = grp * CG, c_cnt = min(CG, row_chunks - c_first);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   TileWalk walk;
-  walk.init(N, (int)blockIdx.x, (int)gridDim.x, false);
+  walk.init(N, (int)blockIdx.x, (int)gridDim.x, false, true);
 
-  const SweepSmem sm = carve(smem_raw, kchunks, CG, stages, false, 0);
+  // [query chunks | key stages | staging of the read-out: STG floats per thread | barriers]
+  const SweepSmem sm = carve(smem_raw, kchunks, CG, stages, false, (uint32_t)kSweepEpiWarps * 32 * STG * 4);
   SweepTail* tail = sm.tail;
-  setup(tail, stages, &tmK, &tmQ, nullptr);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
+    ptx::mbar_init(&tail->q_full, 1);
+    for (int a2 = 0; a2 < 2; ++a2) { ptx::mbar_init(&tail->acc_full[a2], 1); ptx::mbar_init(&tail->acc_empty[a2], kSweepEpiWarps); }
+    tail->abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmK);
+    ptx::prefetch_tensormap(&tmQ);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&tail->tmem_slot, 256);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
   const uint32_t tmem_base = tail->tmem_slot;
   volatile int* abort_flag = &tail->abort_flag;
   const uint32_t q_chunk_bytes = (uint32_t)kchunks * kRowChunk * 128;
@@ -420,26 +443,33 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       }
     }
   } else {
-    const int e = warp - 2;
-    const int q = warp & 3;
-    const int half = e >> 2;
-    // this thread's row in each chunk of the group: its bracket, its list, its count of keys above
+    const int e = warp - 2;                      // 0..15
+    const int q = warp & 3;                      // tensor-memory lane quadrant this warp may read
+    const int cq = e >> 2;                       // which 32 keys of the tile this warp takes
+    const int seg = (int)blockIdx.x * 4 + cq;    // this thread's segment of its rows' lists
+    const int seg_cap = vs.lay.seg_cap(Ncap);
+    // the thread's staging area: STG floats in 16-byte pieces; piece c sits at position c ^ swz, which keeps
+    // the 16-byte stores of a quarter warp on different banks
+    constexpr int kPieces = STG / 4;
+    uint8_t* stg = sm.Os + (size_t)(e * 32 + lane) * (STG * 4);
+    const uint32_t stg_swz = ((uint32_t)lane >> (kPieces == 4 ? 1 : 2)) & (uint32_t)(kPieces - 1);
+    // this thread's row in each chunk of the group: its bracket, its segment, its counts
     float lo[CG], hi[CG];
-    uint32_t abv[CG];
+    uint32_t abv[CG], fill[CG];
     int rowid[CG];
-    uint2* list[CG];
-    const int cap = vs.lay.cap(Ncap);
+    uint2* segp[CG];
 #pragma unroll
     for (int cc = 0; cc < CG; ++cc) {
       const int grow = (c_first + cc) * kRowChunk + q * 32 + lane;       // row within the head group
       abv[cc] = 0;
+      fill[cc] = 0;
       rowid[cc] = -1;
-      list[cc] = nullptr;
+      segp[cc] = nullptr;
       lo[cc] = INFINITY;
       hi[cc] = INFINITY;
       if (cc < c_cnt && grow < G * S) {
         rowid[cc] = (r * Hq + kh * G + grow / S) * S + grow % S;
-        list[cc] = vs.list(kh * G + grow / S, grow % S, S, start, r);
+        segp[cc] = vs.list(kh * G + grow / S, grow % S, S, start, r) + (int64_t)seg * seg_cap;
         const RowBracket b = vs.bracket[rowid[cc]];
         lo[cc] = b.lo;
         hi[cc] = b.hi;
@@ -449,11 +479,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     int n1 = 0;
     for (int it = 0; it < walk.count; ++it) {
       const int t = walk.tile(it);
-      // keys of this half of the tile that exist (a ragged last tile reads whatever follows the row)
-      const int left = N - t * kTileKeys - half * 64;
-      const uint32_t vm0 = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
-      const uint32_t vm1 = left >= 64 ? 0xffffffffu : (left > 32 ? (1u << (left - 32)) - 1u : 0u);
-      const int n0 = t * kTileKeys + half * 64;
+      // keys of this quarter of the tile that exist (a ragged last tile reads whatever follows the row)
+      const int left = N - t * kTileKeys - cq * 32;
+      const uint32_t vm = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
+      const int n0 = t * kTileKeys + cq * 32;
 #pragma unroll
       for (int cc = 0; cc < CG; ++cc) {
         if (cc >= c_cnt) break;
@@ -461,58 +490,57 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         wait_or_abort(&tail->acc_full[a], ((uint32_t)n1 >> 1) & 1u, abort_flag);
         ++n1;
         ptx::tc_fence_after_sync();
-        const uint32_t taddr = tmem_base + (uint32_t)(a * kRowChunk) + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 64);
-        uint32_t v0[32], v1[32];
-        ptx::tmem_ld_32x32(taddr, v0);
-        ptx::tmem_ld_32x32(taddr + 32u, v1);
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(tmem_base + (uint32_t)(a * kRowChunk) + ((uint32_t)(q * 32) << 16) + (uint32_t)(cq * 32), v);
         ptx::tmem_wait_ld();
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&tail->acc_empty[a]);     // the values are in registers: free the accumulator
 
         const float hi_r = hi[cc], lo_r = lo[cc];
-        uint32_t ab0 = 0, ab1 = 0, cb0 = 0, cb1 = 0;
+        uint32_t ab4[4] = {0, 0, 0, 0}, cb4[4] = {0, 0, 0, 0};    // four independent chains of eight keys
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float l0 = __uint_as_float(v0[i]) * scale, l1 = __uint_as_float(v1[i]) * scale;
-          ab0 |= (l0 > hi_r ? 1u : 0u) << i;
-          cb0 |= (l0 >= lo_r ? 1u : 0u) << i;
-          ab1 |= (l1 > hi_r ? 1u : 0u) << i;
-          cb1 |= (l1 >= lo_r ? 1u : 0u) << i;
+          const float l = __uint_as_float(v[i]) * scale;
+          v[i] = __float_as_uint(l);
+          ab4[i >> 3] |= (l > hi_r ? 1u : 0u) << i;
+          cb4[i >> 3] |= (l >= lo_r ? 1u : 0u) << i;
         }
-        ab0 &= vm0; ab1 &= vm1;
-        cb0 &= vm0 & ~ab0; cb1 &= vm1 & ~ab1;
+        const uint32_t ab = (ab4[0] | ab4[1] | ab4[2] | ab4[3]) & vm;
+        const uint32_t cb = (cb4[0] | cb4[1] | cb4[2] | cb4[3]) & vm & ~ab;
         // union step: the warp's 32 rows OR their bits, one atomic per mask word
-        const uint32_t w0 = __reduce_or_sync(0xffffffffu, ab0), w1 = __reduce_or_sync(0xffffffffu, ab1);
-        if (lane == 0) {
-          if (w0) atomicOr(&mrow[(n0 >> 5)], w0);
-          if (w1) atomicOr(&mrow[(n0 >> 5) + 1], w1);
-        }
-        abv[cc] += __popc(ab0) + __popc(ab1);
-        const uint32_t cnt = __popc(cb0) + __popc(cb1);
-        if (cnt) {
-          uint32_t slot = atomicAdd(&vs.ncand[rowid[cc]], cnt);
-          uint2* const lst = list[cc];
+        const uint32_t w = __reduce_or_sync(0xffffffffu, ab);
+        if (lane == 0 && w) atomicOr(&mrow[n0 >> 5], w);
+        abv[cc] += __popc(ab);
+        if (cb) {
+          // the listed keys: their logits go through the thread's staging area, STG at a time, so that they
+          // can be fetched by position
+          uint2* const sp = segp[cc];
+          uint32_t f = fill[cc];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if ((cb0 >> i) & 1u) {
-              if (slot < (uint32_t)cap) lst[slot] = make_uint2(__float_as_uint(__uint_as_float(v0[i]) * scale), (uint32_t)(n0 + i));
-              ++slot;
+          for (int part = 0; part < 32 / STG; ++part) {
+            uint32_t sub = (cb >> (STG * part)) & ((1u << STG) - 1u);
+            if (sub == 0) continue;
+#pragma unroll
+            for (int c = 0; c < kPieces; ++c)
+              *reinterpret_cast<uint4*>(stg + (((uint32_t)c ^ stg_swz) << 4)) =
+                  make_uint4(v[STG * part + 4 * c], v[STG * part + 4 * c + 1], v[STG * part + 4 * c + 2], v[STG * part + 4 * c + 3]);
+            while (sub) {
+              const int j = __ffs(sub) - 1;
+              sub &= sub - 1;
+              const uint32_t bits = *reinterpret_cast<const uint32_t*>(stg + ((((uint32_t)j >> 2) ^ stg_swz) << 4) + ((j & 3) << 2));
+              if (f < (uint32_t)seg_cap) sp[f] = make_uint2(bits, (uint32_t)(n0 + STG * part + j));
+              ++f;
             }
           }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if ((cb1 >> i) & 1u) {
-              if (slot < (uint32_t)cap) lst[slot] = make_uint2(__float_as_uint(__uint_as_float(v1[i]) * scale), (uint32_t)(n0 + 32 + i));
-              ++slot;
-            }
-          }
+          fill[cc] = f;
         }
       }
     }
+    // what this writer met, for every row it owns (zeros too: resolve_kernel reads every segment)
 #pragma unroll
     for (int cc = 0; cc < CG; ++cc)
-      if (rowid[cc] >= 0 && abv[cc]) atomicAdd(&vs.above[rowid[cc]], abv[cc]);
+      if (rowid[cc] >= 0) vs.segstat[(int64_t)rowid[cc] * vs.lay.segs + seg] = make_uint2(abv[cc], fill[cc]);
   }
 
   ptx::tc_fence_before_sync();
@@ -523,7 +551,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   }
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    ptx::tmem_dealloc(tmem_base, 256);
   }
 }
 
@@ -582,9 +610,10 @@ int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const
   const int kchunks = d_k / 64;
   const size_t out_bytes = (size_t)kRowChunk * kTileKeys * 2;
   const size_t qr = align_up((size_t)kchunks * kRealCols * 128, 1024);
-  int stages = 0, n_out = 2;
-  int cg = pick_chunks(row_chunks > 2 ? 2 : row_chunks, kchunks, qr + 2 * out_bytes, 3, &stages);
-  if (cg == 0) { n_out = 1; cg = pick_chunks(row_chunks > 2 ? 2 : row_chunks, kchunks, qr + out_bytes, 2, &stages); }
+  // one staging buffer: a CTA has few sampled tiles, and a deeper ring of key stages is worth more to the stream
+  int stages = 0;
+  const int n_out = 1;
+  const int cg = pick_chunks(row_chunks > 2 ? 2 : row_chunks, kchunks, qr + out_bytes, 2, &stages);
   if (cg == 0) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   const size_t smem = 1024 + (size_t)cg * kchunks * kRowChunk * 128 + qr + (size_t)stages * kchunks * kTileKeys * 128 +
                       n_out * out_bytes + sizeof(SweepTail) + 64;
@@ -613,6 +642,29 @@ int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const
   return GVOTE_OK;
 }
 
+// Chunks per CTA, key stages and CTAs per (request, KV head, chunk group) of the second pass.
+SweepGeom sweep_geometry(const gvote_params* p, int32_t batch, int64_t max_N) {
+  SweepGeom g{0, 0, 1, 1, 16};
+  if (!sweep_umma_supported(p)) return g;
+  const int row_chunks = score_geometry(p).row_chunks;
+  g.cg = pick_chunks(row_chunks, p->d_k / 64, (size_t)kSweepEpiWarps * 32 * 64, 2, &g.stages);
+  // all chunks in one CTA (every key tile fetched once) is worth a smaller staging area
+  const int want = row_chunks >= 3 ? 4 : row_chunks;
+  if (g.cg < want) {
+    int st8 = 0;
+    const int cg8 = pick_chunks(row_chunks, p->d_k / 64, (size_t)kSweepEpiWarps * 32 * 32, 2, &st8);
+    if (cg8 > g.cg) { g.cg = cg8; g.stages = st8; g.stg = 8; }
+  }
+  if (g.cg == 0) return g;
+  g.groups = (row_chunks + g.cg - 1) / g.cg;
+  const int64_t max_tiles = ceil_div(max_N > 0 ? max_N : 1, kTileKeys);
+  int64_t X = (batch == 1 ? 148 : 592) / ((int64_t)p->n_kv_heads * g.groups * batch);
+  if (X > max_tiles) X = max_tiles;
+  if (X < 1) X = 1;
+  g.X = (int)X;
+  return g;
+}
+
 // Second pass (after bracket_kernel).
 int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                            int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
@@ -623,24 +675,19 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
   CUtensorMap tmK, tmQ;
   if (!encode_maps(p, Q, K, k_tok, k_head, batch, total_tokens, &tmK, &tmQ, nullptr)) return GVOTE_ERR_UNSUPPORTED_SHAPE;
   const int kchunks = d_k / 64;
-  int stages = 0;
-  const int cg = pick_chunks(row_chunks, kchunks, 0, 2, &stages);
-  if (cg == 0) return GVOTE_ERR_UNSUPPORTED_SHAPE;
-  const size_t smem = 1024 + (size_t)cg * kchunks * kRowChunk * 128 + (size_t)stages * kchunks * kTileKeys * 128 +
-                      sizeof(SweepTail) + 64;
-  const int groups = (row_chunks + cg - 1) / cg;
-  const int64_t max_tiles = ceil_div(max_N, kTileKeys);
-  int64_t X = (batch == 1 ? 148 : 592) / ((int64_t)Hkv * groups * batch);
-  if (X > max_tiles) X = max_tiles;
-  if (X < 1) X = 1;
-  dim3 grid((unsigned)X, (unsigned)(Hkv * groups), (unsigned)batch);
+  const SweepGeom geo = sweep_geometry(p, batch, max_N);
+  if (geo.cg == 0 || vs.lay.segs != 4 * geo.X) return GVOTE_ERR_UNSUPPORTED_SHAPE;
+  const size_t smem = 1024 + (size_t)geo.cg * kchunks * kRowChunk * 128 + (size_t)geo.stages * kchunks * kTileKeys * 128 +
+                      (size_t)kSweepEpiWarps * 32 * geo.stg * 4 + sizeof(SweepTail) + 64;
+  dim3 grid((unsigned)geo.X, (unsigned)(Hkv * geo.groups), (unsigned)batch);
   const float scale = (float)(1.0 / sqrt((double)d_k));
-  auto kern = cg == 4 ? score_sweep_kernel<4> : (cg == 2 ? score_sweep_kernel<2> : score_sweep_kernel<1>);
+  auto kern = geo.stg == 8 ? (geo.cg == 4 ? score_sweep_kernel<4, 8> : (geo.cg == 2 ? score_sweep_kernel<2, 8> : score_sweep_kernel<1, 8>))
+                           : (geo.cg == 4 ? score_sweep_kernel<4, 16> : (geo.cg == 2 ? score_sweep_kernel<2, 16> : score_sweep_kernel<1, 16>));
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sweep_kernel", st);
-    kern<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, stages, scale, vs, row_words,
-                                            status, kv_len);
+    kern<<<grid, kSweepBThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, scale, vs, row_words,
+                                             status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_sweep_kernel");
   return GVOTE_OK;

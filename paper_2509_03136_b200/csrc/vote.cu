@@ -269,12 +269,11 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
   VoteState vs;
   vs.sample = reinterpret_cast<uint16_t*>(ws + m.sample);
   vs.bracket = reinterpret_cast<RowBracket*>(ws + m.bracket);
-  vs.above = reinterpret_cast<uint32_t*>(ws + m.above);
-  vs.ncand = reinterpret_cast<uint32_t*>(ws + m.ncand);
+  vs.segstat = reinterpret_cast<uint2*>(ws + m.segstat);
   vs.cand = reinterpret_cast<uint2*>(ws + m.cand);
   vs.tmask = reinterpret_cast<uint32_t*>(ws + m.tmask);
   vs.head_bad = reinterpret_cast<uint32_t*>(ws + m.head_bad);
-  vs.lay = cand_layout(batch, total_tokens, max_N);
+  vs.lay = cand_layout(m.cand_segs, batch, total_tokens, max_N);
   vs.sample_slots = m.sample_slots;
   float* real_logits = reinterpret_cast<float*>(ws + m.logits);
   uint32_t* rowmax = reinterpret_cast<uint32_t*>(ws + m.rowmax);

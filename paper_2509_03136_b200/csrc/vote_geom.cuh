@@ -62,40 +62,45 @@ inline int64_t sample_slots_total(int32_t batch, int64_t total_tokens, int64_t m
   return (int64_t)34 * batch + (total_tokens >> 10) + 1;
 }
 
-// Entries a row's candidate list needs.  The bracket spans 2 * (4.5 sqrt(m f (1 - f)) + 6) of the m
-// sampled keys' ranks, at most 4.5 sqrt(m) + 12, i.e. that many times N / m keys of the row; a quarter
-// more covers the spread of the count.  A completely sampled row lists only the keys that share the
-// threshold's 16-bit value or its neighbours'.
-inline int candidate_need(int64_t N) {
-  if (N <= 0) return 256;
+// Keys a row's bracket is expected to hold at most.  It spans 2 * (4.5 sqrt(m f (1 - f)) + 6) of the m
+// sampled keys' ranks, at most 4.5 sqrt(m) + 12, i.e. that many times N / m keys of the row.  A completely
+// sampled row lists only the keys that share the threshold's 16-bit value or its neighbours'.
+inline double candidates_expected(int64_t N) {
+  if (N <= 0) return 64.0;
   const SampleGeom g = sample_geom((int)N);
-  double need = 512.0;
-  if (!g.whole) {
-    const double m = (double)g.ns * kVoteTileKeys;
-    need = 1.25 * (4.5 * sqrt(m) + 12.0) * ((double)N / m) + 256.0;
-  }
-  return ((int)need + 255) & ~255;
+  if (g.whole) return 64.0;
+  const double m = (double)g.ns * kVoteTileKeys;
+  return (4.5 * sqrt(m) + 12.0) * ((double)N / m);
 }
-// Where the lists live: row (g, s) of the batch owns a strip of `strip` entries, request r's list starts
-// at entry cand_offset(r) of the strip and holds cand_cap(N_r) entries.  A single request gets exactly
-// candidate_need(N); in a batch the capacity is the line 512 + 3 N / 32, which lies above candidate_need
-// for every N and has a closed-form running sum over the requests.
+
+// Where the candidate lists live.  The sweep's read-out threads never share a list: thread (CTA x, column
+// quarter c) of a row owns segment x * 4 + c of the row's list, `segs` = 4 X segments in all, and appends
+// to it without atomics.  A CTA's tiles x, x + X, ... are spread evenly over the row, so a segment holds an
+// even share mu of the row's candidates up to counting noise: capacity mu + 4.5 sqrt(mu) + 8 for a single
+// request; in a batch, the line 20 + 29 N / (256 segs) above that, whose running sum over the requests
+// has a closed form (no kernel has to add up the requests before its own).  Row (g, s) owns a strip of
+// `strip` entries; request r's segments start at entry offset(r) of the strip.
 struct CandLayout {
-  int uniform_cap;       // > 0: one request, this capacity
+  int segs;
+  int uniform_seg_cap;   // > 0: one request, this capacity per segment
   int64_t strip;
-  __host__ __device__ __forceinline__ int cap(int N) const { return uniform_cap > 0 ? uniform_cap : 512 + (int)((3 * (int64_t)N) >> 5); }
+  __host__ __device__ __forceinline__ int seg_cap(int N) const {
+    return uniform_seg_cap > 0 ? uniform_seg_cap : 20 + (int)(((29 * (int64_t)N) >> 8) / segs);
+  }
   __host__ __device__ __forceinline__ int64_t offset(int cu_r, int r) const {
-    return uniform_cap > 0 ? 0 : (int64_t)576 * r + ((3 * (int64_t)cu_r) >> 5);
+    return uniform_seg_cap > 0 ? 0 : (int64_t)segs * 20 * r + ((29 * (int64_t)cu_r) >> 8);
   }
 };
-inline CandLayout cand_layout(int32_t batch, int64_t total_tokens, int64_t max_N) {
+inline CandLayout cand_layout(int segs, int32_t batch, int64_t total_tokens, int64_t max_N) {
   CandLayout c;
+  c.segs = segs;
   if (batch == 1) {
-    c.uniform_cap = candidate_need(max_N);
-    c.strip = c.uniform_cap;
+    const double mu = candidates_expected(max_N) / segs;
+    c.uniform_seg_cap = (((int)ceil(mu + 4.5 * sqrt(mu) + 8.0)) + 3) & ~3;
+    c.strip = (int64_t)segs * c.uniform_seg_cap;
   } else {
-    c.uniform_cap = 0;
-    c.strip = (int64_t)576 * batch + ((3 * total_tokens) >> 5) + 1;
+    c.uniform_seg_cap = 0;
+    c.strip = (int64_t)segs * 20 * batch + ((29 * total_tokens) >> 8) + 1;
   }
   return c;
 }
@@ -106,18 +111,21 @@ struct RowBracket { float lo, hi; };    // keys above hi are taken, keys in [lo,
 struct VoteState {
   uint16_t* sample;        // fp16 keys [n_kv_heads][sample slots][row_chunks][128 rows][128 keys]
   RowBracket* bracket;     // [rows]
-  uint32_t* above;         // [rows] keys above the bracket (counted by the sweep)
-  uint32_t* ncand;         // [rows] keys inside the bracket (listed by the sweep, up to `cap`)
+  uint2* segstat;          // [rows][segs] (keys above the bracket, keys inside it) met by each segment's writer
   uint2* cand;             // [n_q_heads * S][strip] (fp32 logit bits, key index), see CandLayout
   CandLayout lay;
   uint32_t* tmask;         // [n_kv_heads][row_words] the union while it is tentative
   uint32_t* head_bad;      // [batch][n_kv_heads] a bracket of the head missed: redo the head exactly
   int64_t sample_slots;
-  // the list of row (g, s) of request r
+  // the first segment of the list of row (g, s) of request r
   __host__ __device__ __forceinline__ uint2* list(int g, int s, int S, int cu_r, int r) const {
     return cand + (int64_t)(g * S + s) * lay.strip + lay.offset(cu_r, r);
   }
 };
+
+// Launch geometry of the second pass (sweep_umma.cu); the segment count of the lists follows from it.
+struct SweepGeom { int cg, stages, groups, X, stg; };
+SweepGeom sweep_geometry(const gvote_params* p, int32_t batch, int64_t max_N);
 
 #ifdef __CUDACC__
 // Exact fp32 logit of key n for one query row (fixed summation order).
