@@ -105,11 +105,9 @@ WorkspaceMap workspace_map(const gvote_params* p, int32_t batch, int64_t total_t
     m.cand_segs = 4 * sweep_geometry(p, batch, max_N).X;
     m.cand_strip = cand_layout(m.cand_segs, batch, total_tokens, max_N).strip;
     m.sample_slots = sample_slots_total(batch, total_tokens, max_N);
-    m.vote_zero = off;
     m.tmask = take((size_t)p->n_kv_heads * m.row_words * sizeof(uint32_t));
     m.head_bad = take((size_t)batch * p->n_kv_heads * sizeof(uint32_t));
-    m.rowmax = take((size_t)batch * p->n_q_heads * sizeof(uint32_t));
-    m.vote_zero_bytes = off - m.vote_zero;
+    m.rowmax = take((size_t)batch * p->n_q_heads * 148 * sizeof(uint32_t));
     m.sample = take((size_t)p->n_kv_heads * m.sample_slots * score_geometry(p).row_chunks * kVoteRowChunk *
                     kVoteTileKeys * sizeof(uint16_t));
     m.bracket = take(rows * sizeof(RowBracket));

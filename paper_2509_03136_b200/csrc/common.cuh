@@ -43,6 +43,25 @@ struct LaunchScope {
     }                                                            \
   } while (0)
 
+// Launch with programmatic dependent launch: the kernel may start (up to its pdl_wait) while the kernel
+// before it on the stream is still running, so that its prologue - barrier set-up, tensor-memory
+// allocation, descriptor prefetch - and the launch latency hide under the predecessor's tail.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -70,11 +89,9 @@ struct WorkspaceMap {
   // the current-query rows, [Hq * total_tokens], and the state of the fused top-k (vote_geom.cuh)
   bool full_rows;
   size_t logits;
-  size_t vote_zero;     // cleared at the start of every vote: [tmask | head_bad | rowmax]
-  size_t vote_zero_bytes;
-  size_t tmask;         // uint32 [Hkv][row_words]
+  size_t tmask;         // uint32 [Hkv][row_words]   (cleared, like head_bad and the keep mask, by the vote's first kernel)
   size_t head_bad;      // uint32 [batch][Hkv]
-  size_t rowmax;        // uint32 [batch][Hq]  row maxima of the current-query rows (topp_real.cu)
+  size_t rowmax;        // uint32 [batch][Hq][<= 148]  maxima of the current-query rows met by the first pass's CTAs
   size_t sample;        // uint16 [Hkv][sample_slots][row_chunks][128][128]
   size_t bracket;       // RowBracket [batch*Hq*S]
   size_t segstat;       // uint2 [batch*Hq*S][cand_segs]
@@ -161,6 +178,14 @@ int32_t launch_overlap(const gvote_params* p, const __nv_bfloat16* Q, const __nv
 
 // ---------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
+
+// Programmatic dependent launch, device side.  pdl_trigger: the next kernel on the stream may begin to
+// launch (called first thing: what it may touch before its own pdl_wait is only its shared and tensor
+// memory).  pdl_wait: every kernel before this one on the stream has completed and its writes are
+// visible; nothing a predecessor writes or reads may be touched before it.  Both do nothing in a kernel
+// launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Monotone map from float to uint32: a > b  <=>  key(a) > key(b)  (no NaNs expected).
 __device__ __forceinline__ uint32_t ordered_key(float f) {

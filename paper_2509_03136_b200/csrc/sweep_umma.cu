@@ -161,25 +161,37 @@ __global__ void __launch_bounds__(kSweepThreads, 1)
 score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                     const __grid_constant__ CUtensorMap tmQr, const int32_t* __restrict__ cu, int Hq, int G, int S,
                     int d_k, int row_chunks, int cg, int X0, int X1, int stages, int n_out, float scale,
-                    float* __restrict__ real_logits, uint32_t* __restrict__ rowmax, uint16_t* __restrict__ sample,
-                    int64_t sample_slots, int32_t* __restrict__ status, const int32_t* __restrict__ kv_len) {
+                    float* __restrict__ real_logits, uint32_t* __restrict__ rowmax_part, uint16_t* __restrict__ sample,
+                    int64_t sample_slots, int32_t* __restrict__ status, const int32_t* __restrict__ kv_len,
+                    uint32_t* __restrict__ zero_a, uint32_t* __restrict__ zero_b, int64_t zero_words,
+                    uint32_t* __restrict__ head_bad, int n_head_bad) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+  pdl_trigger();
   const int groups = (row_chunks + cg - 1) / cg;
   const int r = blockIdx.z;
   const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
   const bool do_real = grp == 0;
-  if ((int)blockIdx.x >= (do_real ? X0 : X1)) return;
-  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
-  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
+  const bool active = (int)blockIdx.x < (do_real ? X0 : X1);
   const int kchunks = d_k / 64;
-  const int c_first = grp * cg, c_cnt = min(cg, row_chunks - c_first);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  TileWalk walk;
-  walk.init(N, (int)blockIdx.x, do_real ? X0 : X1, true, do_real);
-
   const SweepSmem sm = carve(smem_raw, kchunks, cg, stages, true, (uint32_t)n_out * kRowChunk * kTileKeys * 2);
   SweepTail* tail = sm.tail;
-  setup(tail, stages, &tmK, &tmQ, &tmQr);
+  if (active) setup(tail, stages, &tmK, &tmQ, &tmQr);     // barriers, tensor memory: under the tail of the kernel before
+  pdl_wait();
+  // The vote starts from an empty keep mask, an empty tentative mask and no head marked: every CTA of this
+  // first kernel of the vote clears its share (nothing reads them before the kernels that follow).
+  {
+    const int64_t n_thr = (int64_t)gridDim.x * gridDim.y * gridDim.z * blockDim.x;
+    const int64_t me = (((int64_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
+    for (int64_t i = me; i < zero_words; i += n_thr) { zero_a[i] = 0u; zero_b[i] = 0u; }
+    if (me < n_head_bad) head_bad[me] = 0u;
+  }
+  if (!active) return;
+  const int start = cu[r], Ncap = cu[r + 1] - start;       // Ncap: rows of the slab (layout); N: rows that count
+  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
+  const int c_first = grp * cg, c_cnt = min(cg, row_chunks - c_first);
+  TileWalk walk;
+  walk.init(N, (int)blockIdx.x, do_real ? X0 : X1, true, do_real);
   const uint32_t tmem_base = tail->tmem_slot;
   volatile int* abort_flag = &tail->abort_flag;
   const uint32_t q_chunk_bytes = (uint32_t)kchunks * kRowChunk * 128;
@@ -344,8 +356,9 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     atomicExch(&status[0], GVOTE_ERR_TIMEOUT);
     atomicExch(&status[1], 5);
   }
-  if (do_real && (int)threadIdx.x < G && tail->rowmax[threadIdx.x] != 0)
-    atomicMax(&rowmax[r * Hq + kh * G + (int)threadIdx.x], tail->rowmax[threadIdx.x]);
+  // this CTA's maxima of the current-query rows (0 = it met no key): real_topp_kernel takes the largest of the X0
+  if (do_real && (int)threadIdx.x < G)
+    rowmax_part[(int64_t)(r * Hq + kh * G + (int)threadIdx.x) * X0 + blockIdx.x] = tail->rowmax[threadIdx.x];
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -356,60 +369,61 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 // Sixteen read-out warps: four per lane quadrant, each 32 of the tile's 128 keys, so that a thread holds 32
 // consecutive logits of its row.  Four warps per scheduler hide the latencies of the chain (accumulator
 // ready, tensor-memory load, compares, list writes) that two could not.
+//
+// The query rows are the MMA's A operand and live in TENSOR memory here, not in shared memory: each row's
+// d_k bf16 values, two to a 32-bit column, written once by the read-out warps (tcgen05.st) straight from
+// global memory.  With both operands in shared memory a 128 x 128 x 16 instruction has to fetch 8 KB per
+// 64 clocks, all the shared-memory bandwidth there is; with A in tensor memory it fetches only the key
+// tile's 4 KB, and the shared memory the rows would take goes to a deeper ring of key stages.
 constexpr int kSweepEpiWarps = 16;
 constexpr int kSweepBThreads = 64 + 32 * kSweepEpiWarps;
 
 template <int CG, int STG>      // STG: logits a thread stages at a time (16, or 8 when shared memory is short)
 __global__ void __launch_bounds__(kSweepBThreads, 1)
-score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16* __restrict__ Q,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int row_chunks, int stages,
                    float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
                    const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+  pdl_trigger();
   const int groups = (row_chunks + CG - 1) / CG;
   const int r = blockIdx.z;
   const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
-  const int start = cu[r], Ncap = cu[r + 1] - start;
-  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
   const int kchunks = d_k / 64;
   const int c_first = grp * CG, c_cnt = min(CG, row_chunks - c_first);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  TileWalk walk;
-  walk.init(N, (int)blockIdx.x, (int)gridDim.x, false, true);
 
-  // [query chunks | key stages | staging of the read-out: STG floats per thread | barriers]
-  const SweepSmem sm = carve(smem_raw, kchunks, CG, stages, false, (uint32_t)kSweepEpiWarps * 32 * STG * 4);
+  // [key stages | staging of the read-out: STG floats per thread | barriers]
+  const SweepSmem sm = carve(smem_raw, kchunks, 0, stages, false, (uint32_t)kSweepEpiWarps * 32 * STG * 4);
   SweepTail* tail = sm.tail;
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
-    ptx::mbar_init(&tail->q_full, 1);
+    ptx::mbar_init(&tail->q_full, kSweepEpiWarps);
     for (int a2 = 0; a2 < 2; ++a2) { ptx::mbar_init(&tail->acc_full[a2], 1); ptx::mbar_init(&tail->acc_empty[a2], kSweepEpiWarps); }
     tail->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmK);
-    ptx::prefetch_tensormap(&tmQ);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&tail->tmem_slot, 256);
+    ptx::tmem_alloc(&tail->tmem_slot, kTmemCols);            // 2 x 128 accumulator columns, then the query rows
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
+  pdl_wait();
+  const int start = cu[r], Ncap = cu[r + 1] - start;
+  const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
+  TileWalk walk;
+  walk.init(N, (int)blockIdx.x, (int)gridDim.x, false, true);
   const uint32_t tmem_base = tail->tmem_slot;
   volatile int* abort_flag = &tail->abort_flag;
-  const uint32_t q_chunk_bytes = (uint32_t)kchunks * kRowChunk * 128;
   const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
   const int R = G * (S + 1);
+  const uint32_t a_cols = (uint32_t)d_k / 2;               // tensor-memory columns of one chunk's query rows
 
   if (warp == 0) {
     if (lane == 0 && walk.count > 0) {
-      const int group_row = (r * (Hq / G) + kh) * R;
-      ptx::mbar_arrive_expect_tx(&tail->q_full, (uint32_t)c_cnt * q_chunk_bytes);
-      for (int cc = 0; cc < c_cnt; ++cc)
-        for (int c = 0; c < kchunks; ++c)
-          ptx::tma_load_2d(sm.Qs + ((size_t)cc * kchunks + c) * kRowChunk * 128, &tmQ, &tail->q_full, c * 64,
-                           group_row + (c_first + cc) * kRowChunk);
       for (int it = 0; it < walk.count; ++it) {
         const int s = it % stages;
         const uint32_t ph = (uint32_t)(it / stages) & 1u;
@@ -423,8 +437,9 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     }
   } else if (warp == 1) {
     if (lane == 0 && walk.count > 0) {
-      const uint32_t q_addr = ptx::smem_u32(sm.Qs);
-      bool ok = wait_or_abort(&tail->q_full, 0, abort_flag);
+      const uint32_t idesc = ptx::instr_desc_bf16_f32(kRowChunk, kTileKeys);
+      bool ok = wait_or_abort(&tail->q_full, 0, abort_flag);   // the query rows are in tensor memory
+      ptx::tc_fence_after_sync();
       int n1 = 0;
       for (int it = 0; ok && it < walk.count; ++it) {
         const int s = it % stages;
@@ -436,7 +451,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           const int a = n1 & 1;
           if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)n1 >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after_sync();
-          issue_d1(tmem_base + (uint32_t)(a * kRowChunk), q_addr + (uint32_t)cc * q_chunk_bytes, k_addr, d_k);
+          const uint32_t d = tmem_base + (uint32_t)(a * kRowChunk), qa = tmem_base + 256u + (uint32_t)cc * a_cols;
+          const int ksteps = d_k / 16;
+          for (int k = 0; k < ksteps; ++k) {
+            const uint32_t koff = (uint32_t)(k >> 2), kin = (uint32_t)(k & 3) * 32u;
+            const uint64_t dk = ptx::smem_desc_k_sw128(k_addr + koff * (uint32_t)(kTileKeys * 128) + kin);
+            ptx::umma_bf16_ts(d, qa + (uint32_t)k * 8u, dk, idesc, k > 0 ? 1u : 0u);
+          }
           ptx::umma_commit(&tail->acc_full[a]);
         }
         ptx::umma_commit(&tail->empty[s]);
@@ -451,10 +472,11 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     // the thread's staging area: STG floats in 16-byte pieces; piece c sits at position c ^ swz, which keeps
     // the 16-byte stores of a quarter warp on different banks
     constexpr int kPieces = STG / 4;
+    const float inv_scale = 1.0f / scale;
     uint8_t* stg = sm.Os + (size_t)(e * 32 + lane) * (STG * 4);
     const uint32_t stg_swz = ((uint32_t)lane >> (kPieces == 4 ? 1 : 2)) & (uint32_t)(kPieces - 1);
     // this thread's row in each chunk of the group: its bracket, its segment, its counts
-    float lo[CG], hi[CG];
+    __half2 lo[CG], hi[CG];
     uint32_t abv[CG], fill[CG];
     int rowid[CG];
     uint2* segp[CG];
@@ -465,15 +487,39 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       fill[cc] = 0;
       rowid[cc] = -1;
       segp[cc] = nullptr;
-      lo[cc] = INFINITY;
-      hi[cc] = INFINITY;
+      float lo_f = INFINITY, hi_f = INFINITY;              // a row that does not exist takes nothing
       if (cc < c_cnt && grow < G * S) {
         rowid[cc] = (r * Hq + kh * G + grow / S) * S + grow % S;
         segp[cc] = vs.list(kh * G + grow / S, grow % S, S, start, r) + (int64_t)seg * seg_cap;
         const RowBracket b = vs.bracket[rowid[cc]];
-        lo[cc] = b.lo;
-        hi[cc] = b.hi;
+        lo_f = b.lo * inv_scale;
+        hi_f = b.hi * inv_scale;
       }
+      lo[cc] = __half2half2(__float2half_rd(lo_f));        // bounds rounded outwards
+      hi[cc] = __half2half2(__float2half_ru(hi_f));
+    }
+    // the query rows of chunk cc go to tensor memory through the four warps with cq == cc mod 4 (one per lane
+    // quadrant): a thread fetches its row from global memory, 32 columns (64 values) at a time
+    if (walk.count > 0) {
+#pragma unroll
+      for (int cc = 0; cc < CG; ++cc) {
+        if (cc >= c_cnt || (cc & 3) != cq) continue;
+        const int grow = (c_first + cc) * kRowChunk + q * 32 + lane;
+        const uint4* src = reinterpret_cast<const uint4*>(Q + ((int64_t)(r * (Hq / G) + kh) * R + grow) * d_k);
+        for (uint32_t c0 = 0; c0 < a_cols; c0 += 32) {
+          uint32_t w[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 x = grow < G * S ? __ldg(src + (c0 >> 2) + j) : make_uint4(0u, 0u, 0u, 0u);
+            w[4 * j] = x.x; w[4 * j + 1] = x.y; w[4 * j + 2] = x.z; w[4 * j + 3] = x.w;
+          }
+          ptx::tmem_st_32x32(tmem_base + 256u + (uint32_t)cc * a_cols + c0 + ((uint32_t)(q * 32) << 16), w);
+        }
+      }
+      ptx::tmem_wait_st();
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&tail->q_full);
     }
     uint32_t* mrow = vs.tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
     int n1 = 0;
@@ -497,17 +543,28 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&tail->acc_empty[a]);     // the values are in registers: free the accumulator
 
-        const float hi_r = hi[cc], lo_r = lo[cc];
-        uint32_t ab4[4] = {0, 0, 0, 0}, cb4[4] = {0, 0, 0, 0};    // four independent chains of eight keys
+        // Compare as half-precision pairs, two keys per instruction, on the unscaled accumulators (the row's
+        // bounds were divided by the scale and rounded outwards).  Rounding a key to half precision is monotone,
+        // so every key found above the upper bound still exceeds every key that is not; keys that round onto a
+        // bound are listed and settled exactly later.
+        const __half2 hi2 = hi[cc], lo2 = lo[cc];
+        uint32_t ab = 0, cb = 0;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float l = __uint_as_float(v[i]) * scale;
-          v[i] = __float_as_uint(l);
-          ab4[i >> 3] |= (l > hi_r ? 1u : 0u) << i;
-          cb4[i >> 3] |= (l >= lo_r ? 1u : 0u) << i;
+        for (int g8 = 0; g8 < 4; ++g8) {                         // eight keys: bits 2j (low half) and 17 + 2j (high half)
+          uint32_t gacc = 0, cacc = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t pk = key16x2_of(__uint_as_float(v[8 * g8 + 2 * j]), __uint_as_float(v[8 * g8 + 2 * j + 1]));
+            const __half2 h2 = *reinterpret_cast<const __half2*>(&pk);
+            const uint32_t pick = (1u << (2 * j)) | (1u << (17 + 2 * j));
+            gacc |= __hgt2_mask(h2, hi2) & pick;
+            cacc |= __hge2_mask(h2, lo2) & pick;
+          }
+          ab |= ((gacc | (gacc >> 16)) & 0xffu) << (8 * g8);
+          cb |= ((cacc | (cacc >> 16)) & 0xffu) << (8 * g8);
         }
-        const uint32_t ab = (ab4[0] | ab4[1] | ab4[2] | ab4[3]) & vm;
-        const uint32_t cb = (cb4[0] | cb4[1] | cb4[2] | cb4[3]) & vm & ~ab;
+        ab &= vm;
+        cb &= vm & ~ab;
         // union step: the warp's 32 rows OR their bits, one atomic per mask word
         const uint32_t w = __reduce_or_sync(0xffffffffu, ab);
         if (lane == 0 && w) atomicOr(&mrow[n0 >> 5], w);
@@ -528,8 +585,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
             while (sub) {
               const int j = __ffs(sub) - 1;
               sub &= sub - 1;
-              const uint32_t bits = *reinterpret_cast<const uint32_t*>(stg + ((((uint32_t)j >> 2) ^ stg_swz) << 4) + ((j & 3) << 2));
-              if (f < (uint32_t)seg_cap) sp[f] = make_uint2(bits, (uint32_t)(n0 + STG * part + j));
+              const float acc = *reinterpret_cast<const float*>(stg + ((((uint32_t)j >> 2) ^ stg_swz) << 4) + ((j & 3) << 2));
+              if (f < (uint32_t)seg_cap) sp[f] = make_uint2(__float_as_uint(acc * scale), (uint32_t)(n0 + STG * part + j));
               ++f;
             }
           }
@@ -551,7 +608,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   }
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, 256);
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -601,8 +658,8 @@ bool sweep_umma_supported(const gvote_params* p) {
 // caller then takes the SIMT path).
 int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                             int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                            float* real_logits, uint32_t* rowmax, const VoteState& vs, int32_t* status,
-                            const int32_t* kv_len, cudaStream_t st) {
+                            float* real_logits, uint32_t* rowmax_part, int* n_part, const VoteState& vs, uint32_t* mask,
+                            int64_t row_words, int32_t* status, const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, d_k = p->d_k;
   const int row_chunks = score_geometry(p).row_chunks;
   CUtensorMap tmK, tmQ, tmQr;
@@ -634,10 +691,11 @@ int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sample_kernel", st);
-    score_sample_kernel<<<grid, kSweepThreads, smem, st>>>(tmK, tmQ, tmQr, cu, Hq, G, p->S, d_k, row_chunks, cg, (int)X0,
-                                                           (int)X1, stages, n_out, scale, real_logits, rowmax, vs.sample,
-                                                           vs.sample_slots, status, kv_len);
+    launch_pdl(score_sample_kernel, grid, dim3(kSweepThreads), smem, st, tmK, tmQ, tmQr, cu, Hq, G, p->S, d_k, row_chunks, cg,
+               (int)X0, (int)X1, stages, n_out, scale, real_logits, rowmax_part, vs.sample, vs.sample_slots, status, kv_len,
+               vs.tmask, mask, (int64_t)Hkv * row_words, vs.head_bad, (int)(batch * Hkv));
   }
+  *n_part = (int)X0;
   GVOTE_LAUNCH_CHECK("score_sample_kernel");
   return GVOTE_OK;
 }
@@ -647,15 +705,15 @@ SweepGeom sweep_geometry(const gvote_params* p, int32_t batch, int64_t max_N) {
   SweepGeom g{0, 0, 1, 1, 16};
   if (!sweep_umma_supported(p)) return g;
   const int row_chunks = score_geometry(p).row_chunks;
-  g.cg = pick_chunks(row_chunks, p->d_k / 64, (size_t)kSweepEpiWarps * 32 * 64, 2, &g.stages);
-  // all chunks in one CTA (every key tile fetched once) is worth a smaller staging area
-  const int want = row_chunks >= 3 ? 4 : row_chunks;
-  if (g.cg < want) {
-    int st8 = 0;
-    const int cg8 = pick_chunks(row_chunks, p->d_k / 64, (size_t)kSweepEpiWarps * 32 * 32, 2, &st8);
-    if (cg8 > g.cg) { g.cg = cg8; g.stages = st8; g.stg = 8; }
-  }
-  if (g.cg == 0) return g;
+  // chunks per CTA: their query rows share 256 columns of tensor memory, d_k / 2 columns a chunk
+  int cg = 4;
+  while (cg > 1 && (cg * (p->d_k / 2) > 256 || cg / 2 >= row_chunks)) cg >>= 1;
+  g.cg = cg;
+  const size_t stage = (size_t)(p->d_k / 64) * kTileKeys * 128;
+  const size_t fixed = 1024 + (size_t)kSweepEpiWarps * 32 * 64 + sizeof(SweepTail) + 64;
+  g.stages = (int)((kSmemLimit - fixed) / stage);
+  if (g.stages > kMaxStages) g.stages = kMaxStages;
+  if (g.stages < 2) { g.cg = 0; return g; }
   g.groups = (row_chunks + g.cg - 1) / g.cg;
   const int64_t max_tiles = ceil_div(max_N > 0 ? max_N : 1, kTileKeys);
   int64_t X = (batch == 1 ? 148 : 592) / ((int64_t)p->n_kv_heads * g.groups * batch);
@@ -677,8 +735,8 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
   const int kchunks = d_k / 64;
   const SweepGeom geo = sweep_geometry(p, batch, max_N);
   if (geo.cg == 0 || vs.lay.segs != 4 * geo.X) return GVOTE_ERR_UNSUPPORTED_SHAPE;
-  const size_t smem = 1024 + (size_t)geo.cg * kchunks * kRowChunk * 128 + (size_t)geo.stages * kchunks * kTileKeys * 128 +
-                      (size_t)kSweepEpiWarps * 32 * geo.stg * 4 + sizeof(SweepTail) + 64;
+  const size_t smem = 1024 + (size_t)geo.stages * kchunks * kTileKeys * 128 + (size_t)kSweepEpiWarps * 32 * geo.stg * 4 +
+                      sizeof(SweepTail) + 64;
   dim3 grid((unsigned)geo.X, (unsigned)(Hkv * geo.groups), (unsigned)batch);
   const float scale = (float)(1.0 / sqrt((double)d_k));
   auto kern = geo.stg == 8 ? (geo.cg == 4 ? score_sweep_kernel<4, 8> : (geo.cg == 2 ? score_sweep_kernel<2, 8> : score_sweep_kernel<1, 8>))
@@ -686,7 +744,7 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sweep_kernel", st);
-    kern<<<grid, kSweepBThreads, smem, st>>>(tmK, tmQ, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, scale, vs, row_words,
+    launch_pdl(kern, grid, dim3(kSweepBThreads), smem, st, tmK, Q, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, scale, vs, row_words,
                                              status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_sweep_kernel");

@@ -117,9 +117,11 @@ __device__ __forceinline__ void block_scan_pair(uint32_t c, unsigned long long m
 
 __global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kThreads)
 real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G,
-                 const uint32_t* __restrict__ rowmax, float p_nuc, int include_c0, int64_t row_words,
+                 const uint32_t* __restrict__ rowmax_part, int n_part, float p_nuc, int include_c0, int64_t row_words,
                  uint32_t* __restrict__ mask, int32_t* __restrict__ b_step, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint8_t dyn[];
+  pdl_trigger();
+  pdl_wait();
   ClusterShared& cs = *reinterpret_cast<ClusterShared*>(dyn);
   // The generic radix search and the emission (rare routes of the first CTA) work in the space of the
   // candidate list, which is dead by the time they run.
@@ -137,7 +139,9 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
     return;
   }
   const float* L = logits + (int64_t)Hq * start + (int64_t)g * Ncap;       // [n_q_heads][N] per request
-  const float mx = key_to_float(rowmax[r * Hq + g]);
+  uint32_t mx_key = 0;                                       // the row maximum: the largest of the first pass's CTAs'
+  for (int i = 0; i < n_part; ++i) mx_key = max(mx_key, rowmax_part[(int64_t)(r * Hq + g) * n_part + i]);
+  const float mx = key_to_float(mx_key);
   const float cut = tail_cut(N, p_nuc);
   const int per = (N + kClusterCtas - 1) / kClusterCtas;
   const int n0 = min(crank * per, N), n1 = min(n0 + per, N);
@@ -323,14 +327,23 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
     }
     if (m >= 0) {
       // rank by (value descending, index ascending); ranks are distinct, so this is a permutation
+      // (four list entries per step, fetched as two 16-byte loads: the loop is a chain of shared-memory
+      // latencies otherwise; the list is padded with entries that rank below everything)
+      if (tid < 4) { cs.val[m + tid] = -INFINITY; cs.idx[m + tid] = 0x7fffffff; }
+      __syncthreads();
       if (tid < m) {
         const float v = cs.val[tid];
         const int n = cs.idx[tid];
-        int rank = 0;
-        for (int u = 0; u < m; ++u) {
-          const float vu = cs.val[u];
-          rank += (vu > v || (vu == v && cs.idx[u] < n)) ? 1 : 0;
+        int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+        for (int u = 0; u < m; u += 4) {
+          const float4 vu = *reinterpret_cast<const float4*>(&cs.val[u]);
+          const int4 nu = *reinterpret_cast<const int4*>(&cs.idx[u]);
+          r0 += (vu.x > v || (vu.x == v && nu.x < n)) ? 1 : 0;
+          r1 += (vu.y > v || (vu.y == v && nu.y < n)) ? 1 : 0;
+          r2 += (vu.z > v || (vu.z == v && nu.z < n)) ? 1 : 0;
+          r3 += (vu.w > v || (vu.w == v && nu.w < n)) ? 1 : 0;
         }
+        const int rank = r0 + r1 + r2 + r3;
         cs.rank[tid] = rank;
         cs.smass[rank] = mass_fix(v, mx);
       }
@@ -386,9 +399,9 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
 
 }  // namespace
 
-// `rowmax` [batch][n_q_heads]: the row maxima (order-preserving images) the first pass of the vote leaves.
+// `rowmax_part` [batch][n_q_heads][n_part]: the maxima (order-preserving images) the CTAs of the vote's first pass met.
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         const uint32_t* rowmax, int64_t row_words, uint32_t* mask, int32_t* b_step,
+                         const uint32_t* rowmax_part, int n_part, int64_t row_words, uint32_t* mask, int32_t* b_step,
                          const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   (void)max_N;
@@ -398,7 +411,7 @@ int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32
   dim3 grid((unsigned)kClusterCtas, (unsigned)Hq, (unsigned)batch);
   {
     LaunchScope scope_("real_topp_kernel", st);
-    real_topp_kernel<<<grid, kThreads, sizeof(ClusterShared), st>>>(logits, cu, Hq, G, rowmax, p->p_nuc,
+    launch_pdl(real_topp_kernel, grid, dim3(kThreads), sizeof(ClusterShared), st, logits, cu, Hq, G, rowmax_part, n_part, p->p_nuc,
                                                                     p->include_c0, row_words, mask, b_step, kv_len);
   }
   GVOTE_LAUNCH_CHECK("real_topp_kernel");

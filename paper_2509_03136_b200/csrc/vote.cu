@@ -230,8 +230,8 @@ int32_t launch_score_umma(const gvote_params* p, const __nv_bfloat16* Q, const _
                           float* logits, int32_t* status, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                             int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                            float* real_logits, uint32_t* rowmax, const VoteState& vs, int32_t* status,
-                            const int32_t* kv_len, cudaStream_t st);
+                            float* real_logits, uint32_t* rowmax_part, int* n_part, const VoteState& vs, uint32_t* mask,
+                            int64_t row_words, int32_t* status, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                            int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                            const VoteState& vs, int64_t row_words, int32_t* status, const int32_t* kv_len,
@@ -244,7 +244,7 @@ int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_
                       const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs, int64_t row_words,
                       uint32_t* mask, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
-                         const uint32_t* rowmax, int64_t row_words, uint32_t* mask, int32_t* b_step,
+                         const uint32_t* rowmax_part, int n_part, int64_t row_words, uint32_t* mask, int32_t* b_step,
                          const int32_t* kv_len, cudaStream_t st);
 
 namespace {
@@ -278,14 +278,13 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
   float* real_logits = reinterpret_cast<float*>(ws + m.logits);
   uint32_t* rowmax = reinterpret_cast<uint32_t*>(ws + m.rowmax);
   int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
-  // tentative mask, per-head flags and row maxima start from zero
-  GVOTE_CUDA_CHECK(cudaMemsetAsync(ws + m.vote_zero, 0, m.vote_zero_bytes, st));
-  const int32_t rc = launch_score_sample(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, real_logits, rowmax, vs,
-                                         status, kv_len, st);
+  // (the first kernel also clears the keep mask, the tentative mask and the per-head flags)
+  int n_part = 1;
+  const int32_t rc = launch_score_sample(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, real_logits, rowmax, &n_part,
+                                         vs, mask, m.row_words, status, kv_len, st);
   if (rc != GVOTE_OK) return rc;
-  GVOTE_CUDA_CHECK(cudaMemsetAsync(mask, 0, (size_t)p->n_kv_heads * m.row_words * sizeof(uint32_t), st));
 #define GVOTE_STEP(expr) do { const int32_t rc__ = (expr); if (rc__ != GVOTE_OK) return rc__; } while (0)
-  GVOTE_STEP(launch_real_topp(p, real_logits, cu, batch, max_N, rowmax, m.row_words, mask, b_step, kv_len, st));
+  GVOTE_STEP(launch_real_topp(p, real_logits, cu, batch, max_N, rowmax, n_part, m.row_words, mask, b_step, kv_len, st));
   GVOTE_STEP(launch_bracket(p, cu, batch, b_step, vs, kv_len, st));
   GVOTE_STEP(launch_score_sweep(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, vs, m.row_words, status, kv_len,
                                 st));

@@ -8,10 +8,27 @@ on `torch.distributed` (NCCL on GPUs, gloo in the CPU tests).
 """
 from __future__ import annotations
 
+import socket
+import sys
 from dataclasses import replace
-from typing import List
+from typing import List, Mapping, Optional, Sequence
 
 import torch
+
+
+def self_launch_command(script: str, argv: Sequence[str], n_gpus: int, env: Mapping[str, str],
+                        port: Optional[int] = None) -> Optional[List[str]]:
+    """The command that starts one rank per GPU for `script argv`, or None when nothing has to be started:
+    a single GPU, or a launcher has already set up the ranks (WORLD_SIZE in the environment: its RANK /
+    LOCAL_RANK / MASTER_* are used as they are).  The rendezvous is on 127.0.0.1 (one node)."""
+    if n_gpus <= 1 or "WORLD_SIZE" in env:
+        return None
+    if port is None:
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), script, *argv]
 
 
 def rank_workload(cfg, rank: int):

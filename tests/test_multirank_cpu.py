@@ -52,3 +52,17 @@ def test_single_process_is_a_no_op():
     assert shard.max_over_ranks(3.5) == 3.5
     b = torch.ones(1, 2, dtype=torch.int32)
     assert shard.gather_budgets(b)[0] is b
+
+
+def test_bench_starts_its_own_ranks_only_when_no_launcher_did():
+    """`bench.py --gpus N` without a launcher's environment re-launches itself under torch.distributed.run
+    with one process per GPU on 127.0.0.1; under a launcher, or for one GPU, it runs as it is."""
+    argv = ["--gpus", "4", "--steps", "3"]
+    cmd = shard.self_launch_command("/x/bench.py", argv, 4, {}, port=29511)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert "--nproc-per-node=4" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "29511" and cmd[-5:] == ["/x/bench.py"] + argv
+    assert shard.self_launch_command("/x/bench.py", argv, 4, {"WORLD_SIZE": "4", "RANK": "1"}) is None
+    assert shard.self_launch_command("/x/bench.py", ["--gpus", "1"], 1, {}) is None
+    port = int(shard.self_launch_command("/x/bench.py", argv, 2, {})[8])       # a free port is picked when none is given
+    assert 1024 < port < 65536
