@@ -190,6 +190,73 @@ def workload_config(cfg, args):
             "timing": "sum of per-step CUDA-event intervals on the launch stream"}
 
 
+# ----------------------------------------------------------------------------- S and p sweeps
+def select_once(gv, torch, cfg, li, d, S, p_nuc, mu, var, h_last, reps=5):
+    """gvote_sample + gvote_project + gvote_vote + gvote_overlap for one (S, p) on one layer's device tensors.
+    Returns (mask, budget [batch, Hkv], overlap [batch, Hq], milliseconds of the select step)."""
+    from dataclasses import replace
+    c = replace(cfg, S=S, p_nuc=p_nuc)
+    p = gv.params_from_config(c)
+    geom = (c.batch, c.total_tokens, max(c.seq_lens))
+    ws = gv.alloc_workspace(p, *geom)
+    Ht = torch.empty(c.batch, S, c.d_h, device="cuda")
+    Q = torch.empty(c.batch, c.n_kv_heads, c.G * (S + 1), c.d_k, dtype=torch.bfloat16, device="cuda")
+    mask = torch.empty(c.n_kv_heads, gv.mask_row_words(c.total_tokens, c.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(c.batch, c.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(c.batch, c.n_q_heads, dtype=torch.int32, device="cuda")
+    ov = torch.empty(c.batch, c.n_q_heads, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ms = 0.0
+    for i in range(reps + 2):
+        torch.cuda.synchronize()
+        e0.record()
+        gv.gvote_sample(p, mu, var, c.batch, Ht)
+        gv.gvote_project(p, Ht, h_last, d["W_q"], d["b_q"], d["cu"], c.batch, Q, ws)
+        gv.gvote_vote(p, Q, d["K"], d["cu"], geom, mask, budget, b_step, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            ms += e0.elapsed_time(e1)
+    gv.gvote_overlap(p, Q, d["K"], mask, d["cu"], geom, ov, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    return mask.cpu().numpy(), budget.cpu().numpy(), ov.cpu().numpy(), ms / reps
+
+
+def run_sweep(args, cfg):
+    """Section 4.4's ablations on synthetic data: the budget the vote arrives at, the share of the current
+    query's attention the kept keys hold (Section 3.3's yardstick) and the time of the select step, over
+    S at p = 0.95 and over p at S = 32.  One JSON line per setting."""
+    import torch
+    from paper_2509_03136_b200 import build as gbuild, gvote as gv, synth
+    gbuild.build()
+    gv.load()
+    torch.cuda.set_device(0)
+    li = synth.make_layer(cfg, 0)
+    d = {"W_q": gv.bf16_from_bits(li.W_q), "b_q": None, "K": gv.bf16_from_bits(li.K),
+         "cu": torch.from_numpy(li.cu_seqlens).cuda()}
+    h = torch.from_numpy(li.h).cuda()
+    p0 = gv.params_from_config(cfg)
+    geom = (cfg.batch, cfg.total_tokens, max(cfg.seq_lens))
+    ws = gv.alloc_workspace(p0, *geom)
+    mu = torch.empty(cfg.batch, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p0, h, d["cu"], geom, mu, var, ws)
+    cu = li.cu_seqlens
+    h_last = torch.stack([h[int(cu[r + 1]) - 1] for r in range(cfg.batch)]).contiguous()
+    rows = [("S", S, 0.95) for S in (1, 2, 4, 8, 16, 32, 64)] + [("p", 32, pn) for pn in (0.8, 0.9, 0.95, 0.98, 0.99)]
+    prev_mask = None
+    for axis, S, pn in rows:
+        mask, budget, ov, ms = select_once(gv, torch, cfg, li, d, S, pn, mu, var, h_last)
+        nested = None
+        if axis == "S" and prev_mask is not None:
+            nested = bool(np.all((prev_mask & ~mask) == 0))          # the smaller S's keep set lies inside this one
+        prev_mask = mask if axis == "S" else None
+        print(json.dumps({"sweep": axis, "workload": cfg.name, "S": S, "p_nuc": pn,
+                          "kept_fraction": float(budget.sum() / (cfg.n_kv_heads * cfg.total_tokens)),
+                          "budget_per_head": budget.reshape(-1).tolist(),
+                          "attention_on_kept_keys_mean": float(ov.mean()), "attention_on_kept_keys_min": float(ov.min()),
+                          "select_ms": ms, "contains_previous_S": nested}))
+
+
 # ----------------------------------------------------------------------------- native arm
 def main():
     ap = argparse.ArgumentParser()
@@ -206,6 +273,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-upstream-row", action="store_true")
     ap.add_argument("--no-recompress-row", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark: budget, attention kept and select time over S and over p "
+                         "(one layer of --workload, default c1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -222,6 +292,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, base_cfg, rank, world)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args, base_cfg if "--workload" in sys.argv else synth.make_config("c1"))
         return
 
     import torch

@@ -96,7 +96,14 @@ static inline int64_t gvote_mask_word_offset(int64_t cu_seqlens_r, int32_t r) {
 
 /* Bytes of scratch every entry point below accepts as `ws` for a batch of this size.  The
  * first 256 bytes hold the status word; a workspace must be zero-filled once after
- * allocation (the library keeps it consistent afterwards).  Returns 0 on invalid params. */
+ * allocation (the library keeps it consistent afterwards).  Returns 0 on invalid params.
+ * The size depends on p->sel_mode.  GVOTE_SEL_TOPK_C0 (Algorithm 1) keeps no logits matrix: per synthetic
+ * query a few thousand sampled 16-bit keys and a short candidate list, per current query one fp32 row
+ * (Section 4.4 names the S x N matrix as what runs out of memory beyond 128K context).  GVOTE_SEL_TOPP
+ * needs every row's softmax mass and keeps the fp32 logits of all (S+1) x n_q_heads rows:
+ * 4 (S+1) n_q_heads total_tokens bytes more.  A call that asks for the softmax rows (dbg_probs) needs the
+ * GVOTE_SEL_TOPP size whatever its mode, as do shapes the tensor-core kernels do not take (d_k not a
+ * multiple of 64, more than 16 query heads per KV head). */
 GVOTE_API size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
 /* Step 2 of Section 3.2 (the Gaussian fit of Algorithm 1).  mu[r][c], var[r][c] = mean and unbiased variance over rows
@@ -276,8 +283,19 @@ GVOTE_API int32_t gvote_compress_host(const gvote_params* p, const void* h, cons
                             uint32_t* mask, int32_t* budget, int32_t* b_step);
 GVOTE_API void gvote_host_arena_release(void);
 
-/* Reads the status word of a workspace (synchronises the stream): GVOTE_OK or GVOTE_ERR_TIMEOUT. */
+/* Reads the status word of a workspace (synchronises the stream): GVOTE_OK, GVOTE_ERR_TIMEOUT (a bounded
+ * device-side wait ran out) or GVOTE_ERR_WORKSPACE_TOO_SMALL (gvote_pack: capacity_rows too small).  The word
+ * is only ever set by kernels and STAYS set: every later poll of that workspace reports it again until the
+ * caller clears it, with gvote_clear_status (enqueued on the stream) or by zero-filling the first 256 bytes.
+ * gvote_compress_host clears the status of its own arena at the start of every call. */
 GVOTE_API int32_t gvote_poll_status(void* ws, void* stream);
+GVOTE_API int32_t gvote_clear_status(void* ws, void* stream);
+
+/* Diagnostic of the default selection mode (Algorithm 1's TopK step): how many (request, KV head) pairs
+ * had to be selected again by the exact route because a row's sampled bracket missed its k-th logit or a
+ * candidate list overflowed, since the workspace's status block was last cleared (synchronises the
+ * stream).  The result is the same either way; the exact route only costs time.  Negative: an error code. */
+GVOTE_API int64_t gvote_exact_heads(void* ws, void* stream);
 
 /* Per-kernel timing for benchmarks.  While enabled, every kernel launch of the library is
  * bracketed by two CUDA events on its stream.  Enabling (or disabling) drops earlier records.

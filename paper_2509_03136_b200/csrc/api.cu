@@ -430,6 +430,8 @@ int32_t gvote_compress_host(const gvote_params* p, const void* h, const void* W_
   }
   char* d = g_arena.base;
   cudaStream_t st = g_arena.stream;
+  // a status left by an earlier call on this arena must not be reported again
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(d + o_ws, 0, kStatusBytes, st));
   GVOTE_CUDA_CHECK(cudaMemcpyAsync(d + o_cu, cu_seqlens_host, b_cu, cudaMemcpyHostToDevice, st));
   GVOTE_CUDA_CHECK(cudaMemcpyAsync(d + o_h, h, b_h, cudaMemcpyHostToDevice, st));
   GVOTE_CUDA_CHECK(cudaMemcpyAsync(d + o_w, W_q, b_w, cudaMemcpyHostToDevice, st));
@@ -457,6 +459,20 @@ int32_t gvote_poll_status(void* ws, void* stream) {
   int32_t status = 0;
   GVOTE_CUDA_CHECK(cudaMemcpy(&status, ws, sizeof(status), cudaMemcpyDeviceToHost));
   return status;
+}
+
+int32_t gvote_clear_status(void* ws, void* stream) {
+  if (!ws) return GVOTE_ERR_INVALID_ARG;
+  GVOTE_CUDA_CHECK(cudaMemsetAsync(ws, 0, kStatusBytes, (cudaStream_t)stream));
+  return GVOTE_OK;
+}
+
+int64_t gvote_exact_heads(void* ws, void* stream) {
+  if (!ws) return GVOTE_ERR_INVALID_ARG;
+  GVOTE_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  int32_t words[4] = {0, 0, 0, 0};
+  GVOTE_CUDA_CHECK(cudaMemcpy(words, ws, sizeof(words), cudaMemcpyDeviceToHost));
+  return words[2];
 }
 
 void gvote_profile_enable(int32_t on) {

@@ -284,7 +284,8 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
   }
   const uint32_t A = sh.total_above, C = sh.total_cand;
   if (sh.overflow || A > (uint32_t)k || A + C < (uint32_t)k || ((uint32_t)k > A && C > (uint32_t)smem_keys)) {
-    if (tid == 0) atomicExch(&vs.head_bad[r * Hkv + kh], 1u);   // the bracket missed or a list overflowed
+    // the bracket missed or a list overflowed: the head goes the exact way (counted once per head)
+    if (tid == 0 && atomicExch(&vs.head_bad[r * Hkv + kh], 1u) == 0u) atomicAdd(&vs.status[2], 1);
     return;
   }
   const uint32_t need = (uint32_t)k - A;

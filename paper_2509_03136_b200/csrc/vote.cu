@@ -273,6 +273,7 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
   vs.cand = reinterpret_cast<uint2*>(ws + m.cand);
   vs.tmask = reinterpret_cast<uint32_t*>(ws + m.tmask);
   vs.head_bad = reinterpret_cast<uint32_t*>(ws + m.head_bad);
+  vs.status = reinterpret_cast<int32_t*>(ws + m.status);
   vs.lay = cand_layout(m.cand_segs, batch, total_tokens, max_N);
   vs.sample_slots = m.sample_slots;
   float* real_logits = reinterpret_cast<float*>(ws + m.logits);

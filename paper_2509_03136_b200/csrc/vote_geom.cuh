@@ -116,6 +116,7 @@ struct VoteState {
   CandLayout lay;
   uint32_t* tmask;         // [n_kv_heads][row_words] the union while it is tentative
   uint32_t* head_bad;      // [batch][n_kv_heads] a bracket of the head missed: redo the head exactly
+  int32_t* status;         // the workspace's status block; word 2 counts the heads redone exactly
   int64_t sample_slots;
   // the first segment of the list of row (g, s) of request r
   __host__ __device__ __forceinline__ uint2* list(int g, int s, int S, int cu_r, int r) const {

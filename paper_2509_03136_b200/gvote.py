@@ -24,7 +24,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 EXPORTS = (
     "gvote_workspace_bytes", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
     "gvote_compact", "gvote_pack", "gvote_overlap", "gvote_compress", "gvote_compress_moments", "gvote_recompress", "gvote_compress_host", "gvote_host_arena_release",
-    "gvote_poll_status", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
+    "gvote_poll_status", "gvote_clear_status", "gvote_exact_heads", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
 
 
@@ -97,6 +97,10 @@ def load():
     lib.gvote_host_arena_release.argtypes = []
     lib.gvote_poll_status.restype = i32
     lib.gvote_poll_status.argtypes = [vp, vp]
+    lib.gvote_clear_status.restype = i32
+    lib.gvote_clear_status.argtypes = [vp, vp]
+    lib.gvote_exact_heads.restype = i64
+    lib.gvote_exact_heads.argtypes = [vp, vp]
     lib.gvote_profile_enable.restype = None
     lib.gvote_profile_enable.argtypes = [i32]
     lib.gvote_profile_report.restype = sz
@@ -356,6 +360,16 @@ def gvote_host_arena_release() -> None:
 
 def gvote_poll_status(ws) -> int:
     return int(load().gvote_poll_status(_ptr(ws), _stream()))
+
+
+def gvote_clear_status(ws) -> None:
+    _check(load().gvote_clear_status(_ptr(ws), _stream()), "gvote_clear_status")
+
+
+def gvote_exact_heads(ws) -> int:
+    """(request, KV head) pairs the default mode had to select again by the exact route since the
+    status block was last cleared."""
+    return int(load().gvote_exact_heads(_ptr(ws), _stream()))
 
 
 def gvote_profile_enable(on: bool) -> None:

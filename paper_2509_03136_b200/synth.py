@@ -70,6 +70,8 @@ class GVoteConfig:
     heavy_gain: float = 2.5          # planted rows also carry this multiple of the N(0,1) row
     local_window: int = 0            # last tokens with a weaker planted offset
     local_scale: float = 0.25
+    key_scale: float = 1.0           # standard deviation of an ordinary key row's entries
+    heavy_all_heads: bool = False    # planted keys line up with every query head of the group, not only its first
 
     @property
     def G(self) -> int:
@@ -197,6 +199,11 @@ def make_layer(cfg: GVoteConfig, layer: int = 0, with_bias: bool = False) -> Lay
             var = np.exp(rng.uniform(np.log(0.1), np.log(10.0), size=d_h))
             z *= np.sqrt(var).astype(np.float32)
             z += mu
+        elif cfg.h_mode == "mean":
+            # hidden states that hardly move around a large mean: every query, current or synthetic,
+            # then points almost the same way (the regime in which planted keys have a known fate)
+            z *= np.float32(0.02)
+            z += rng.standard_normal(d_h).astype(np.float32)
         h[a:b] = z
         mean_h = h[a + min(cfg.n_s, max(N - 1, 0)):b].mean(axis=0, dtype=np.float64)
 
@@ -209,8 +216,11 @@ def make_layer(cfg: GVoteConfig, layer: int = 0, with_bias: bool = False) -> Lay
         pos_star = N + 0.5 * (cfg.n_f - 1)
 
         for kh in range(Hkv):
-            Kn = rng.standard_normal((N, d_k), dtype=np.float32)
+            Kn = rng.standard_normal((N, d_k), dtype=np.float32) * np.float32(cfg.key_scale)
             mhat = _planted_direction(W_f32, mean_h, kh * G, d_k, cfg.rope_theta, pos_star)
+            if cfg.heavy_all_heads:
+                for g in range(kh * G + 1, (kh + 1) * G):
+                    mhat = mhat + _planted_direction(W_f32, mean_h, g, d_k, cfg.rope_theta, pos_star)
             # norm of the mean query seen through this head (before rotation; rotation keeps it)
             m_norm = np.linalg.norm(W_f32[kh * G * d_k:(kh * G + 1) * d_k].astype(np.float64) @ mean_h)
             alpha = cfg.heavy_lead * np.sqrt(d_k) / max(m_norm, 1e-12)
@@ -227,6 +237,18 @@ def make_layer(cfg: GVoteConfig, layer: int = 0, with_bias: bool = False) -> Lay
     V = rng.standard_normal((Hkv, T, d_k), dtype=np.float32)
     return LayerInputs(h=h, W_q=W_bits, b_q=b_q, K=f32_to_bf16_bits(K), V=f32_to_bf16_bits(V),
                        cu_seqlens=cu, layer_id=layer, heavy_positions=heavy_positions)
+
+
+def make_planted(n_heavy: int, seed: int = 40, N: int = 600, S: int = 8, p_nuc: float = 0.9,
+                 n_q_heads: int = 4, n_kv_heads: int = 2, d_k: int = 64, d_h: int = 64) -> GVoteConfig:
+    """A workload whose answer is known by construction: hidden states with a dominant mean (all queries
+    nearly parallel), small ordinary keys, and n_heavy planted keys per KV head lined up with every query
+    head of the group, far enough ahead that they hold more than p of every query's attention between
+    them.  The nucleus of every query then lies inside the planted set, and so does every vote."""
+    return GVoteConfig(name=f"planted{n_heavy}", d_h=d_h, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, d_k=d_k,
+                       rope_theta=1.0e4, S=S, p_nuc=p_nuc, seq_lens=(N,), n_f=8, n_s=2, seed=seed, h_mode="mean",
+                       n_outlier_channels=0, heavy_count=n_heavy, heavy_lead=16.0, heavy_norm_cap=1.0e6,
+                       heavy_gain=0.0, key_scale=0.25, heavy_all_heads=True)
 
 
 def make_small(seed: int, d_h: int = 64, n_q_heads: int = 4, n_kv_heads: int = 2, d_k: int = 32,

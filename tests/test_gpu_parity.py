@@ -168,6 +168,7 @@ def _run_vote(gv, cfg, li, Q_or, sel_mode, include_c0, want_probs):
         probs = torch.empty(cfg.n_q_heads * (cfg.S + 1) * cfg.total_tokens, device="cuda")
     gv.gvote_vote(p, Qd, K, cu, geom, mask, budget, b_step, ws, probs)
     assert gv.gvote_poll_status(ws) == 0
+    _run_vote.exact_heads = gv.gvote_exact_heads(ws)
     return mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), None if probs is None else probs.cpu().numpy()
 
 
@@ -251,6 +252,51 @@ def test_vote_topp_long_rows_strict_band(gv, N):
     _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topp", want_probs=False)
 
 
+def test_budget_grows_with_S_and_with_p(gv):
+    """Section 3.5 / Section 4.4: more synthetic queries or a larger nucleus can only add keys.  The samples
+    are counter based, so the first S' draws of an S-run are the S'-run: keep masks are nested in S (bit for
+    bit); budgets do not shrink as p grows; and every setting's budget agrees with the oracle's."""
+    import bench
+    cfg = synth.make_small(23, seq_lens=(700, 333), S=8, d_h=128, n_q_heads=4, n_kv_heads=2, d_k=64, p_nuc=0.9,
+                           heavy_frac=(0.03,))
+    li = synth.make_layer(cfg, 0)
+    d = pu.upload_layer(li, gv, torch)
+    p0 = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p0, *geom)
+    mu = torch.empty(cfg.batch, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p0, d["h"], d["cu"], geom, mu, var, ws)
+    cu = li.cu_seqlens
+    h_last = torch.from_numpy(np.stack([li.h[int(cu[r + 1]) - 1] for r in range(cfg.batch)])).cuda()
+    W = o.bf16_bits_to_f64(li.W_q)
+
+    def oracle_budget(S, pn):
+        out = []
+        for r in range(cfg.batch):
+            a, b = int(cu[r]), int(cu[r + 1])
+            kw = pu.oracle_kwargs(cfg)
+            kw.update(S=S, p_nuc=float(np.float32(pn)))
+            out.append(o.compress_request(li.h[a:b].astype(np.float64), W, li.b_q, o.bf16_bits_to_f64(li.K[:, a:b]),
+                                          request_id=r, **kw).budget)
+        return np.stack(out)
+
+    prev = None
+    for S in (1, 2, 4, 8, 16):
+        mask, budget, ov, _ = bench.select_once(gv, torch, cfg, li, d, S, 0.9, mu, var, h_last, reps=1)
+        if prev is not None:
+            assert np.all((prev & ~mask) == 0)                                  # nested in S
+        prev = mask
+        assert np.all(np.abs(budget - oracle_budget(S, 0.9)) <= 4)
+        assert np.all((ov >= 0) & (ov <= 1 + 1e-5))
+    last = None
+    for pn in (0.5, 0.8, 0.9, 0.97):
+        _, budget, ov, _ = bench.select_once(gv, torch, cfg, li, d, 8, pn, mu, var, h_last, reps=1)
+        if last is not None:
+            assert np.all(budget >= last)                                       # monotone in p
+        last = budget
+        assert np.all(np.abs(budget - oracle_budget(8, pn)) <= 4)
+
+
 def test_vote_degenerate_all_keys_equal(gv):
     """Every logit ties: top-p keeps ceil(p N) keys and top-k keeps exactly k, lowest indices first."""
     cfg = synth.make_small(5, seq_lens=(100,), S=3, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=32, p_nuc=0.5)
@@ -281,10 +327,11 @@ def test_vote_single_dominant_key(gv):
 
 @pytest.mark.parametrize("shift_sampled,shift_sign", [(0.0, 0.0), (-6.0, 0.0), (+6.0, 0.0), (0.0, 1.0)])
 def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
-    """Rows long enough for the sampled one-sweep top-k.  The kernel samples fixed positions (128
-    evenly spaced runs of 32 keys); shifting the logits at exactly those positions makes the sample's
-    bracket miss the true threshold, so the exact route has to take over.  shift_sign = 1 centres
-    the logits on zero with tiny magnitudes (half-precision codes are densest there)."""
+    """Rows long enough for the sampled bracket of the fused top-k.  The kernels sample whole 128-key tiles
+    (one from every stretch of `stride` tiles, at a hashed offset); shifting the logits of exactly those
+    tiles makes the sample's bracket miss the true threshold, so the exact route has to take over.
+    shift_sign = 1 centres the logits on zero with tiny magnitudes (half-precision codes are densest
+    there)."""
     N, d_k, S = 16384, 64, 6
     cfg = synth.make_small(11, seq_lens=(N,), S=S, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=d_k, p_nuc=0.9)
     li = synth.make_layer(cfg, 0)
@@ -293,17 +340,20 @@ def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
     e /= np.linalg.norm(e)
     v = rng.normal(size=N) * (1e-3 if shift_sign else 1.0)
     sampled = np.zeros(N, dtype=bool)
-    nv8 = N // 8
-    stride = nv8 // 128                                  # 128 runs of four 8-key vectors
-    for t in range(128):
-        first = t * stride + ((stride // 2) & ~3)
-        sampled[first * 8:(first + 4) * 8] = True
+    n_tiles = N // 128
+    want = min(max(n_tiles >> 3, 32), 128)               # the sampling plan of the kernels (vote_geom.cuh)
+    stride = n_tiles // want
+    for j in range(want):
+        t = j * stride + (((j * 2654435761) & 0xFFFFFFFF) >> 15) % stride
+        sampled[t * 128:(t + 1) * 128] = True
     v[sampled] += shift_sampled
     Kf = (v[:, None] * e[None, :] * math.sqrt(d_k)).astype(np.float32)[None]          # logit of key n = v_n q.e
     li.K = synth.f32_to_bf16_bits(Kf)
     q = o.round_to_bf16(np.stack([e * (1.0 + 0.05 * r) for r in range(S + 1)]))     # rows differ a little
     Q_or = [np.stack([q, q[::-1].copy()])]
     mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    # a shifted sample makes the bracket miss: the head must have gone the exact way (and only then)
+    assert _run_vote.exact_heads == (1 if shift_sampled else 0), _run_vote.exact_heads
     Kr = o.bf16_bits_to_f64(li.K)
     gm = np.stack([gv.unpack_mask(mask[0], 0, N)])
     pu.check_vote_against_oracle(Q_or[0], Kr, float(np.float32(cfg.p_nuc)), "topk", False, gm, b_step[0])
@@ -463,7 +513,9 @@ def test_pack_varlen_reports_buffers_that_are_too_small(gv):
     assert gv.gvote_poll_status(ws) == -3
     assert cuk.cpu().numpy().tolist() == [0, 600, 1200]
     assert np.array_equal(gv.bits_from_bf16(Kp)[:600], K[0])          # what fits is written
-    ws.zero_()
+    assert gv.gvote_poll_status(ws) == -3                               # the status stays until it is cleared
+    gv.gvote_clear_status(ws)
+    assert gv.gvote_poll_status(ws) == 0
 
 
 # ----------------------------------------------------------------------------- whole pass
@@ -513,6 +565,22 @@ def test_compress_small(gv, idx):
 def test_compress_configs(gv, name, mode):
     cfg = synth.make_config(name)
     _check_compress(gv, cfg, synth.make_layer(cfg, 0), mode)
+
+
+@pytest.mark.parametrize("n_heavy,p_nuc", [(4, 0.99), (12, 0.99), (40, 0.99), (40, 0.9), (120, 0.9)])
+def test_compress_planted_answer(gv, n_heavy, p_nuc):
+    """Inputs whose answer is known by construction (see synth.make_planted): at p = 0.99 the keep mask is
+    exactly the planted positions; at p = 0.9 nothing outside them is kept.  And the oracle agrees."""
+    cfg = synth.make_planted(n_heavy, p_nuc=p_nuc)
+    li = synth.make_layer(cfg, 0)
+    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li)
+    for kh in range(cfg.n_kv_heads):
+        kept = np.nonzero(gv.unpack_mask(mask[kh], 0, cfg.total_tokens))[0]
+        planted = li.heavy_positions[(0, kh)]
+        assert np.isin(kept, planted).all()
+        if p_nuc == 0.99:
+            assert np.array_equal(kept, planted) and budget[0, kh] == n_heavy
+    _check_compress(gv, cfg, li)
 
 
 def _run_compress_bf16_h(gv, cfg, li, sel_mode="topk", layer_id=0):

@@ -711,3 +711,57 @@ def test_recompress_head_with_no_rows():
                                n_f=2, seed=1, layer_id=0, request_id=0, token_pos=[np.arange(9), np.zeros(0, dtype=int)])
     assert res.budget[1] == 0 and res.masks[1].shape == (0,) and res.token_pos[1].shape == (0,)
     assert res.b_step[2] == 0 and res.b_step[3] == 0 and res.budget[0] >= res.b_step[:2].max() > 0
+
+
+# ----------------------------------------------------------------------------- planted structure, end to end
+def _planted_run(n_heavy, p_nuc):
+    from paper_2509_03136_b200 import synth
+    cfg = synth.make_planted(n_heavy, p_nuc=p_nuc)
+    li = synth.make_layer(cfg, 0)
+    res, _, _ = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, n_q_heads=cfg.n_q_heads, d_k=cfg.d_k,
+                                 theta=cfg.rope_theta, S=cfg.S, p_nuc=float(np.float32(cfg.p_nuc)), n_f=cfg.n_f,
+                                 n_s=cfg.n_s, seed=cfg.seed, layer_id=0)
+    return cfg, li, res[0]
+
+
+@pytest.mark.parametrize("n_heavy", [4, 12, 40])
+def test_planted_keys_are_exactly_what_the_pass_keeps(n_heavy):
+    """End to end on inputs whose answer is known by construction (Section 3.3: the union keeps what the
+    queries need).  All queries nearly parallel, n_heavy planted keys per KV head that hold more than
+    99.7 % of every query's attention between them in near-equal shares: with p = 0.99 the nucleus of
+    the current query is the whole planted set, every synthetic query's top-k is that set, and the keep
+    mask is exactly the planted positions - no more, no less."""
+    cfg, li, r = _planted_run(n_heavy, 0.99)
+    assert r.b_step.tolist() == [n_heavy] * cfg.n_q_heads
+    for kh in range(cfg.n_kv_heads):
+        assert np.array_equal(np.nonzero(r.mask[kh])[0], li.heavy_positions[(0, kh)])
+        assert r.budget[kh] == n_heavy
+
+
+def test_budget_tracks_the_planted_count():
+    """Same construction at p = 0.9: near-equal planted weights make the nucleus ceil(0.9 n) of the n planted
+    keys (up to the small spread of their weights), nothing outside the planted set is ever kept, and the
+    budget grows with the planted count: the budget is set by the data, not by a quota."""
+    budgets = []
+    for n_heavy in (4, 12, 40, 120):
+        cfg, li, r = _planted_run(n_heavy, 0.9)
+        for kh in range(cfg.n_kv_heads):
+            kept = np.nonzero(r.mask[kh])[0]
+            assert np.isin(kept, li.heavy_positions[(0, kh)]).all()
+            assert math.ceil(0.9 * n_heavy) <= r.budget[kh] <= n_heavy
+            assert r.budget[kh] >= r.b_step[kh * cfg.G:(kh + 1) * cfg.G].max()       # |union| >= |C| (Section 3.3)
+        budgets.append(int(r.budget.min()))
+    assert budgets == sorted(budgets) and len(set(budgets)) == 4
+
+
+def test_planted_positions_of_the_small_workloads_are_kept():
+    """The heavy positions planted in the two small benchmark workloads are all in the keep mask."""
+    from paper_2509_03136_b200 import synth
+    for name in ("c0", "c1"):
+        cfg = synth.make_config(name)
+        li = synth.make_layer(cfg, 0)
+        res, _, _ = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, n_q_heads=cfg.n_q_heads,
+                                     d_k=cfg.d_k, theta=cfg.rope_theta, S=cfg.S, p_nuc=float(np.float32(cfg.p_nuc)),
+                                     n_f=cfg.n_f, n_s=cfg.n_s, seed=cfg.seed, layer_id=0)
+        for kh in range(cfg.n_kv_heads):
+            assert res[0].mask[kh][li.heavy_positions[(0, kh)]].all()
