@@ -49,8 +49,8 @@ struct SweepTail {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
   uint64_t q_full;
-  uint64_t acc_full[2];
-  uint64_t acc_empty[2];
+  uint64_t acc_full[3];
+  uint64_t acc_empty[3];
   uint64_t real_full[2];
   uint64_t real_empty[2];
   uint32_t tmem_slot;
@@ -382,7 +382,7 @@ template <int CG, int STG>      // STG: logits a thread stages at a time (16, or
 __global__ void __launch_bounds__(kSweepBThreads, 1)
 score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16* __restrict__ Q,
                    const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, int row_chunks, int stages,
-                   float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
+                   int nbuf, float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
                    const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   pdl_trigger();
@@ -399,13 +399,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { ptx::mbar_init(&tail->full[s], 1); ptx::mbar_init(&tail->empty[s], 1); }
     ptx::mbar_init(&tail->q_full, kSweepEpiWarps);
-    for (int a2 = 0; a2 < 2; ++a2) { ptx::mbar_init(&tail->acc_full[a2], 1); ptx::mbar_init(&tail->acc_empty[a2], kSweepEpiWarps); }
+    for (int a2 = 0; a2 < 3; ++a2) { ptx::mbar_init(&tail->acc_full[a2], 1); ptx::mbar_init(&tail->acc_empty[a2], kSweepEpiWarps); }
     tail->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmK);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&tail->tmem_slot, kTmemCols);            // 2 x 128 accumulator columns, then the query rows
+    ptx::tmem_alloc(&tail->tmem_slot, kTmemCols);            // nbuf x 128 accumulator columns, then the query rows
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before_sync();
@@ -421,6 +421,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
   const uint32_t stage_bytes = (uint32_t)kchunks * kTileKeys * 128;
   const int R = G * (S + 1);
   const uint32_t a_cols = (uint32_t)d_k / 2;               // tensor-memory columns of one chunk's query rows
+  const uint32_t a_base = (uint32_t)nbuf * kRowChunk;      // they follow the accumulators
 
   if (warp == 0) {
     if (lane == 0 && walk.count > 0) {
@@ -448,10 +449,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
         ptx::tc_fence_after_sync();
         const uint32_t k_addr = ptx::smem_u32(sm.Ks + (size_t)s * stage_bytes);
         for (int cc = 0; cc < c_cnt; ++cc, ++n1) {
-          const int a = n1 & 1;
-          if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)n1 >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          const int a = n1 % nbuf;
+          if (!wait_or_abort(&tail->acc_empty[a], (((uint32_t)(n1 / nbuf)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint32_t d = tmem_base + (uint32_t)(a * kRowChunk), qa = tmem_base + 256u + (uint32_t)cc * a_cols;
+          const uint32_t d = tmem_base + (uint32_t)(a * kRowChunk), qa = tmem_base + a_base + (uint32_t)cc * a_cols;
           const int ksteps = d_k / 16;
           for (int k = 0; k < ksteps; ++k) {
             const uint32_t koff = (uint32_t)(k >> 2), kin = (uint32_t)(k & 3) * 32u;
@@ -513,7 +514,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
             const uint4 x = grow < G * S ? __ldg(src + (c0 >> 2) + j) : make_uint4(0u, 0u, 0u, 0u);
             w[4 * j] = x.x; w[4 * j + 1] = x.y; w[4 * j + 2] = x.z; w[4 * j + 3] = x.w;
           }
-          ptx::tmem_st_32x32(tmem_base + 256u + (uint32_t)cc * a_cols + c0 + ((uint32_t)(q * 32) << 16), w);
+          ptx::tmem_st_32x32(tmem_base + a_base + (uint32_t)cc * a_cols + c0 + ((uint32_t)(q * 32) << 16), w);
         }
       }
       ptx::tmem_wait_st();
@@ -532,8 +533,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
 #pragma unroll
       for (int cc = 0; cc < CG; ++cc) {
         if (cc >= c_cnt) break;
-        const int a = n1 & 1;
-        wait_or_abort(&tail->acc_full[a], ((uint32_t)n1 >> 1) & 1u, abort_flag);
+        const int a = n1 % nbuf;
+        wait_or_abort(&tail->acc_full[a], ((uint32_t)(n1 / nbuf)) & 1u, abort_flag);
         ++n1;
         ptx::tc_fence_after_sync();
         uint32_t v[32];
@@ -744,7 +745,9 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sweep_kernel", st);
-    launch_pdl(kern, grid, dim3(kSweepBThreads), smem, st, tmK, Q, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, scale, vs, row_words,
+    // accumulators: three when the query rows leave room in the 512 columns of tensor memory, else two
+    const int nbuf = (512 - geo.cg * (d_k / 2)) / kRowChunk >= 3 ? 3 : 2;
+    launch_pdl(kern, grid, dim3(kSweepBThreads), smem, st, tmK, Q, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, nbuf, scale, vs, row_words,
                                              status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_sweep_kernel");
