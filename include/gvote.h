@@ -102,8 +102,8 @@ static inline int64_t gvote_mask_word_offset(int64_t cu_seqlens_r, int32_t r) {
  * (Section 4.4 names the S x N matrix as what runs out of memory beyond 128K context).  GVOTE_SEL_TOPP
  * needs every row's softmax mass and keeps the fp32 logits of all (S+1) x n_q_heads rows:
  * 4 (S+1) n_q_heads total_tokens bytes more.  A call that asks for the softmax rows (dbg_probs) needs the
- * GVOTE_SEL_TOPP size whatever its mode, as do shapes the tensor-core kernels do not take (d_k not a
- * multiple of 64, more than 16 query heads per KV head). */
+ * GVOTE_SEL_TOPP size whatever its mode, as do shapes the fused kernels do not take (d_k other than 64
+ * or 128, more than 16 query heads per KV head): gvote_workspace_bytes accounts for that. */
 GVOTE_API size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
 /* Step 2 of Section 3.2 (the Gaussian fit of Algorithm 1).  mu[r][c], var[r][c] = mean and unbiased variance over rows

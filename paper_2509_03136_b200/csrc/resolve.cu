@@ -489,10 +489,10 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   dim3 grid(p->S, Hq, batch);
   // shared memory: the segments' offsets and the images of the listed keys.  Room for twice the keys a
-  // row is expected to list at most, within 64 KB; a row that lists more goes the exact way.
+  // row is expected to list at most, within 160 KB; a row that lists more goes the exact way.
   (void)max_N;
   int64_t cap_all = (int64_t)vs.lay.segs * (vs.lay.uniform_seg_cap > 0 ? vs.lay.uniform_seg_cap : vs.lay.seg_cap((int)max_N));
-  if (cap_all > 16000) cap_all = 16000;
+  if (cap_all > 40000) cap_all = 40000;
   const int smem_keys = (int)cap_all;
   const size_t smem = ((size_t)vs.lay.segs + 1 + (size_t)smem_keys) * sizeof(uint32_t);
   if (smem > 48 * 1024)

@@ -651,8 +651,10 @@ bool encode_maps(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloa
 
 }  // namespace
 
+// Head dimensions of 64 and 128 (a key tile of 128 x d_k bf16 values, the query rows of a chunk and the
+// staging areas share 227 KB of shared memory with at least two stages), at most 16 query heads per KV head.
 bool sweep_umma_supported(const gvote_params* p) {
-  return p->d_k % 64 == 0 && p->d_k <= 256 && p->n_q_heads / p->n_kv_heads <= kRealCols;
+  return p->d_k % 64 == 0 && p->d_k <= 128 && p->n_q_heads / p->n_kv_heads <= kRealCols;
 }
 
 // First pass.  Returns GVOTE_ERR_UNSUPPORTED_SHAPE when the tensor maps cannot describe the operands (the

@@ -297,6 +297,15 @@ def test_budget_grows_with_S_and_with_p(gv):
         assert np.all(np.abs(budget - oracle_budget(8, pn)) <= 4)
 
 
+@pytest.mark.parametrize("d_k,G", [(256, 2), (192, 1), (64, 17)])
+def test_vote_shapes_outside_the_fused_route(gv, d_k, G):
+    """Head dimensions above 128 and more than 16 query heads per KV head are served by the kernels that keep
+    fp32 rows (the workspace is sized for them): same answers, same bands."""
+    cfg = synth.make_small(24, seq_lens=(300, 1100), S=5, d_h=64, n_q_heads=2 * G, n_kv_heads=2, d_k=d_k, p_nuc=0.9)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
+    _check_compress(gv, cfg, synth.make_layer(cfg, 0))
+
+
 def test_vote_degenerate_all_keys_equal(gv):
     """Every logit ties: top-p keeps ceil(p N) keys and top-k keeps exactly k, lowest indices first."""
     cfg = synth.make_small(5, seq_lens=(100,), S=3, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=32, p_nuc=0.5)
