@@ -1,15 +1,15 @@
 // Algorithm 1, the pruning step: prune K and V to the keep-set, in place.
 //
 // Two kernels.  mask_scan_kernel turns each (request, KV head) bit row into an exclusive popcount
-// prefix per 32-key word and the head's budget.  compact_kernel then moves the kept rows of one
-// 128-token tile per CTA to their destination rows: thread = token, one bulk copy per row into
-// shared memory and one out of it.
+// prefix per 32-key word and the head's budget.  compact_kernel then fills one tile of 128 DESTINATION
+// rows per CTA: thread = destination row, which finds its source row from the prefix, fetches it with
+// one bulk copy into shared memory; the tile is written with one bulk copy.
 //
-// In-place safety.  Row i moves to row prefix(i) <= i, so a tile's destination may still hold
-// rows that an EARLIER tile of the same slab has not read yet.  Each CTA therefore (1) takes a
-// ticket of its slab, which orders tiles so that a lower tile of a slab is always taken by a CTA
-// that is already running, (2) loads its kept rows into shared memory, (3) publishes a "loaded" flag,
-// (4) waits until the (at most two) earlier tiles whose rows its destination range overlaps have
+// In-place safety.  Row i moves to row prefix(i) <= i, so the rows a tile overwrites may still be
+// unread sources of an EARLIER tile of the same slab (never of a later one).  Each CTA therefore
+// (1) takes a ticket of its slab, which orders tiles so that a lower tile of a slab is always taken by a
+// CTA that is already running, (2) loads its rows into shared memory, (3) publishes a "loaded" flag,
+// (4) waits until the (at most two) earlier tiles whose sources lie in the range it overwrites have
 // published theirs, (5) stores.  The wait is bounded: when it runs out the CTA records
 // GVOTE_ERR_TIMEOUT in the workspace status word, skips its stores and returns.
 #include "common.cuh"
@@ -90,29 +90,49 @@ __device__ __forceinline__ int find_request(const int32_t* __restrict__ cu, int 
   return lo;
 }
 
-constexpr int kCompactThreads = kCompactTile;    // one thread per token of the tile
+constexpr int kCompactThreads = kCompactTile;    // one thread per row of the tile
 constexpr int kSpinLimit = 1 << 22;
 
+// Position of the (rank+1)-th kept key of a request: the last mask word whose prefix does not exceed
+// `rank`, then the bit inside it.  `pf` / `m`: the request's prefix and mask words, `words` of them.
+__device__ __forceinline__ int kept_position(const int32_t* __restrict__ pf, const uint32_t* __restrict__ m, int words,
+                                             int rank) {
+  int lo = 0, hi = words - 1;                      // pf[lo] <= rank always (pf[0] = 0)
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (pf[mid] <= rank) lo = mid; else hi = mid - 1;
+  }
+  const int bit = __fns(m[lo], 0, rank - pf[lo] + 1);      // the (rank - pf[lo] + 1)-th set bit of the word
+  return lo * 32 + bit;
+}
+
+// One CTA per 128 DESTINATION rows of a slab (a head's K or V of one request): thread j fetches the row
+// that ends up at row 128 t + j - it finds its source position from the mask's popcount prefix - with one
+// bulk copy into shared-memory slot j, and the tile leaves in one bulk copy (the destination rows are
+// contiguous; with strided rows, one copy per row).  Tiles whose rows all stay where they are (the prefix of
+// the slab up to the first dropped key) move nothing.
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, int64_t tok, int64_t head,
                const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
                const int32_t* __restrict__ cu, const int32_t* __restrict__ budget, int batch, int Hkv, int d_k,
                int64_t row_words, int64_t n_tiles, int32_t* flags, int32_t* ticket, int32_t* status) {
-  extern __shared__ __align__(128) uint8_t rows_sm[];   // [kept rows][d_k * 2 bytes]
+  extern __shared__ __align__(128) uint8_t rows_sm[];   // [128 rows][d_k * 2 bytes], in destination order
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ int s_ticket;
   __shared__ int s_ok;
+  __shared__ int s_moves;
   const int tid = threadIdx.x;
   pdl_trigger();
   pdl_wait();
-  // A CTA belongs to one slab (a head's K or V) by its block index and takes that slab's next tile:
-  // within a slab, a lower tile is always taken by a CTA that is already running.  One counter per
-  // slab (on a line of its own) instead of one for all keeps the atomics from queueing on one address.
+  // A CTA belongs to one slab by its block index and takes that slab's next tile: within a slab, a lower
+  // tile is always taken by a CTA that is already running.  One counter per slab (on a line of its own)
+  // instead of one for all keeps the atomics from queueing on one address.
   const int slabs = 2 * Hkv;
   const int slab = (int)(blockIdx.x % slabs);
   const int h = slab >> 1;
   if (tid == 0) {
     s_ticket = atomicAdd(&ticket[slab * kTicketPitch], 1);
+    s_moves = 0;
     ptx::mbar_init(&s_bar, kCompactThreads);
     ptx::fence_barrier_init();
   }
@@ -122,37 +142,27 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   const int r = batch == 1 ? 0 : find_request(cu, batch, gt);
   const int start = cu[r], N = cu[r + 1] - start;
   const int t = (int)(gt - tile_offset(start, r));
-  const int tiles = (N + kCompactTile - 1) / kCompactTile;
-  if (t >= tiles) return;   // padding slot of the tile list
+  const int kept_all = budget[r * Hkv + h];
+  // tiles beyond the kept rows (and the padding slots of the tile list) have nothing to do, nor has a head
+  // that keeps every key; nobody waits for their flags
+  if (kept_all == N || (int64_t)t * kCompactTile >= kept_all) return;
   __nv_bfloat16* base = ((slab & 1) ? Vp : Kp) + (int64_t)h * head + (int64_t)start * tok;
   int32_t* my_flags = flags + (int64_t)slab * n_tiles + tile_offset(start, r);
+  const int64_t woff = (int64_t)h * row_words + mask_word_offset(start, r);
+  const int words = (N + 31) >> 5;
+  const int dst0 = t * kCompactTile;
+  const int cnt = min(kCompactTile, kept_all - dst0);
 
-  // the tile's four mask words and its destination offset: every load below is issued before the
-  // first of them is needed
-  const int64_t woff = (int64_t)h * row_words + mask_word_offset(start, r) + (int64_t)t * (kCompactTile / 32);
-  const int words = min(kCompactTile / 32, ((N + 31) >> 5) - t * (kCompactTile / 32));
-  const int w_mine = min(tid >> 5, words - 1), lastw = words - 1;
-  const int kept_all = budget[r * Hkv + h];
-  const int dst0 = prefix[woff];
-  const uint32_t mw = mask[woff + w_mine];
-  const int pw = prefix[woff + w_mine];
-  const int p_last = prefix[woff + lastw];
-  const uint32_t m_last = mask[woff + lastw];
-  // a head that keeps every key moves nothing, and none of its tiles waits for another
-  if (kept_all == N) return;
-  const int cnt = p_last - dst0 + __popc(m_last);
-
-  // Thread = token.  A kept token whose destination differs from its source (the rows that stay
-  // put form a prefix of the slab) is fetched with one bulk copy of the whole row into the slot of
-  // its rank; every thread arrives on the mbarrier, the fetching ones with their byte count.
+  // thread = destination row: where does it come from?
   const uint32_t row_bytes = (uint32_t)d_k * 2u;
-  const int b = tid & 31;
-  const bool kept = (tid >> 5) < words && ((mw >> b) & 1u);
-  const int rank = (pw - dst0) + __popc(mw & ((1u << b) - 1u));
-  const int src = t * kCompactTile + tid;
-  const bool moves = kept && src != dst0 + rank;
-  uint8_t* slot = rows_sm + (size_t)rank * row_bytes;
-  if (moves) {
+  const bool have = tid < cnt;
+  int src = -1;
+  if (have) src = kept_position(prefix + woff, mask + woff, words, dst0 + tid);
+  if (have && src != dst0 + tid) s_moves = 1;              // (same value from every writer)
+  __syncthreads();
+  const bool tile_moves = s_moves != 0;
+  uint8_t* slot = rows_sm + (size_t)tid * row_bytes;
+  if (have && tile_moves) {
     ptx::mbar_arrive_expect_tx(&s_bar, row_bytes);
     ptx::bulk_load(slot, base + (int64_t)src * tok, row_bytes, &s_bar);
   } else {
@@ -164,17 +174,25 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   if (tid == 0) {
     __threadfence();
     atomicExch(&my_flags[t], 1);                    // our source rows are safe in shared memory
-    // destination rows [dst0, dst0+cnt) live in tiles ta..tb (<= t); wait for those below t
+    // The rows [dst0, dst0 + cnt) we are about to overwrite are sources of the tiles that hold the ranks of
+    // the kept keys among positions dst0 .. dst0 + 127: tiles ta .. tb (at most two, none above t).  Wait
+    // for those below t to have loaded.
     int ok = 1;
-    if (cnt > 0) {
-      const int ta = dst0 / kCompactTile, tb = (dst0 + cnt - 1) / kCompactTile;
-      for (int w = ta; w <= tb && w < t; ++w) {
-        int spins = 0;
-        while (atomicAdd(&my_flags[w], 0) == 0) {
-          if (++spins > kSpinLimit) { ok = 0; break; }
-          __nanosleep(64);
+    if (tile_moves) {
+      const int w0 = dst0 >> 5;                                         // word of position dst0 (dst0 < N here)
+      const int w1 = min(w0 + kCompactTile / 32, words) - 1;            // last word of the 128 positions
+      const int r0 = prefix[woff + w0];
+      const int r1 = prefix[woff + w1] + __popc(mask[woff + w1]);       // ranks [r0, r1) live at those positions
+      if (r1 > r0) {
+        const int ta = r0 / kCompactTile, tb = (r1 - 1) / kCompactTile;
+        for (int w = ta; w <= tb && w < t; ++w) {
+          int spins = 0;
+          while (atomicAdd(&my_flags[w], 0) == 0) {
+            if (++spins > kSpinLimit) { ok = 0; break; }
+            __nanosleep(64);
+          }
+          if (!ok) break;
         }
-        if (!ok) break;
       }
       if (!ok) { atomicExch(&status[0], GVOTE_ERR_TIMEOUT); atomicExch(&status[1], 1); }
       __threadfence();
@@ -183,11 +201,18 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   }
   if (!landed) { atomicExch(&status[0], GVOTE_ERR_TIMEOUT); atomicExch(&status[1], 4); }
   __syncthreads();
-  if (!s_ok || !landed) return;
-  if (moves) {
-    ptx::bulk_store(base + (int64_t)(dst0 + rank) * tok, slot, row_bytes);
+  if (!s_ok || !landed || !tile_moves) return;
+  if (tok == d_k) {                                 // dense rows: the tile leaves in one copy
+    if (tid == 0) {
+      ptx::fence_proxy_async();
+      ptx::bulk_store(base + (int64_t)dst0 * tok, rows_sm, (uint32_t)cnt * row_bytes);
+      ptx::bulk_commit();
+      ptx::bulk_wait_read<0>();                     // shared memory must outlive the copy's reads
+    }
+  } else if (have) {
+    ptx::bulk_store(base + (int64_t)(dst0 + tid) * tok, slot, row_bytes);
     ptx::bulk_commit();
-    ptx::bulk_wait_read<0>();                       // shared memory must outlive the copy's reads
+    ptx::bulk_wait_read<0>();
   }
 }
 
