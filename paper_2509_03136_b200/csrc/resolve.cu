@@ -71,7 +71,8 @@ __device__ __forceinline__ void warp_find_bin256(const uint32_t* hist, uint32_t 
 // the keys whose high byte is the one found, for the two ranks side by side.  Integer counts only: the
 // same bits on every run.
 constexpr int kBrThreads = 128;
-constexpr int kBrVecs = 16;     // 16-byte vectors of sampled keys per thread: 128 * 16 * 8 = 16384 keys at most
+// (NV: 16-byte vectors of sampled keys a thread holds: 4 for samples of up to 4096 keys - fewer registers,
+// twice the CTAs per SM - and 16 for the largest, 128 * 16 * 8 = 16384 keys)
 
 // High byte of a key's code from the high byte hb of its half bits.
 __device__ __forceinline__ uint32_t ord_hi(uint32_t hb) { return hb >= 0x80u ? 0xffu - hb : 0x80u + hb; }
@@ -84,6 +85,7 @@ struct BracketShared {
   uint32_t above[2];
 };
 
+template <int NV>
 __global__ void __launch_bounds__(kBrThreads)
 bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const int32_t* __restrict__ cu, int Hq,
                int G, int S, int row_chunks, const int32_t* __restrict__ b_step, RowBracket* __restrict__ bracket,
@@ -112,16 +114,18 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
   const int64_t slot_stride = (int64_t)row_chunks * kVoteRowChunk * kVoteTileKeys;
   const uint16_t* base = sample + ((((int64_t)kh * sample_slots + sample_slot_offset(start, r)) * row_chunks + chunk) *
                                    kVoteRowChunk + crow) * kVoteTileKeys;
-  uint4 v[kBrVecs];
+  uint4 v[NV];
   const int n_vecs = geo.ns * 16;
   const int have = (n_vecs + kBrThreads - 1) / kBrThreads;   // the same for every thread of the CTA
 #pragma unroll
-  for (int u = 0; u < kBrVecs; ++u) {
+  for (int u = 0; u < NV; ++u) {
     const int i = u * kBrThreads + tid;
     v[u] = make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u);     // -inf: below every rank asked for
     if (u < have && i < n_vecs) v[u] = *reinterpret_cast<const uint4*>(base + (int64_t)(i >> 4) * slot_stride + (i & 15) * 8);
   }
-  for (int i = tid; i < 128 * 32; i += kBrThreads) sh.lanes[i] = 0;     // (while the loads are in flight)
+  const bool small = have <= 2;                            // the same for every thread of the CTA
+  if (small) { for (int i = tid; i < 256; i += kBrThreads) sh.bins[i] = 0; }
+  else { for (int i = tid; i < 128 * 32; i += kBrThreads) sh.lanes[i] = 0; }     // (while the loads are in flight)
   for (int i = tid; i < 512; i += kBrThreads) sh.low[i] = 0;
   // ranks (1-based, among the sampled keys; the pad counts as -inf keys) whose keys become the bounds
   const int m = sample_keys(geo, N);
@@ -139,8 +143,23 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
   }
   __syncthreads();
   // ---- level 1
+  if (small) {
+    // a sample of at most 2048 keys: plain atomics on the 256 bins queue little, and nothing has to be folded
+    for (int u = 0; u < 2; ++u) {
+      if (u >= have) break;
+      const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
-  for (int u = 0; u < kBrVecs; ++u) {
+      for (int j = 0; j < 4; ++j) {
+        uint32_t h0 = w[j] & 0xffffu, h1 = w[j] >> 16;
+        if (h0 == 0x8000u) h0 = 0u;
+        if (h1 == 0x8000u) h1 = 0u;
+        atomicAdd(&sh.bins[ord_hi(h0 >> 8)], 1u);
+        atomicAdd(&sh.bins[ord_hi(h1 >> 8)], 1u);
+      }
+    }
+  } else {
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
     if (u >= have) break;
     const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
@@ -152,8 +171,9 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
       atomicAdd(&sh.lanes[(h1 >> 9) * 32 + lane], 1u << ((h1 >> 4) & 16u));
     }
   }
+  }
   __syncthreads();
-  {
+  if (!small) {
     // thread t sums word row t (raw high bytes 2t, 2t+1) over the lanes, starting at its own lane: no conflicts
     uint32_t acc = 0;
     const uint32_t* wrow = &sh.lanes[tid * 32];
@@ -180,7 +200,7 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
     const uint32_t raw_lo = bin_lo < 0x80u ? 0xffu - bin_lo : bin_lo - 0x80u, flip_lo = bin_lo < 0x80u ? 0xffu : 0u;
     const uint32_t raw_hi = bin_hi < 0x80u ? 0xffu - bin_hi : bin_hi - 0x80u, flip_hi = bin_hi < 0x80u ? 0xffu : 0u;
 #pragma unroll
-    for (int u = 0; u < kBrVecs; ++u) {
+    for (int u = 0; u < NV; ++u) {
       if (u >= have) break;
       const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
@@ -221,7 +241,7 @@ constexpr int kRowThreads = 256;
 struct ResolveShared {
   uint32_t hist[256];
   uint32_t red[2][kRowThreads / 32];
-  uint32_t seg_off[kRowThreads / 32];   // scan scratch
+  uint32_t seg_off[kRowThreads / 32];   // scan scratch  (sized for the larger of the two CTA sizes)
   uint32_t total_above, total_cand, overflow;
   uint32_t kmin, kmax;
   int bin;
@@ -233,7 +253,10 @@ struct ResolveShared {
 // the sweep); their order-preserving 32-bit images are gathered into shared memory and the threshold is
 // found by a most-significant-digit radix search over them (256 bins per pass, starting at the first bit
 // in which the images differ); integer counts only, so two runs give the same bits.
-__global__ void __launch_bounds__(kRowThreads)
+// NT threads per CTA: 256 for long rows, 64 where a row lists at most a couple of thousand candidates (a
+// batch of short requests has many rows and little work in each: what counts there is CTAs per SM).
+template <int NT>
+__global__ void __launch_bounds__(NT)
 resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32_t* __restrict__ b_step,
                const VoteState vs, int smem_keys, int64_t row_words, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint32_t dyn[];         // [seg offsets: segs + 1][keys: smem_keys]
@@ -258,7 +281,7 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
   {
     const uint2* st = vs.segstat + (int64_t)rowid * segs;
     uint32_t run = 0;                                      // candidates in the segments before this round
-    for (int base = 0; base < segs; base += kRowThreads) {
+    for (int base = 0; base < segs; base += NT) {
       const int i = base + tid;
       const uint2 v = i < segs ? st[i] : make_uint2(0u, 0u);
       if (v.y > (uint32_t)seg_cap) sh.overflow = 1u;
@@ -274,7 +297,7 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
       __syncthreads();
       uint32_t before = run, all = 0;
 #pragma unroll
-      for (int w = 0; w < kRowThreads / 32; ++w) { if (w < warp) before += sh.seg_off[w]; all += sh.seg_off[w]; }
+      for (int w = 0; w < NT / 32; ++w) { if (w < warp) before += sh.seg_off[w]; all += sh.seg_off[w]; }
       if (i < segs) seg_off[i] = before + inc - v.y;
       run += all;
       __syncthreads();
@@ -294,7 +317,7 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
   uint32_t* mrow = vs.tmask + (int64_t)kh * row_words + mask_word_offset(start, r);
   // one warp per segment, a lane per entry
   if (need == C) {                                         // every listed key is taken
-    for (int sg = warp; sg < segs; sg += kRowThreads / 32) {
+    for (int sg = warp; sg < segs; sg += NT / 32) {
       const uint32_t cnt = seg_off[sg + 1] - seg_off[sg];
       for (uint32_t i = lane; i < cnt; i += 32) {
         const uint32_t n = list[(int64_t)sg * seg_cap + i].y;
@@ -317,16 +340,16 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
   // gather the order-preserving images of the listed logits
   {
     uint32_t mn = 0xffffffffu, mx = 0u;
-    for (uint32_t base = 0; base < C; base += 4 * kRowThreads) {
+    for (uint32_t base = 0; base < C; base += 4 * NT) {
       uint32_t x[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t e = base + u * kRowThreads + tid;
+        const uint32_t e = base + u * NT + tid;
         x[u] = e < C ? entry_of(e)->x : 0u;
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t e = base + u * kRowThreads + tid;
+        const uint32_t e = base + u * NT + tid;
         if (e < C) {
           const uint32_t kx = ordered_key(__uint_as_float(x[u]));
           keys[e] = kx;
@@ -352,9 +375,9 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
     while (top >= 0) {
       const int lo_bit = top >= 7 ? top - 7 : 0;
       const uint32_t digit_mask = (top - lo_bit == 31) ? 0xffffffffu : (((2u << (top - lo_bit)) - 1u));
-      sh.hist[tid] = 0;
+      for (int i = tid; i < 256; i += NT) sh.hist[i] = 0;
       __syncthreads();
-      for (uint32_t i = tid; i < C; i += kRowThreads) {
+      for (uint32_t i = tid; i < C; i += NT) {
         const uint32_t x = keys[i];
         if ((x & known) == prefix) atomicAdd(&sh.hist[(x >> lo_bit) & digit_mask], 1u);
       }
@@ -386,7 +409,7 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
     for (int bit = 31 - __clz(max(N - 1, 1)); bit >= 0; --bit) {
       const uint32_t trial = vlim | (1u << bit);
       uint32_t c = 0;
-      for (int sg = warp; sg < segs; sg += kRowThreads / 32) {
+      for (int sg = warp; sg < segs; sg += NT / 32) {
         const uint32_t o = seg_off[sg], cnt = seg_off[sg + 1] - o;
         for (uint32_t i = lane; i < cnt; i += 32)
           c += (keys[o + i] == prefix && list[(int64_t)sg * seg_cap + i].y < trial) ? 1u : 0u;
@@ -397,18 +420,18 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
       __syncthreads();
       uint32_t tot = 0;
 #pragma unroll
-      for (int w = 0; w < kRowThreads / 32; ++w) tot += row[w];
+      for (int w = 0; w < NT / 32; ++w) tot += row[w];
       if (tot < ties) vlim = trial;
     }
     idx_max = vlim;
   }
   const bool all_of_bin = whole_bin || ties >= eq;
-  for (uint32_t base = 0; base < C; base += 4 * kRowThreads) {
+  for (uint32_t base = 0; base < C; base += 4 * NT) {
     uint32_t n[4];
     bool want[4], tie[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const uint32_t e = base + u * kRowThreads + tid;
+      const uint32_t e = base + u * NT + tid;
       const uint32_t x = e < C ? keys[e] : 0u;
       const bool in_bin = e < C && (x & known) == prefix;
       want[u] = e < C && (x > (prefix | ~known) || (in_bin && all_of_bin));
@@ -471,14 +494,18 @@ commit_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restri
 }  // namespace
 
 // The three launchers: before the sweep, after it, and the commit.
-int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs,
-                       const int32_t* kv_len, cudaStream_t st) {
+int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, int64_t max_N, const int32_t* b_step,
+                       const VoteState& vs, const int32_t* kv_len, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   dim3 grid(p->S, Hq, batch);
   {
     LaunchScope scope_("bracket_kernel", st);
-    launch_pdl(bracket_kernel, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S, score_geometry(p).row_chunks,
-                                                b_step, vs.bracket, kv_len);
+    if (sample_geom((int)max_N).ns * 16 <= 4 * kBrThreads)
+      launch_pdl(bracket_kernel<4>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
+                 score_geometry(p).row_chunks, b_step, vs.bracket, kv_len);
+    else
+      launch_pdl(bracket_kernel<16>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
+                 score_geometry(p).row_chunks, b_step, vs.bracket, kv_len);
   }
   GVOTE_LAUNCH_CHECK("bracket_kernel");
   return GVOTE_OK;
@@ -496,10 +523,13 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
   const int smem_keys = (int)cap_all;
   const size_t smem = ((size_t)vs.lay.segs + 1 + (size_t)smem_keys) * sizeof(uint32_t);
   if (smem > 48 * 1024)
-    GVOTE_CUDA_CHECK(cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    GVOTE_CUDA_CHECK(cudaFuncSetAttribute(resolve_kernel<kRowThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("resolve_kernel", st);
-    launch_pdl(resolve_kernel, grid, dim3(kRowThreads), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
+    if (smem_keys <= 4096)
+      launch_pdl(resolve_kernel<64>, grid, dim3(64), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
+    else
+      launch_pdl(resolve_kernel<kRowThreads>, grid, dim3(kRowThreads), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
   }
   GVOTE_LAUNCH_CHECK("resolve_kernel");
   return GVOTE_OK;

@@ -236,8 +236,8 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
                            int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                            const VoteState& vs, int64_t row_words, int32_t* status, const int32_t* kv_len,
                            cudaStream_t st);
-int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs,
-                       const int32_t* kv_len, cudaStream_t st);
+int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, int64_t max_N, const int32_t* b_step,
+                       const VoteState& vs, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, int64_t max_N, const int32_t* b_step,
                        const VoteState& vs, int64_t row_words, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
@@ -286,7 +286,7 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
   if (rc != GVOTE_OK) return rc;
 #define GVOTE_STEP(expr) do { const int32_t rc__ = (expr); if (rc__ != GVOTE_OK) return rc__; } while (0)
   GVOTE_STEP(launch_real_topp(p, real_logits, cu, batch, max_N, rowmax, n_part, m.row_words, mask, b_step, kv_len, st));
-  GVOTE_STEP(launch_bracket(p, cu, batch, b_step, vs, kv_len, st));
+  GVOTE_STEP(launch_bracket(p, cu, batch, max_N, b_step, vs, kv_len, st));
   GVOTE_STEP(launch_score_sweep(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, vs, m.row_words, status, kv_len,
                                 st));
   GVOTE_STEP(launch_resolve(p, cu, batch, max_N, b_step, vs, m.row_words, kv_len, st));
