@@ -2,7 +2,7 @@
 //
 //   bracket_kernel   before the sweep: two order statistics of a row's sampled half-precision keys that
 //                    enclose its k-th largest logit (k = B_step of the row's query head), as fp32 bounds
-//                    [lo, hi]; also clears the row's counters.
+//                    [lo, hi].
 //   resolve_kernel   after the sweep: a row whose bracket held (#above <= k <= #above + #listed, list not
 //                    overflowed) takes the k - #above largest of its listed candidates by (fp32 logit
 //                    descending, key index ascending) and ORs them into the tentative mask; a row whose
@@ -12,9 +12,8 @@
 //                    again by the exact route (fp32 logits recomputed from Q and K, radix search over the
 //                    row, no sample involved), so a missed bracket costs time, never correctness.
 //
-// Order statistics are found by bisection on an order-preserving integer image of the values: one
-// count over the thread's elements and one block-wide sum per bit, no sorting, no atomics, the same
-// bits on every run.
+// Order statistics are found by radix searches over order-preserving integer images of the values
+// (histograms of integer counts: no sorting, and the same bits on every run).
 #include <cuda_fp16.h>
 
 #include "select_common.cuh"

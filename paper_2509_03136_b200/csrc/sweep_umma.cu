@@ -11,17 +11,19 @@
 //       row, from which bracket_kernel takes two order statistics [lo, hi] that enclose the row's k-th
 //       largest logit.
 //   score_sweep_kernel   second pass.  Every tile, every row chunk.  The read-out thread of a row holds
-//       64 consecutive logits of its row in registers and compares them with the row's own bracket:
+//       32 consecutive logits of its row in registers and compares them with the row's own bracket:
 //       keys above hi are certainly among the k largest - their bits are OR-ed over the 32 rows of the
 //       warp and then into the head's tentative mask (the union step), and counted per row; keys
-//       inside [lo, hi] are appended, as (fp32 logit, index), to the row's short candidate list.
-//       Nothing else leaves the SM.  resolve_kernel later picks the k - #above largest candidates.
+//       inside [lo, hi] are appended, as (fp32 logit, index), to the thread's own segment of the row's
+//       short candidate list.  Nothing else leaves the SM.  resolve_kernel later picks the k - #above
+//       largest candidates.
 //
-// A CTA holds the query rows of up to four 128-row chunks in shared memory and walks the key tiles
-// x, x+X, ... of one (request, KV head): a tile is fetched once (TMA, 128-byte swizzle) and multiplied
-// with every chunk.  warp 0: TMA producer; warp 1: tensor-memory allocation and tcgen05.mma issue;
-// warps 2-9: read-out, two warps per lane quadrant, each 64 of the tile's 128 keys.  Accumulators are
-// double buffered so that the MMAs of one product overlap the read-out of the one before.
+// A CTA walks the key tiles x, x+X, ... of one (request, KV head): a tile is fetched once (TMA, 128-byte
+// swizzle) and multiplied with up to four 128-row chunks of query rows.  warp 0: TMA producer; warp 1:
+// tensor-memory allocation and tcgen05.mma issue; the other warps: read-out (first pass: two per lane
+// quadrant, 64 keys each; second pass: four per quadrant, 32 keys each).  The first pass keeps the query
+// rows in shared memory; the second keeps them in tensor memory, as the MMA's A operand.  Accumulators
+// are double or triple buffered so that the MMAs of one product overlap the read-out of the one before.
 //
 // Every wait on an mbarrier is bounded.  When one runs out the CTA raises a shared abort flag and
 // records GVOTE_ERR_TIMEOUT in the workspace status word; the remaining waits then give up at once,
