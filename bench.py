@@ -400,6 +400,8 @@ def main():
     launches = gv.gvote_launch_count() - n0
     for w in ws_s:
         assert gv.gvote_poll_status(w) == 0, "a device-side wait timed out"
+    # (request, KV head) pairs that had to be selected again by the exact route (warm-up and timed steps)
+    exact_heads = sum(gv.gvote_exact_heads(w) for w in ws_s)
     total_ms = shard.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
     value = shard.job_throughput(cfg.total_tokens, world, ms_per_step * 1e-3)
@@ -686,7 +688,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, args),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "exact_route_heads": int(exact_heads),
+            "roofline": roofline,
             "cpu_baseline": cpu_baseline, "pass_roofline": pass_roofline, "one_stream_row": one_stream_row,
             "upstream_fit_row": upstream, "recompress_row": recompress, "bf16_h_row": bf16_row, "kernels": per_kernel,
             "setup_s": {"generate": t_gen},
