@@ -44,8 +44,9 @@ constexpr int kRealCols = 16;     // current-query rows per KV head the thin pro
 constexpr int kEpiWarps = 8;
 constexpr int kSweepThreads = 64 + 32 * kEpiWarps;
 constexpr int kMaxStages = 6;
-constexpr int kTmemCols = 512;    // 2 x 128 (D1) + 2 x 32 (D2, 16 used)
+constexpr int kTmemCols = 512;    // first pass: 2 x 128 (D1) + 8 x 32 (D2, 16 used)
 constexpr int kD2Col = 256;
+constexpr int kD2Bufs = 8;        // thin accumulators in flight: the MMA of a tile never waits for a read-out
 
 struct SweepTail {
   uint64_t full[kMaxStages];
@@ -53,8 +54,8 @@ struct SweepTail {
   uint64_t q_full;
   uint64_t acc_full[3];
   uint64_t acc_empty[3];
-  uint64_t real_full[2];
-  uint64_t real_empty[2];
+  uint64_t real_full[kD2Bufs];
+  uint64_t real_empty[kD2Bufs];
   uint32_t tmem_slot;
   volatile int abort_flag;
   uint32_t rowmax[kRealCols];         // running maximum (order-preserving image) of each current-query row
@@ -127,6 +128,8 @@ __device__ __forceinline__ void setup(SweepTail* tail, int stages, const CUtenso
     for (int a2 = 0; a2 < 2; ++a2) {
       ptx::mbar_init(&tail->acc_full[a2], 1);
       ptx::mbar_init(&tail->acc_empty[a2], kEpiWarps);
+    }
+    for (int a2 = 0; a2 < kD2Bufs; ++a2) {
       ptx::mbar_init(&tail->real_full[a2], 1);
       ptx::mbar_init(&tail->real_empty[a2], kEpiWarps / 2);
     }
@@ -239,8 +242,8 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t k_addr = ptx::smem_u32(sm.Ks + (size_t)s * stage_bytes);
         if (it >= walk.n_samp) {
           const int is = it - walk.n_samp;                 // streamed tiles so far
-          const int ar = is & 1;
-          if (!wait_or_abort(&tail->real_empty[ar], (((uint32_t)is >> 1) & 1u) ^ 1u, abort_flag)) break;
+          const int ar = is % kD2Bufs;
+          if (!wait_or_abort(&tail->real_empty[ar], (((uint32_t)(is / kD2Bufs)) & 1u) ^ 1u, abort_flag)) break;
           ptx::tc_fence_after_sync();
           const uint32_t d2 = tmem_base + (uint32_t)(kD2Col + ar * 32);
           const int ksteps = d_k / 16;
@@ -277,8 +280,8 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       // ---- current-query rows: thread = key, exact fp32 logits and their running maximum
       if (it >= walk.n_samp && half == 0) {
         const int is = it - walk.n_samp;
-        const int ar = is & 1;
-        const bool got = wait_or_abort(&tail->real_full[ar], ((uint32_t)is >> 1) & 1u, abort_flag);
+        const int ar = is % kD2Bufs;
+        const bool got = wait_or_abort(&tail->real_full[ar], ((uint32_t)(is / kD2Bufs)) & 1u, abort_flag);
         ptx::tc_fence_after_sync();
         uint32_t w[16];
         ptx::tmem_ld_32x16(tmem_base + (uint32_t)(kD2Col + ar * 32) + ((uint32_t)(q * 32) << 16), w);
