@@ -243,6 +243,18 @@ def test_vote_many_row_chunks_strict_band(gv):
     _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
 
 
+@pytest.mark.parametrize("lens", [(4097,), (4224, 8191, 127), (4096, 2, 3, 129), (12345,)])
+def test_vote_lengths_around_the_sampling_switch(gv, lens):
+    """Rows of exactly 32 key tiles are still sampled completely, 33 tiles are the first sampled in part
+    (stride 1: every full tile, the ragged one left out); ragged batches mix both kinds, two-key and three-key
+    requests included.  G = 3 heads of S = 50 synthetic queries give 150 rows per KV head: a second row chunk
+    that is mostly empty.  Oracle's queries, default 1e-3 bands."""
+    cfg = synth.make_small(25, seq_lens=lens, S=50, d_h=64, n_q_heads=6, n_kv_heads=2, d_k=64, p_nuc=0.93,
+                           heavy_frac=(0.02,), n_s=0)
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
+    assert _run_vote.exact_heads == 0
+
+
 @pytest.mark.parametrize("N", [33000, 50001])
 def test_vote_topp_long_rows_strict_band(gv, N):
     """Per-sample top-p on rows of more than 32K keys (N = 50001 no longer fits the shared-memory
