@@ -243,6 +243,17 @@ def test_vote_many_row_chunks_strict_band(gv):
     _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
 
 
+@pytest.mark.parametrize("lens", [(3000,), (9001, 700)])
+def test_vote_more_row_chunks_than_one_cta_holds(gv, lens):
+    """S = 330 synthetic queries for each of 2 heads per KV head: 660 rows, six 128-row chunks, more than the
+    four a CTA of the second pass holds (two chunk groups there, three in the first pass), the last chunk
+    partly empty.  Oracle's queries, default 1e-3 bands."""
+    cfg = synth.make_small(26, seq_lens=lens, S=330, d_h=64, n_q_heads=4, n_kv_heads=2, d_k=128, p_nuc=0.9,
+                           heavy_frac=(0.01,))
+    _check_vote(gv, cfg, synth.make_layer(cfg, 0), "topk", want_probs=False)
+    assert _run_vote.exact_heads == 0
+
+
 @pytest.mark.parametrize("lens", [(4097,), (4224, 8191, 127), (4096, 2, 3, 129), (12345,)])
 def test_vote_lengths_around_the_sampling_switch(gv, lens):
     """Rows of exactly 32 key tiles are still sampled completely, 33 tiles are the first sampled in part
