@@ -43,22 +43,15 @@ struct LaunchScope {
     }                                                            \
   } while (0)
 
-// Launch with programmatic dependent launch: the kernel may start (up to its pdl_wait) while the kernel
-// before it on the stream is still running, so that its prologue - barrier set-up, tensor-memory
-// allocation, descriptor prefetch - and the launch latency hide under the predecessor's tail.
+// One kernel launch on a stream (typed: the arguments are converted to the kernel's parameter types).
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                              Args&&... args) {
+inline cudaError_t launch_on(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -178,14 +171,6 @@ int32_t launch_overlap(const gvote_params* p, const __nv_bfloat16* Q, const __nv
 
 // ---------------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
-
-// Programmatic dependent launch, device side.  pdl_trigger: the next kernel on the stream may begin to
-// launch (called first thing: what it may touch before its own pdl_wait is only its shared and tensor
-// memory).  pdl_wait: every kernel before this one on the stream has completed and its writes are
-// visible; nothing a predecessor writes or reads may be touched before it.  Both do nothing in a kernel
-// launched the ordinary way.
-__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Monotone map from float to uint32: a > b  <=>  key(a) > key(b)  (no NaNs expected).
 __device__ __forceinline__ uint32_t ordered_key(float f) {

@@ -29,8 +29,6 @@ mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ 
                  int64_t n_tiles, int32_t* __restrict__ ticket) {
   __shared__ int warp_tot[kScanThreads / 32];
   __shared__ int carry;
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.y, h = blockIdx.x;
   const int start = cu[r], N = cu[r + 1] - start;
   const int words = (N + 31) >> 5;
@@ -122,8 +120,6 @@ compact_kernel(__nv_bfloat16* __restrict__ Kp, __nv_bfloat16* __restrict__ Vp, i
   __shared__ int s_ok;
   __shared__ int s_moves;
   const int tid = threadIdx.x;
-  pdl_trigger();
-  pdl_wait();
   // A CTA belongs to one slab by its block index and takes that slab's next tile: within a slab, a lower
   // tile is always taken by a CTA that is already running.  One counter per slab (on a line of its own)
   // instead of one for all keeps the atomics from queueing on one address.
@@ -257,7 +253,7 @@ int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int3
   dim3 gs(Hkv, batch);
   {
     LaunchScope scope_("mask_scan_kernel", st);
-    launch_pdl(mask_scan_kernel, gs, dim3(kScanThreads), 0, st, mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
+    launch_on(mask_scan_kernel, gs, dim3(kScanThreads), 0, st, mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
   }
   GVOTE_LAUNCH_CHECK("mask_scan_kernel");
   return GVOTE_OK;
@@ -279,7 +275,7 @@ int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V
   const int64_t ctas = m.n_tiles * 2 * Hkv;
   {
     LaunchScope scope_("compact_kernel", st);
-    launch_pdl(compact_kernel, dim3((unsigned)ctas), dim3(kCompactThreads), smem, st, K, V, tok, head, mask, prefix, cu, budget, batch, Hkv,
+    launch_on(compact_kernel, dim3((unsigned)ctas), dim3(kCompactThreads), smem, st, K, V, tok, head, mask, prefix, cu, budget, batch, Hkv,
                                                                   p->d_k, m.row_words, m.n_tiles, flags, ticket, status);
   }
   GVOTE_LAUNCH_CHECK("compact_kernel");

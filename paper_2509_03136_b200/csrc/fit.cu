@@ -75,7 +75,6 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int col0 = blockIdx.x * kFitStripCols;
   const int width = min(kFitStripCols, d_h - col0);
-  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], kFitConsumers / 32); }
     abort_flag = 0;
@@ -83,7 +82,6 @@ fit_partial_kernel(const __grid_constant__ CUtensorMap tmH, const T* __restrict_
     ptx::prefetch_tensormap(&tmH);
   }
   __syncthreads();
-  pdl_wait();               // the hidden states may be the output of the kernel before this one on the stream
   int a, b;
   fit_chunk_rows(cu[r] + n_s, cu[r + 1], chunks, c, a, b);
   const int n_it = (b > a) ? (b - a + R - 1) / R : 0;
@@ -288,11 +286,11 @@ int32_t launch_fit_partial(const gvote_params* p, const void* h, int64_t ld, con
     LaunchScope scope_("fit_partial_kernel", st);
     if (p->h_dtype == GVOTE_DTYPE_F32) {
       GVOTE_CUDA_CHECK(cudaFuncSetAttribute(fit_partial_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      launch_pdl(fit_partial_kernel<float>, grid, dim3(kFitThreads), smem, st, tmH, (const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks,
+      launch_on(fit_partial_kernel<float>, grid, dim3(kFitThreads), smem, st, tmH, (const float*)h, ld, cu, p->n_s, p->d_h, fit_chunks,
                                                                  stages, partial, status);
     } else {
       GVOTE_CUDA_CHECK(cudaFuncSetAttribute(fit_partial_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      launch_pdl(fit_partial_kernel<__nv_bfloat16>, grid, dim3(kFitThreads), smem, st, tmH, (const __nv_bfloat16*)h, ld, cu, p->n_s,
+      launch_on(fit_partial_kernel<__nv_bfloat16>, grid, dim3(kFitThreads), smem, st, tmH, (const __nv_bfloat16*)h, ld, cu, p->n_s,
                                                                          p->d_h, fit_chunks, stages, partial, status);
     }
   }

@@ -131,8 +131,6 @@ project_simt_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __
 __global__ void project_finish_kernel(const float* __restrict__ qf, int splits, int64_t split_stride,
                                       const float* __restrict__ bias, const float* __restrict__ table, int S,
                                       int Hq, int G, int d_k, __nv_bfloat16* __restrict__ Q) {
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.z, row = blockIdx.y;
   const int half = d_k / 2;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;   // over Hq * half
@@ -191,7 +189,7 @@ int32_t launch_project_staged(const gvote_params* p, const __nv_bfloat16* X, con
   dim3 gf((unsigned)ceil_div((int64_t)p->n_q_heads * (p->d_k / 2), 128), S + 1, batch);
   {
     LaunchScope scope_("project_finish_kernel", st);
-    launch_pdl(project_finish_kernel, gf, dim3(128), 0, st, qf, splits, (int64_t)rows_total * F, b_q, rope_table, S, p->n_q_heads,
+    launch_on(project_finish_kernel, gf, dim3(128), 0, st, qf, splits, (int64_t)rows_total * F, b_q, rope_table, S, p->n_q_heads,
                                               p->n_q_heads / p->n_kv_heads, p->d_k, Q);
   }
   GVOTE_LAUNCH_CHECK("project_finish_kernel");

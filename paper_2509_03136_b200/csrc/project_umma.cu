@@ -45,7 +45,6 @@ project_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     int rows_total, int F, int kchunks_total, int kchunks_per_split, int NC, int acc_cols,
                     int stages, float* __restrict__ part, int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  pdl_trigger();
   const int m_tile = blockIdx.x, split = blockIdx.y, rchunk = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kc0 = split * kchunks_per_split;
@@ -73,7 +72,6 @@ project_umma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
-  pdl_wait();                                    // X is the output of the kernel before this one
   const uint32_t tmem_base = tail->tmem_slot;
   volatile int* abort_flag = &tail->abort_flag;
 
@@ -203,7 +201,7 @@ int32_t launch_project_umma(const gvote_params* p, const __nv_bfloat16* X, const
   dim3 grid((unsigned)ceil_div(F, kFeatTile), (unsigned)splits, (unsigned)rchunks);
   {
     LaunchScope scope_("project_umma_kernel", st);
-    launch_pdl(project_umma_kernel, grid, dim3(kProjThreads), smem, st, tmW, tmX, rows_total, F, kchunks, per, NC, acc_cols, stages,
+    launch_on(project_umma_kernel, grid, dim3(kProjThreads), smem, st, tmW, tmX, rows_total, F, kchunks, per, NC, acc_cols, stages,
                                                           part, status);
   }
   GVOTE_LAUNCH_CHECK("project_umma_kernel");

@@ -90,8 +90,6 @@ bracket_kernel(const uint16_t* __restrict__ sample, int64_t sample_slots, const 
                int G, int S, int row_chunks, const int32_t* __restrict__ b_step, RowBracket* __restrict__ bracket,
                const int32_t* __restrict__ kv_len) {
   __shared__ BracketShared sh;
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int rowid = (r * Hq + g) * S + s;
   const int start = cu[r];
@@ -260,8 +258,6 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
                const VoteState vs, int smem_keys, int64_t row_words, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint32_t dyn[];         // [seg offsets: segs + 1][keys: smem_keys]
   __shared__ ResolveShared sh;
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int rowid = (r * Hq + g) * S + s;
   const int start = cu[r], Ncap = cu[r + 1] - start;
@@ -457,8 +453,6 @@ commit_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restri
               uint32_t* __restrict__ mask, const uint32_t* __restrict__ head_bad, const int32_t* __restrict__ kv_len) {
   __shared__ SelShared sh;
   __shared__ __align__(16) __nv_bfloat16 qf[512];
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
   const int start = cu[r], Ncap = cu[r + 1] - start;
   const int kh = g / G, Hkv = Hq / G;
@@ -500,10 +494,10 @@ int32_t launch_bracket(const gvote_params* p, const int32_t* cu, int32_t batch, 
   {
     LaunchScope scope_("bracket_kernel", st);
     if (sample_geom((int)max_N).ns * 16 <= 4 * kBrThreads)
-      launch_pdl(bracket_kernel<4>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
+      launch_on(bracket_kernel<4>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
                  score_geometry(p).row_chunks, b_step, vs.bracket, kv_len);
     else
-      launch_pdl(bracket_kernel<16>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
+      launch_on(bracket_kernel<16>, grid, dim3(kBrThreads), 0, st, vs.sample, vs.sample_slots, cu, Hq, G, p->S,
                  score_geometry(p).row_chunks, b_step, vs.bracket, kv_len);
   }
   GVOTE_LAUNCH_CHECK("bracket_kernel");
@@ -526,9 +520,9 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
   {
     LaunchScope scope_("resolve_kernel", st);
     if (smem_keys <= 4096)
-      launch_pdl(resolve_kernel<64>, grid, dim3(64), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
+      launch_on(resolve_kernel<64>, grid, dim3(64), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
     else
-      launch_pdl(resolve_kernel<kRowThreads>, grid, dim3(kRowThreads), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
+      launch_on(resolve_kernel<kRowThreads>, grid, dim3(kRowThreads), smem, st, cu, Hq, G, p->S, b_step, vs, smem_keys, row_words, kv_len);
   }
   GVOTE_LAUNCH_CHECK("resolve_kernel");
   return GVOTE_OK;
@@ -542,7 +536,7 @@ int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_
   const float scale = (float)(1.0 / sqrt((double)p->d_k));
   {
     LaunchScope scope_("commit_kernel", st);
-    launch_pdl(commit_kernel, grid, dim3(kRowThreads), 0, st, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, scale, b_step, vs.tmask,
+    launch_on(commit_kernel, grid, dim3(kRowThreads), 0, st, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, scale, b_step, vs.tmask,
                                                 row_words, mask, vs.head_bad, kv_len);
   }
   GVOTE_LAUNCH_CHECK("commit_kernel");

@@ -74,8 +74,6 @@ prep_kernel(const float2* __restrict__ partial, int chunks, const T* __restrict_
             float* __restrict__ var, __nv_bfloat16* __restrict__ X, float* __restrict__ table) {
   __shared__ FitMoments sm[8][32];
   __shared__ float s_mu[32], s_sd[32];
-  pdl_trigger();
-  pdl_wait();
   const int r = blockIdx.y;
   const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
   const int col0 = blockIdx.x * 32, col = col0 + tx;
@@ -177,11 +175,11 @@ int32_t launch_prep(const gvote_params* p, const float2* partial, int fit_chunks
   {
     LaunchScope scope_("prep_kernel", st);
     if (p->h_dtype == GVOTE_DTYPE_F32)
-      launch_pdl(prep_kernel<float>, grid, dim3(256), 0, st, partial, fit_chunks, (const float*)h_last, h_last_ld,
+      launch_on(prep_kernel<float>, grid, dim3(256), 0, st, partial, fit_chunks, (const float*)h_last, h_last_ld,
                                                h_last_rows_from_cu, cu, p->n_s, p->d_h, p->S, p->d_k, p->rope_theta,
                                                p->n_f, k0, k1, p->layer_id, mu, var, X, rope_table);
     else
-      launch_pdl(prep_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, partial, fit_chunks, (const __nv_bfloat16*)h_last, h_last_ld,
+      launch_on(prep_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, partial, fit_chunks, (const __nv_bfloat16*)h_last, h_last_ld,
                                                        h_last_rows_from_cu, cu, p->n_s, p->d_h, p->S, p->d_k,
                                                        p->rope_theta, p->n_f, k0, k1, p->layer_id, mu, var, X,
                                                        rope_table);

@@ -171,7 +171,6 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     uint32_t* __restrict__ zero_a, uint32_t* __restrict__ zero_b, int64_t zero_words,
                     uint32_t* __restrict__ head_bad, int n_head_bad) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  pdl_trigger();
   const int groups = (row_chunks + cg - 1) / cg;
   const int r = blockIdx.z;
   const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
@@ -181,8 +180,7 @@ score_sample_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const SweepSmem sm = carve(smem_raw, kchunks, cg, stages, true, (uint32_t)n_out * kRowChunk * kTileKeys * 2);
   SweepTail* tail = sm.tail;
-  if (active) setup(tail, stages, &tmK, &tmQ, &tmQr);     // barriers, tensor memory: under the tail of the kernel before
-  pdl_wait();
+  if (active) setup(tail, stages, &tmK, &tmQ, &tmQr);     // barriers, tensor memory
   // The vote starts from an empty keep mask, an empty tentative mask and no head marked: every CTA of this
   // first kernel of the vote clears its share (nothing reads them before the kernels that follow).
   {
@@ -390,7 +388,6 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
                    int nbuf, float scale, const VoteState vs, int64_t row_words, int32_t* __restrict__ status,
                    const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  pdl_trigger();
   const int groups = (row_chunks + CG - 1) / CG;
   const int r = blockIdx.z;
   const int kh = blockIdx.y / groups, grp = blockIdx.y % groups;
@@ -416,7 +413,6 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap tmK, const __nv_bfloat16*
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
-  pdl_wait();
   const int start = cu[r], Ncap = cu[r + 1] - start;
   const int N = valid_keys(kv_len, r, Hq / G, kh, Ncap);
   TileWalk walk;
@@ -699,7 +695,7 @@ int32_t launch_score_sample(const gvote_params* p, const __nv_bfloat16* Q, const
   GVOTE_CUDA_CHECK(cudaFuncSetAttribute(score_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope scope_("score_sample_kernel", st);
-    launch_pdl(score_sample_kernel, grid, dim3(kSweepThreads), smem, st, tmK, tmQ, tmQr, cu, Hq, G, p->S, d_k, row_chunks, cg,
+    launch_on(score_sample_kernel, grid, dim3(kSweepThreads), smem, st, tmK, tmQ, tmQr, cu, Hq, G, p->S, d_k, row_chunks, cg,
                (int)X0, (int)X1, stages, n_out, scale, real_logits, rowmax_part, vs.sample, vs.sample_slots, status, kv_len,
                vs.tmask, mask, (int64_t)Hkv * row_words, vs.head_bad, (int)(batch * Hkv));
   }
@@ -754,7 +750,7 @@ int32_t launch_score_sweep(const gvote_params* p, const __nv_bfloat16* Q, const 
     LaunchScope scope_("score_sweep_kernel", st);
     // accumulators: three when the query rows leave room in the 512 columns of tensor memory, else two
     const int nbuf = (512 - geo.cg * (d_k / 2)) / kRowChunk >= 3 ? 3 : 2;
-    launch_pdl(kern, grid, dim3(kSweepBThreads), smem, st, tmK, Q, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, nbuf, scale, vs, row_words,
+    launch_on(kern, grid, dim3(kSweepBThreads), smem, st, tmK, Q, cu, Hq, G, p->S, d_k, row_chunks, geo.stages, nbuf, scale, vs, row_words,
                                              status, kv_len);
   }
   GVOTE_LAUNCH_CHECK("score_sweep_kernel");

@@ -120,8 +120,6 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
                  const uint32_t* __restrict__ rowmax_part, int n_part, float p_nuc, int include_c0, int64_t row_words,
                  uint32_t* __restrict__ mask, int32_t* __restrict__ b_step, const int32_t* __restrict__ kv_len) {
   extern __shared__ __align__(16) uint8_t dyn[];
-  pdl_trigger();
-  pdl_wait();
   ClusterShared& cs = *reinterpret_cast<ClusterShared*>(dyn);
   // The generic radix search and the emission (rare routes of the first CTA) work in the space of the
   // candidate list, which is dead by the time they run.
@@ -411,7 +409,7 @@ int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32
   dim3 grid((unsigned)kClusterCtas, (unsigned)Hq, (unsigned)batch);
   {
     LaunchScope scope_("real_topp_kernel", st);
-    launch_pdl(real_topp_kernel, grid, dim3(kThreads), sizeof(ClusterShared), st, logits, cu, Hq, G, rowmax_part, n_part, p->p_nuc,
+    launch_on(real_topp_kernel, grid, dim3(kThreads), sizeof(ClusterShared), st, logits, cu, Hq, G, rowmax_part, n_part, p->p_nuc,
                                                                     p->include_c0, row_words, mask, b_step, kv_len);
   }
   GVOTE_LAUNCH_CHECK("real_topp_kernel");
