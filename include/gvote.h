@@ -106,6 +106,15 @@ static inline int64_t gvote_mask_word_offset(int64_t cu_seqlens_r, int32_t r) {
  * or 128, more than 16 query heads per KV head): gvote_workspace_bytes accounts for that. */
 GVOTE_API size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
 
+/* Where gvote_select and the whole-pass entry points (gvote_compress, gvote_compress_moments, gvote_recompress) leave the
+ * rotated queries of Algorithm 1 that their vote used - Q0 (exact position) and the S synthetic queries
+ * (averaged cos/sin) of every query head: byte offset into `ws` of a bf16 array
+ * [batch][n_kv_heads][G (S+1)][d_k], G = n_q_heads / n_kv_heads, the layout gvote_project writes (per KV
+ * head the G*S synthetic rows, query head by query head, then the G current-query rows).  They stay valid
+ * until the next call that uses the workspace; gvote_overlap and a caller's own checks can read them there.
+ * Returns 0 on invalid params (offset 0 is the status block, never the queries). */
+GVOTE_API size_t gvote_workspace_queries(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N);
+
 /* Step 2 of Section 3.2 (the Gaussian fit of Algorithm 1).  mu[r][c], var[r][c] = mean and unbiased variance over rows
  * cu_seqlens[r]+n_s .. cu_seqlens[r+1]-1 of h [total_tokens, d_h] (row stride h_row_stride
  * elements).  Every request needs N_r - n_s >= 2 (the result is NaN otherwise; the host cannot

@@ -137,6 +137,11 @@ size_t gvote_workspace_bytes(const gvote_params* p, int32_t batch, int64_t total
   return workspace_map(p, batch, total_tokens, max_N).total;
 }
 
+size_t gvote_workspace_queries(const gvote_params* p, int32_t batch, int64_t total_tokens, int64_t max_N) {
+  if (validate_params(p) != GVOTE_OK || validate_batch(batch, total_tokens, max_N) != GVOTE_OK) return 0;
+  return workspace_map(p, batch, total_tokens, max_N).q_bf16;
+}
+
 int32_t gvote_fit(const gvote_params* p, const void* h, int64_t h_row_stride, const int32_t* cu_seqlens,
                   int32_t batch, int64_t total_tokens, int64_t max_N, float* mu, float* var, void* ws,
                   size_t ws_bytes, void* stream) {

@@ -22,7 +22,7 @@ SEL_TOPK_C0, SEL_TOPP = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = (
-    "gvote_workspace_bytes", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
+    "gvote_workspace_bytes", "gvote_workspace_queries", "gvote_fit", "gvote_fit_update", "gvote_fit_finish", "gvote_fit_static", "gvote_sample", "gvote_project", "gvote_vote", "gvote_select",
     "gvote_compact", "gvote_pack", "gvote_overlap", "gvote_compress", "gvote_compress_moments", "gvote_recompress", "gvote_compress_host", "gvote_host_arena_release",
     "gvote_poll_status", "gvote_clear_status", "gvote_exact_heads", "gvote_profile_enable", "gvote_profile_report", "gvote_launch_count", "gvote_status_string", "gvote_last_cuda_error",
 )
@@ -60,6 +60,8 @@ def load():
     P, vp, i32, i64, sz = ctypes.POINTER(GVoteParams), ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     lib.gvote_workspace_bytes.restype = sz
     lib.gvote_workspace_bytes.argtypes = [P, i32, i64, i64]
+    lib.gvote_workspace_queries.restype = sz
+    lib.gvote_workspace_queries.argtypes = [P, i32, i64, i64]
     lib.gvote_fit.restype = i32
     lib.gvote_fit.argtypes = [P, vp, i64, vp, i32, i64, i64, vp, vp, vp, sz, vp]
     lib.gvote_fit_update.restype = i32
@@ -171,6 +173,16 @@ def batch_geometry(cu_seqlens_host: Sequence[int]) -> Tuple[int, int, int]:
 
 def gvote_workspace_bytes(p: GVoteParams, batch: int, total_tokens: int, max_N: int) -> int:
     return int(load().gvote_workspace_bytes(ctypes.byref(p), batch, total_tokens, max_N))
+
+
+def workspace_queries(p: GVoteParams, ws: torch.Tensor, batch: int, total_tokens: int, max_N: int) -> torch.Tensor:
+    """The rotated queries a whole-pass call left in `ws`: a bf16 view [batch, n_kv_heads, G*(S+1), d_k]."""
+    off = int(load().gvote_workspace_queries(ctypes.byref(p), batch, total_tokens, max_N))
+    if off == 0:
+        raise GVoteError(-1, "gvote_workspace_queries")
+    G = p.n_q_heads // p.n_kv_heads
+    n = batch * p.n_kv_heads * G * (p.S + 1) * p.d_k
+    return ws[off:off + 2 * n].view(torch.bfloat16).view(batch, p.n_kv_heads, G * (p.S + 1), p.d_k)
 
 
 def alloc_workspace(p: GVoteParams, batch: int, total_tokens: int, max_N: int, device="cuda",

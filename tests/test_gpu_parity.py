@@ -4,6 +4,7 @@ normal draws 1e-5 absolute on z; rotated queries within one bf16 step; softmax r
 where the weight is >= 1e-6; masks identical outside the 1e-3 band around each selection
 threshold; budgets within 0.5 % of N."""
 import math
+from dataclasses import replace
 
 import numpy as np
 import pytest
@@ -551,6 +552,25 @@ def test_pack_varlen_reports_buffers_that_are_too_small(gv):
 
 
 # ----------------------------------------------------------------------------- whole pass
+def _queries_left_in(gv, p, ws, geom):
+    """The rotated queries a whole-pass call left in its workspace, [batch, H_kv, G (S+1), d_k] as fp64."""
+    return gv.workspace_queries(p, ws, *geom).float().cpu().numpy().astype(np.float64)
+
+
+def _check_mask_against_own_queries(gv, cfg, Qg_r, Qo, K64, p_nuc, sel_mode, gm, b_step_r):
+    """Whole pass, second half: the mask against the oracle's vote on the queries the GPU itself used, inside
+    the 1e-3 bands.  Those queries against the oracle's: the GPU fits in fp32 and draws with fp32
+    Box-Muller, so an entry of X can land on the neighbouring bf16 value and move every product of its row
+    by |w| ulp(x): bounded here by one bf16 step of the entry plus 2^-6 of the row's largest entry (a wrong
+    sign, index or rotation is off by the query's own magnitude), and nine entries in ten must be equal."""
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    Qr = pu.from_group_major(Qg_r, G)
+    scale = np.abs(Qo).max(axis=-1, keepdims=True)
+    assert np.all(np.abs(Qr - Qo) <= 2.0 ** -7 * np.abs(Qo) + 2.0 ** -6 * scale), np.abs(Qr - Qo).max()
+    assert (Qr == Qo).mean() > 0.9
+    pu.check_vote_against_oracle(Qr, K64, p_nuc, sel_mode, False, gm, b_step_r)          # 1e-3 bands
+
+
 def _run_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
     p = gv.params_from_config(cfg, layer_id=layer_id, sel_mode=gv.SEL_TOPP if sel_mode == "topp" else gv.SEL_TOPK_C0)
     geom = _geom(cfg)
@@ -562,14 +582,16 @@ def _run_compress(gv, cfg, li, sel_mode="topk", layer_id=0):
     gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget, b_step, ws)
     assert gv.gvote_poll_status(ws) == 0
     return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
-            gv.bits_from_bf16(d["V"]))
+            gv.bits_from_bf16(d["V"]), _queries_left_in(gv, p, ws, geom))
 
 
 def _check_compress(gv, cfg, li, sel_mode="topk", layer_id=0, runner=None):
     """End to end.  The GPU draws its own samples (fp32 fit and Box-Muller), so a few query values
-    land on the neighbouring bf16 step; masks are compared inside the score tolerance (2e-2) band
-    and budgets to 0.5 % of N.  Compaction is checked bit-exactly against the GPU's own mask."""
-    mask, budget, b_step, Kg, Vg = (runner or _run_compress)(gv, cfg, li, sel_mode, layer_id)
+    land on the neighbouring bf16 step: masks are compared with the oracle's own run inside the score
+    tolerance (2e-2) band, budgets to 0.5 % of N, and - the strict check - with the oracle's vote on the
+    queries the GPU left in its workspace inside the 1e-3 bands.  Compaction is checked bit-exactly
+    against the GPU's own mask."""
+    mask, budget, b_step, Kg, Vg, Qg = (runner or _run_compress)(gv, cfg, li, sel_mode, layer_id)
     kw = pu.oracle_kwargs(cfg, layer_id)
     res, _, _ = o.compress_layer(li.h, li.W_q, li.b_q, li.K, li.V, li.cu_seqlens, sel_mode=sel_mode, **kw)
     pf = kw["p_nuc"]
@@ -579,6 +601,7 @@ def _check_compress(gv, cfg, li, sel_mode="topk", layer_id=0, runner=None):
         gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N) for h in range(cfg.n_kv_heads)])
         Kr = o.bf16_bits_to_f64(li.K[:, a:b])
         pu.check_vote_against_oracle(res[r].Q, Kr, pf, sel_mode, False, gm, b_step[r], mass_band=2e-2, logit_band=2e-2)
+        _check_mask_against_own_queries(gv, cfg, Qg[r], res[r].Q, Kr, pf, sel_mode, gm, b_step[r])
         assert np.all(np.abs(budget[r] - res[r].budget) <= max(2, 0.005 * N)), (budget[r], res[r].budget)
         Kc, Vc = o.compact(li.K[:, a:b], li.V[:, a:b], gm)
         for h in range(cfg.n_kv_heads):
@@ -605,7 +628,7 @@ def test_compress_planted_answer(gv, n_heavy, p_nuc):
     exactly the planted positions; at p = 0.9 nothing outside them is kept.  And the oracle agrees."""
     cfg = synth.make_planted(n_heavy, p_nuc=p_nuc)
     li = synth.make_layer(cfg, 0)
-    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li)
+    mask, budget, b_step, Kg, Vg, _ = _run_compress(gv, cfg, li)
     for kh in range(cfg.n_kv_heads):
         kept = np.nonzero(gv.unpack_mask(mask[kh], 0, cfg.total_tokens))[0]
         planted = li.heavy_positions[(0, kh)]
@@ -626,7 +649,7 @@ def _run_compress_bf16_h(gv, cfg, li, sel_mode="topk", layer_id=0):
     gv.gvote_compress(p, d["h"].bfloat16(), d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget, b_step, ws)
     assert gv.gvote_poll_status(ws) == 0
     return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
-            gv.bits_from_bf16(d["V"]))
+            gv.bits_from_bf16(d["V"]), _queries_left_in(gv, p, ws, geom))
 
 
 @pytest.mark.parametrize("name", ["small2", "c1", "c3"])
@@ -693,7 +716,7 @@ def _run_compress_moments(gv, cfg, li, sel_mode="topk", layer_id=0):
                               b_step, ws)
     assert gv.gvote_poll_status(ws) == 0
     return (mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy(), gv.bits_from_bf16(d["K"]),
-            gv.bits_from_bf16(d["V"]))
+            gv.bits_from_bf16(d["V"]), _queries_left_in(gv, p, ws, geom))
 
 
 @pytest.mark.parametrize("name", ["small2", "c0", "c1", "c3"])
@@ -761,6 +784,7 @@ def _check_recompress(gv, cfg, li, sel_mode="topk", n_new=5, empty_head=None, se
     assert gv.gvote_poll_status(ws) == 0
     mask, budget, b_step = mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy()
     Kg, Vg, pos_g = gv.bits_from_bf16(dK), gv.bits_from_bf16(dV), d_pos.cpu().numpy()
+    Qg = _queries_left_in(gv, p, ws, geom)
 
     W = o.bf16_bits_to_f64(li.W_q)
     kw = pu.oracle_kwargs(cfg)
@@ -783,6 +807,11 @@ def _check_recompress(gv, cfg, li, sel_mode="topk", n_new=5, empty_head=None, se
                 continue
             pu.check_vote_against_oracle(res.Q[h * G:(h + 1) * G], heads[h][None], kw["p_nuc"], sel_mode, False,
                                          gm[None], b_step[r, h * G:(h + 1) * G], mass_band=2e-2, logit_band=2e-2)
+            # and, inside the 1e-3 bands, against the oracle's vote on the queries the GPU used (per head: a
+            # head's rows are its own kv_len)
+            one_head = replace(cfg, n_q_heads=G, n_kv_heads=1)
+            _check_mask_against_own_queries(gv, one_head, Qg[r, h:h + 1], res.Q[h * G:(h + 1) * G], heads[h][None],
+                                            kw["p_nuc"], sel_mode, gm[None], b_step[r, h * G:(h + 1) * G])
             assert abs(int(budget[r, h]) - int(res.budget[h])) <= max(2, 0.005 * n)
             keep = np.nonzero(gm)[0]
             assert budget[r, h] == keep.shape[0]
@@ -888,7 +917,7 @@ def test_compress_with_an_empty_request(gv):
     full = synth.make_small(8, seq_lens=(40, 33), S=4, d_h=64, n_q_heads=4, n_kv_heads=2, d_k=64)
     li = synth.make_layer(full, 0)
     li.cu_seqlens = np.array([0, 40, 40, 73], dtype=np.int32)
-    mask, budget, b_step, Kg, Vg = _run_compress(gv, cfg, li)
+    mask, budget, b_step, Kg, Vg, Qg = _run_compress(gv, cfg, li)
     assert budget[1].tolist() == [0, 0] and b_step[1].tolist() == [0] * 4
     W = o.bf16_bits_to_f64(li.W_q)
     kw = pu.oracle_kwargs(cfg)
@@ -898,6 +927,8 @@ def test_compress_with_an_empty_request(gv):
         gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), b - a) for h in range(cfg.n_kv_heads)])
         pu.check_vote_against_oracle(res.Q, o.bf16_bits_to_f64(li.K[:, a:b]), kw["p_nuc"], "topk", False, gm, b_step[r],
                                      mass_band=2e-2, logit_band=2e-2)
+        _check_mask_against_own_queries(gv, cfg, Qg[r], res.Q, o.bf16_bits_to_f64(li.K[:, a:b]), kw["p_nuc"], "topk", gm,
+                                        b_step[r])
         assert np.all(np.abs(budget[r] - res.budget) <= 2)
         Kc, Vc = o.compact(li.K[:, a:b], li.V[:, a:b], gm)
         for h in range(cfg.n_kv_heads):
@@ -1019,7 +1050,7 @@ def test_recompress_full_size_c2_layer(gv):
 def test_compress_host_variant_matches_device_variant(gv):
     cfg = synth.make_config("c0")
     li = synth.make_layer(cfg, 0)
-    mask_d, budget_d, b_step_d, Kd, Vd = _run_compress(gv, cfg, li)
+    mask_d, budget_d, b_step_d, Kd, Vd, _ = _run_compress(gv, cfg, li)
     p = gv.params_from_config(cfg)
     h = torch.from_numpy(li.h).pin_memory()
     W = gv.bf16_from_bits(li.W_q, "cpu", pin=True)
