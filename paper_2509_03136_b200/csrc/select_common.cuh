@@ -57,6 +57,17 @@ __device__ __forceinline__ unsigned long long mass_fix(float l, float mx) {
   return __float2ull_rn(expf(l - mx) * kFixScale);
 }
 
+// Adds m to a 64-bit sum in shared memory with 32-bit atomics (the low word, then the carry and the high
+// word when there is one - a mass has 41 bits, so mostly there is not): the sum is exact whatever the order
+// of arrival, and a 32-bit shared-memory atomic does not loop.
+__device__ __forceinline__ void add_mass(unsigned long long* sum, unsigned long long m) {
+  uint32_t* w = reinterpret_cast<uint32_t*>(sum);
+  const uint32_t lo = (uint32_t)m;
+  const uint32_t old = atomicAdd(&w[0], lo);
+  const uint32_t hi = (uint32_t)(m >> 32) + ((old + lo < old) ? 1u : 0u);
+  if (hi) atomicAdd(&w[1], hi);
+}
+
 // Find the highest bin b of hist[0..nbins) whose suffix sum (bins >= b) reaches `need`;
 // publish b and the sum of the bins above it.  MASS selects which histogram decides; the count
 // of elements above is always published too.  Requires total >= need (else bin 0 is returned).
@@ -139,7 +150,7 @@ __device__ void radix_threshold(const Row& row, int N, float mx, unsigned long l
       if ((key & known_mask) == prefix && keep(l)) {
         const int b = (key >> shifts[pass]) & (nb - 1);
         atomicAdd(&sh.cnt[b], 1u);
-        if (MASS) atomicAdd(&sh.mass[b], mass_fix(l, mx));
+        if (MASS) add_mass(&sh.mass[b], mass_fix(l, mx));
       }
     }
     __syncthreads();

@@ -172,7 +172,7 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
             tail_m += m;
           } else {
             atomicAdd(&cs.cnt[b], 1u);
-            if (m) atomicAdd(&cs.mass[b], m);
+            if (m) add_mass(&cs.mass[b], m);
           }
         }
       }
@@ -281,7 +281,7 @@ real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ c
         const int b = sub_of(cs.val[i]);
         atomicAdd(&cs.sub_cnt[b], 1u);
         const unsigned long long w = mass_fix(cs.val[i], mx);
-        if (w) atomicAdd(&cs.sub_mass[b], w);
+        if (w) add_mass(&cs.sub_mass[b], w);
       }
       __syncthreads();
       const uint32_t sc = cs.sub_cnt[tid];
