@@ -273,6 +273,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-upstream-row", action="store_true")
     ap.add_argument("--no-recompress-row", action="store_true")
+    ap.add_argument("--no-graph-row", action="store_true", help="skip the one-stream pass replayed as a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark: budget, attention kept and select time over S and over p "
                          "(one layer of --workload, default c1)")
@@ -464,6 +465,32 @@ def main():
                       "ms_per_step": one_ms, "per_layer_us": one_ms * 1e3 / L,
                       "full_bytes_frac": full_t / (one_ms * 1e-3 / L), "literal_frac": lit_t / (one_ms * 1e-3 / L),
                       "note": "extra row: the same pass with every layer on one stream, no per-kernel events; not the headline"}
+    # the same one-stream pass recorded once as a CUDA graph and replayed: what an engine that compresses layer
+    # by layer gets when it captures the calls instead of enqueueing twelve launches per layer from the host
+    if not args.no_graph_row:
+        graph = torch.cuda.CUDAGraph()
+        restore()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+            one_pass(spread=False)
+        torch.cuda.synchronize()
+        g_ms = 0.0
+        for i in range(2 + args.steps):                  # two untimed replays first
+            restore()
+            barrier()
+            ev0.record()
+            graph.replay()
+            ev1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                g_ms += ev0.elapsed_time(ev1)
+        g_ms = shard.max_over_ranks(g_ms, dist, dev) / args.steps
+        del graph
+        assert gv.gvote_poll_status(ws) == 0, "a device-side wait timed out"
+        one_stream_row["as_cuda_graph"] = {
+            "value": shard.job_throughput(cfg.total_tokens, world, g_ms * 1e-3), "unit": UNIT, "ms_per_step": g_ms,
+            "per_layer_us": g_ms * 1e3 / L, "full_bytes_frac": full_t / (g_ms * 1e-3 / L),
+            "note": "the one-stream pass captured once (torch.cuda.graph around the same gvote_compress calls) and replayed"}
     roofline["pass"] = {
         "note": "whole pass against its own roofline: the slower of the bf16 flops at the tensor peak and the bytes at "
                 "the HBM peak; 'literal' counts the K read and the K/V compaction bytes only, 'full_bytes' also the "
