@@ -701,14 +701,19 @@ def main():
     # ---- the oracle on the host cores, on a bounded sample (rank 0, one GPU only)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        t_or, res = time_oracle_layer(cfg, layers[0], 0)
-        ob = np.stack([r.budget for r in res])
-        gb = d_budget[0].cpu().numpy()
+        # whole layers, until about ten seconds of oracle time have gone by (three layers of the 32K workload)
+        t_or, n_or, ok = 0.0, 0, True
         tol = np.maximum(2, 0.005 * np.asarray(cfg.seq_lens)[:, None])
-        cpu_baseline = {"value": cfg.total_tokens / (t_or * L), "unit": UNIT, "cores": blas_threads(),
-                        "kind": "oracle", "sample": f"layer 0 of {L} ({cfg.total_tokens} tokens) took {t_or:.1f} s in the fp64 "
-                        f"NumPy oracle as it stands (matmul, sort, cumsum are NumPy's; BLAS threads = cores); value = tokens / "
-                        f"(that time x {L} layers)", "budgets_within_tolerance": bool(np.all(np.abs(ob - gb) <= tol))}
+        while n_or < L and (n_or == 0 or t_or < 10.0):
+            t_l, res = time_oracle_layer(cfg, layers[n_or], n_or)
+            ob = np.stack([r.budget for r in res])
+            ok = ok and bool(np.all(np.abs(ob - d_budget[n_or].cpu().numpy()) <= tol))
+            t_or += t_l
+            n_or += 1
+        cpu_baseline = {"value": cfg.total_tokens * n_or / (t_or * L), "unit": UNIT, "cores": blas_threads(),
+                        "kind": "oracle", "sample": f"layers 0..{n_or - 1} of {L} ({cfg.total_tokens} tokens each) took {t_or:.1f} s "
+                        f"in the fp64 NumPy oracle as it stands (matmul, sort, cumsum are NumPy's; BLAS threads = cores); "
+                        f"value = tokens / (the mean layer time x {L} layers)", "budgets_within_tolerance": ok}
 
     if rank == 0:
         out = {
