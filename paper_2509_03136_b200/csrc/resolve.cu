@@ -332,27 +332,35 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
     }
     return list + (int64_t)a * seg_cap + (e - seg_off[a]);
   };
-  // gather the order-preserving images of the listed logits
-  {
-    uint32_t mn = 0xffffffffu, mx = 0u;
-    for (uint32_t base = 0; base < C; base += 4 * NT) {
-      uint32_t x[4];
+  // gather the order-preserving images of the listed logits; the key indices of the first kHold rounds stay
+  // in registers for the emission below (a row of the usual length is all of them: no second trip to the lists)
+  constexpr int kHold = 3;
+  uint32_t held[kHold][4];
+  auto gather_round = [&](uint32_t base, uint32_t* hy, uint32_t& mn, uint32_t& mx) {
+    uint2 ent[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const uint32_t e = base + u * NT + tid;
-        x[u] = e < C ? entry_of(e)->x : 0u;
-      }
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t e = base + u * NT + tid;
+      ent[u] = e < C ? *entry_of(e) : make_uint2(0u, 0u);
+    }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const uint32_t e = base + u * NT + tid;
-        if (e < C) {
-          const uint32_t kx = ordered_key(__uint_as_float(x[u]));
-          keys[e] = kx;
-          mn = min(mn, kx);
-          mx = max(mx, kx);
-        }
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t e = base + u * NT + tid;
+      if (hy) hy[u] = ent[u].y;
+      if (e < C) {
+        const uint32_t kx = ordered_key(__uint_as_float(ent[u].x));
+        keys[e] = kx;
+        mn = min(mn, kx);
+        mx = max(mx, kx);
       }
     }
+  };
+  {
+    uint32_t mn = 0xffffffffu, mx = 0u;
+#pragma unroll
+    for (int b = 0; b < kHold; ++b)
+      if ((uint32_t)(b * 4 * NT) < C) gather_round((uint32_t)(b * 4 * NT), held[b], mn, mx);
+    for (uint32_t base = kHold * 4 * NT; base < C; base += 4 * NT) gather_round(base, nullptr, mn, mx);
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
     if (lane == 0) { atomicMin(&sh.kmin, mn); atomicMax(&sh.kmax, mx); }
@@ -421,7 +429,7 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
     idx_max = vlim;
   }
   const bool all_of_bin = whole_bin || ties >= eq;
-  for (uint32_t base = 0; base < C; base += 4 * NT) {
+  auto emit_round = [&](uint32_t base, const uint32_t* hy) {
     uint32_t n[4];
     bool want[4], tie[4];
 #pragma unroll
@@ -431,12 +439,16 @@ resolve_kernel(const int32_t* __restrict__ cu, int Hq, int G, int S, const int32
       const bool in_bin = e < C && (x & known) == prefix;
       want[u] = e < C && (x > (prefix | ~known) || (in_bin && all_of_bin));
       tie[u] = in_bin && !all_of_bin;
-      n[u] = (want[u] || tie[u]) ? entry_of(e)->y : 0u;
+      n[u] = hy ? hy[u] : ((want[u] || tie[u]) ? entry_of(e)->y : 0u);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
       if (want[u] || (tie[u] && n[u] <= idx_max)) atomicOr(&mrow[n[u] >> 5], 1u << (n[u] & 31));
-  }
+  };
+#pragma unroll
+  for (int b = 0; b < kHold; ++b)
+    if ((uint32_t)(b * 4 * NT) < C) emit_round((uint32_t)(b * 4 * NT), held[b]);
+  for (uint32_t base = kHold * 4 * NT; base < C; base += 4 * NT) emit_round(base, nullptr);
 }
 
 // ------------------------------------------------------------------------------------ commit
