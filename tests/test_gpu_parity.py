@@ -1065,3 +1065,41 @@ def test_compress_host_variant_matches_device_variant(gv):
         assert np.array_equal(mask.numpy(), mask_d) and np.array_equal(budget.numpy(), budget_d)
         assert np.array_equal(gv.bits_from_bf16(K), Kd) and np.array_equal(gv.bits_from_bf16(V), Vd)
     gv.gvote_host_arena_release()
+
+
+@pytest.mark.parametrize("name", ["small2", "c1", "c3"])
+def test_workspace_queries_are_the_staged_projection(gv, name):
+    """gvote_workspace_queries: the rotated queries the whole pass leaves in its workspace are those of the
+    staged calls (fit -> sample -> project) on the same inputs: the same draws, the same roundings.  The fused
+    middle of the pass merges the fit's partial sums in one step instead of two, so a mean may differ in its
+    last bit and a query entry by one bf16 step: nearly all entries are equal, none is further than a step."""
+    cfg = _small_cfgs()[2] if name == "small2" else synth.make_config(name)
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    B, S, G = cfg.batch, cfg.S, cfg.n_q_heads // cfg.n_kv_heads
+    d = pu.upload_layer(li, gv, torch)
+    ws = gv.alloc_workspace(p, *geom)
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, B), dtype=torch.int32, device="cuda")
+    budget = torch.empty(B, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(B, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    K, V = d["K"].clone(), d["V"].clone()
+    gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], K, V, d["cu"], geom, mask, budget, b_step, ws)
+    Q_pass = gv.workspace_queries(p, ws, *geom).float().cpu().numpy()
+    ws2 = gv.alloc_workspace(p, *geom)
+    mu = torch.empty(B, cfg.d_h, device="cuda"); var = torch.empty_like(mu)
+    gv.gvote_fit(p, d["h"], d["cu"], geom, mu, var, ws2)
+    Ht = torch.empty(B, S, cfg.d_h, device="cuda")
+    gv.gvote_sample(p, mu, var, B, Ht)
+    cu = li.cu_seqlens
+    h_last = torch.from_numpy(np.stack([li.h[int(cu[r + 1]) - 1] for r in range(B)])).cuda()
+    Q = torch.empty(B, cfg.n_kv_heads, G * (S + 1), cfg.d_k, dtype=torch.bfloat16, device="cuda")
+    gv.gvote_project(p, Ht, h_last, d["W_q"], d["b_q"], d["cu"], B, Q, ws2)
+    assert gv.gvote_poll_status(ws) == 0 and gv.gvote_poll_status(ws2) == 0
+    Q_staged = Q.float().cpu().numpy()
+    assert Q_pass.shape == Q_staged.shape
+    assert (Q_pass == Q_staged).mean() > 0.99
+    assert np.all(np.abs(Q_pass - Q_staged) <= 2.0 ** -7 * np.abs(Q_staged) + 1e-30)
+    # the current-query rows do not depend on the fit at all: bit for bit
+    cur = slice(G * S, G * (S + 1))
+    assert np.array_equal(Q_pass[:, :, cur], Q_staged[:, :, cur])
