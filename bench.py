@@ -500,6 +500,7 @@ def main():
         "fit_read_over_literal_roofline": (ab["fit"] / (hbm_gbs * 1e9)) / lit_t}
     pass_roofline = {
         "kept_fraction": kept_frac, "per_layer_us": layer_s * 1e6, "stage_us_per_layer": stage_us,
+        "token_layers_per_s": value * L,
         "per_layer_us_one_stream_instrumented": serial_ms * 1e3 / L,
         "full_bytes_roofline_us": full_t * 1e6, "full_bytes_frac": full_t / layer_s,
         "literal_roofline_us": lit_t * 1e6, "literal_frac_whole_pass": lit_t / layer_s,
