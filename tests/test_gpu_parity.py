@@ -394,6 +394,42 @@ def test_vote_long_rows_with_misleading_sample(gv, shift_sampled, shift_sign):
     assert abs(int(budget[0, 0]) - int(ob[0])) <= 0.005 * N
 
 
+def test_vote_exact_route_for_some_heads_of_a_batch(gv):
+    """Three requests, two KV heads each, 512 synthetic rows (four row chunks) per head.  The samples of the
+    first and the last request are shifted so that their brackets miss: four (request, KV head) pairs are
+    selected again by the exact route while the request in the middle keeps its sampled result."""
+    N, d_k, S, Hq, Hkv = 8192, 64, 64, 16, 2
+    cfg = synth.make_small(12, seq_lens=(N, N, N), S=S, d_h=64, n_q_heads=Hq, n_kv_heads=Hkv, d_k=d_k, p_nuc=0.9)
+    li = synth.make_layer(cfg, 0)
+    rng = np.random.default_rng(5)
+    e = rng.normal(size=d_k)
+    e /= np.linalg.norm(e)
+    n_tiles = N // 128
+    want = min(max(n_tiles >> 3, 32), 128)               # the sampling plan of the kernels (vote_geom.cuh)
+    stride = n_tiles // want
+    sampled = np.zeros(N, dtype=bool)
+    for j in range(want):
+        t = j * stride + (((j * 2654435761) & 0xFFFFFFFF) >> 15) % stride
+        sampled[t * 128:(t + 1) * 128] = True
+    Kf = np.empty((Hkv, 3 * N, d_k), dtype=np.float32)
+    for r in range(3):
+        v = rng.normal(size=N)
+        if r != 1:
+            v[sampled] -= 6.0
+        Kf[:, r * N:(r + 1) * N] = (v[:, None] * e[None, :] * math.sqrt(d_k)).astype(np.float32)[None]
+    li.K = synth.f32_to_bf16_bits(Kf)
+    q = o.round_to_bf16(np.stack([e * (1.0 + 0.01 * i) for i in range(S + 1)]))
+    Q_or = [np.stack([q if g % 2 == 0 else q[::-1].copy() for g in range(Hq)]) for _ in range(3)]
+    mask, budget, b_step, _ = _run_vote(gv, cfg, li, Q_or, "topk", False, False)
+    assert _run_vote.exact_heads == 4, _run_vote.exact_heads
+    for r in range(3):
+        Kr = o.bf16_bits_to_f64(li.K[:, r * N:(r + 1) * N])
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(r * N, r), N) for h in range(Hkv)])
+        pu.check_vote_against_oracle(Q_or[r], Kr, float(np.float32(cfg.p_nuc)), "topk", False, gm, b_step[r])
+        om, ob, _, _, _ = o.vote(Q_or[r], Kr, p_nuc=float(np.float32(cfg.p_nuc)))
+        assert np.all(np.abs(budget[r] - ob) <= 0.005 * N)
+
+
 # ----------------------------------------------------------------------------- compact
 @pytest.mark.parametrize("lens,Hkv,d_k,density", [((40,), 2, 32, 0.5), ((129, 31, 257), 2, 64, 0.2),
                                                   ((5000, 300), 3, 128, 0.7), ((4096,), 8, 128, 0.05),
