@@ -278,10 +278,11 @@ int32_t compress_from_moments(const gvote_params* p, const float* mu, const floa
   PROPAGATE(launch_sample(p, mu, var, batch, Ht, nullptr, st));
   PROPAGATE(launch_project(p, Ht, h_last, p->d_h, nullptr, W_q, wq_ld, b_q_or_null, cu_seqlens, batch, m, w, Q, st,
                            seq_len));
+  bool merge_deferred = false;   // whether the settled heads' union still waits in the tentative mask
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st, kv_len));
+                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st, kv_len, &merge_deferred));
   PROPAGATE(launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
-                           total_tokens, max_N, budget, m, w, st));
+                           total_tokens, max_N, budget, m, w, st, merge_deferred));
   if (token_pos) PROPAGATE(launch_remap(p, token_pos, mask, cu_seqlens, batch, total_tokens, max_N, budget, m, w, st));
   return GVOTE_OK;
 }
@@ -371,10 +372,11 @@ int32_t gvote_compress(const gvote_params* p, const void* h, int64_t h_row_strid
     PROPAGATE(launch_prep(p, reinterpret_cast<const float2*>(w + m.fit_partial), m.fit_chunks, h, h_row_stride,
                           cu_seqlens, cu_seqlens, batch, mu, var, X, rope, st));
   PROPAGATE(launch_project_staged(p, X, rope, W_q, wq_ld, b_q_or_null, batch, m, w, Q, st));
+  bool merge_deferred = false;   // whether the settled heads' union still waits in the tentative mask
   PROPAGATE(launch_vote(p, Q, (const __nv_bfloat16*)K, tok_stride, head_stride, cu_seqlens, batch, total_tokens,
-                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st));   // budgets come from the scan below
+                        max_N, mask, nullptr, b_step, nullptr, w, ws_bytes, st, nullptr, &merge_deferred));
   return launch_compact(p, (__nv_bfloat16*)K, (__nv_bfloat16*)V, tok_stride, head_stride, mask, cu_seqlens, batch,
-                        total_tokens, max_N, budget, m, w, st);
+                        total_tokens, max_N, budget, m, w, st, merge_deferred);   // (budgets come from its scan)
 }
 
 // ------------------------------------------------------------------------------------ host variant

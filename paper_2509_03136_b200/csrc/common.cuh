@@ -155,10 +155,15 @@ int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bf
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                     uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs,
                     char* ws, size_t ws_bytes, cudaStream_t st,
-                    const int32_t* kv_len = nullptr);   // [batch][n_kv_heads] rows that count, or all
+                    const int32_t* kv_len = nullptr,    // [batch][n_kv_heads] rows that count, or all
+                    bool* merge_deferred = nullptr);    // given: the vote may leave the union of the settled heads in
+                                                        // the workspace's tentative mask for launch_compact's scan
+                                                        // to merge (*merge_deferred says whether it did)
+// merge_tentative: see launch_vote; the mask is then written, too.
 int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
                        const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens,
-                       int64_t max_N, int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
+                       int64_t max_N, int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st,
+                       bool merge_tentative = false);
 
 int32_t launch_pack(const gvote_params* p, const __nv_bfloat16* K, const __nv_bfloat16* V, int64_t tok, int64_t head,
                     const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,

@@ -23,17 +23,22 @@ constexpr int kTicketPitch = 32;     // ints between two slabs' ticket counters 
 
 // One CTA per (request, head): prefix[h][word] = kept keys of the request before this word.
 // Also clears the compaction flags of the request's tiles (and the head's two ticket counters).
+// When the mask comes straight from the vote of the whole pass (`tmask` given), the head's tentative mask is
+// OR-ed into the keep mask in the same sweep over the words - the union becoming final - unless the head was
+// marked for the exact route, whose rows have written the keep mask themselves.
 __global__ void __launch_bounds__(kScanThreads)
-mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ cu, int Hkv, int64_t row_words,
-                 int32_t* __restrict__ prefix, int32_t* __restrict__ budget, int32_t* __restrict__ flags,
-                 int64_t n_tiles, int32_t* __restrict__ ticket) {
+mask_scan_kernel(uint32_t* __restrict__ mask, const uint32_t* __restrict__ tmask, const uint32_t* __restrict__ head_bad,
+                 const int32_t* __restrict__ cu, int Hkv, int64_t row_words, int32_t* __restrict__ prefix,
+                 int32_t* __restrict__ budget, int32_t* __restrict__ flags, int64_t n_tiles,
+                 int32_t* __restrict__ ticket) {
   __shared__ int warp_tot[kScanThreads / 32];
   __shared__ int carry;
   const int r = blockIdx.y, h = blockIdx.x;
   const int start = cu[r], N = cu[r + 1] - start;
   const int words = (N + 31) >> 5;
   const int64_t woff = mask_word_offset(start, r);
-  const uint32_t* m = mask + (int64_t)h * row_words + woff;
+  uint32_t* m = mask + (int64_t)h * row_words + woff;
+  const uint32_t* merge = (tmask && !head_bad[r * Hkv + h]) ? tmask + (int64_t)h * row_words + woff : nullptr;
   int32_t* pf = prefix + (int64_t)h * row_words + woff;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) carry = 0;
@@ -51,15 +56,24 @@ mask_scan_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ 
   // its own four, the CTA scans the threads' totals
   for (int base = 0; base < words; base += 4 * kScanThreads) {
     const int w0 = base + 4 * tid;
+    uint32_t v[4], t[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[j] = (w0 + j < words) ? m[w0 + j] : 0u;
+      t[j] = (merge && w0 + j < words) ? merge[w0 + j] : 0u;
+    }
     int c[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) c[j] = (w0 + j < words) ? __popc(m[w0 + j]) : 0;
+    for (int j = 0; j < 4; ++j) {
+      if (t[j] & ~v[j]) { v[j] |= t[j]; m[w0 + j] = v[j]; }
+      c[j] = __popc(v[j]);
+    }
     const int mine = c[0] + c[1] + c[2] + c[3];
     int inc = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
+      const int u = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += u;
     }
     if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
@@ -244,8 +258,11 @@ remap_store_kernel(int32_t* __restrict__ token_pos, int64_t slab, const int32_t*
 
 }  // namespace
 
+// `tmask`, `head_bad` (or null): the tentative mask of the vote that made this mask and its per-head flags; the
+// scan then merges it into `mask` (see mask_scan_kernel).  Without them `mask` is only read.
 int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int32_t* cu, int32_t batch,
-                         int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st) {
+                         int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st, const uint32_t* tmask,
+                         const uint32_t* head_bad) {
   const int Hkv = p->n_kv_heads;
   int32_t* prefix = reinterpret_cast<int32_t*>(ws + m.prefix);
   int32_t* flags = reinterpret_cast<int32_t*>(ws + m.flags);
@@ -253,7 +270,8 @@ int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int3
   dim3 gs(Hkv, batch);
   {
     LaunchScope scope_("mask_scan_kernel", st);
-    launch_on(mask_scan_kernel, gs, dim3(kScanThreads), 0, st, mask, cu, Hkv, m.row_words, prefix, budget, flags, m.n_tiles, ticket);
+    launch_on(mask_scan_kernel, gs, dim3(kScanThreads), 0, st, const_cast<uint32_t*>(mask), tmask, head_bad, cu, Hkv, m.row_words,
+              prefix, budget, flags, m.n_tiles, ticket);
   }
   GVOTE_LAUNCH_CHECK("mask_scan_kernel");
   return GVOTE_OK;
@@ -261,13 +279,16 @@ int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int3
 
 int32_t launch_compact(const gvote_params* p, __nv_bfloat16* K, __nv_bfloat16* V, int64_t tok, int64_t head,
                        const uint32_t* mask, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
-                       int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st) {
+                       int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st, bool merge_tentative) {
   const int Hkv = p->n_kv_heads;
   const int32_t* prefix = reinterpret_cast<const int32_t*>(ws + m.prefix);
   int32_t* flags = reinterpret_cast<int32_t*>(ws + m.flags);
   int32_t* ticket = flags + (size_t)2 * Hkv * m.n_tiles;
   int32_t* status = reinterpret_cast<int32_t*>(ws + m.status);
-  const int32_t rc = launch_mask_scan(p, mask, cu, batch, budget, m, ws, st);
+  // (merge_tentative: the vote of this pass left its union in the workspace's tentative mask, see launch_vote)
+  const int32_t rc = launch_mask_scan(p, mask, cu, batch, budget, m, ws, st,
+                                      merge_tentative ? reinterpret_cast<const uint32_t*>(ws + m.tmask) : nullptr,
+                                      merge_tentative ? reinterpret_cast<const uint32_t*>(ws + m.head_bad) : nullptr);
   if (rc != GVOTE_OK) return rc;
   const size_t smem = (size_t)kCompactTile * p->d_k * sizeof(__nv_bfloat16);
   if (smem > 48 * 1024)

@@ -15,7 +15,8 @@
 namespace gvote {
 
 int32_t launch_mask_scan(const gvote_params* p, const uint32_t* mask, const int32_t* cu, int32_t batch,
-                         int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st);
+                         int32_t* budget, const WorkspaceMap& m, char* ws, cudaStream_t st, const uint32_t* tmask = nullptr,
+                         const uint32_t* head_bad = nullptr);
 
 namespace {
 

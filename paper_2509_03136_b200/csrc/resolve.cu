@@ -458,42 +458,64 @@ struct ExactRow {
   __device__ __forceinline__ float operator()(int n) const { return dot(n); }
 };
 
+// Grid: (row s, query head of the group, z).  CTA z walks the (request, KV head) pairs z, z + gridDim.z, ...:
+// a large batch would otherwise launch a CTA per row of every head only to find the head settled.  copy_good:
+// the tentative mask of a settled head is OR-ed into the keep mask here (the head's G * S CTAs a slice each);
+// when the pruning step follows, its mask scan does that on its way over the words and the CTAs of settled
+// heads have nothing to do.
 __global__ void __launch_bounds__(kRowThreads)
 commit_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K, int64_t k_tok, int64_t k_head,
               const int32_t* __restrict__ cu, int Hq, int G, int S, int d_k, float scale,
               const int32_t* __restrict__ b_step, const uint32_t* __restrict__ tmask, int64_t row_words,
-              uint32_t* __restrict__ mask, const uint32_t* __restrict__ head_bad, const int32_t* __restrict__ kv_len) {
+              uint32_t* __restrict__ mask, const uint32_t* __restrict__ head_bad, const int32_t* __restrict__ kv_len,
+              int n_pairs, int copy_good) {
   __shared__ SelShared sh;
   __shared__ __align__(16) __nv_bfloat16 qf[512];
-  const int r = blockIdx.z, g = blockIdx.y, s = blockIdx.x;
-  const int start = cu[r], Ncap = cu[r + 1] - start;
-  const int kh = g / G, Hkv = Hq / G;
+  const int s = blockIdx.x, gl = blockIdx.y;
+  const int Hkv = Hq / G;
   const int tid = threadIdx.x;
-  const int64_t woff = (int64_t)kh * row_words + mask_word_offset(start, r);
-  if (!head_bad[r * Hkv + kh]) {
-    // the G * S rows of the head share the copy of its words
-    const int words = (Ncap + 31) >> 5;
-    const int idx = (g % G) * S + s;
-    for (int w = idx * kRowThreads + tid; w < words; w += G * S * kRowThreads) {
-      const uint32_t v = tmask[woff + w];
-      if (v) mask[woff + w] |= v;
+  const int step = (int)gridDim.z;
+  for (int base = (int)blockIdx.z; base < n_pairs; base += 32 * step) {
+    // which of the next (up to) 32 pairs of this CTA's walk need work: the flags are fetched together
+    uint32_t todo = 0;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) {
+      const int pair = base + i * step;
+      if (pair < n_pairs && (copy_good || head_bad[pair])) todo |= 1u << i;
     }
-    return;
+    while (todo) {
+      const int i = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int pair = base + i * step;
+      const int r = pair / Hkv, kh = pair % Hkv, g = kh * G + gl;
+      const int start = cu[r], Ncap = cu[r + 1] - start;
+      const int64_t woff = (int64_t)kh * row_words + mask_word_offset(start, r);
+      if (!head_bad[pair]) {
+        // (copy_good) the G * S rows of the head share the copy of its words
+        const int words = (Ncap + 31) >> 5;
+        const int idx = gl * S + s;
+        for (int w = idx * kRowThreads + tid; w < words; w += G * S * kRowThreads) {
+          const uint32_t v = tmask[woff + w];
+          if (v) mask[woff + w] |= v;
+        }
+        continue;
+      }
+      // a bracket of this head missed: this row again, exactly
+      const int N = valid_keys(kv_len, r, Hkv, kh, Ncap);
+      const int k = N > 0 ? min(b_step[r * Hq + g], N) : 0;
+      if (k <= 0) continue;
+      const int grow = gl * S + s;
+      const __nv_bfloat16* qrow = Q + (((int64_t)r * Hkv + kh) * (G * (S + 1)) + grow) * d_k;
+      __syncthreads();                                     // the row before this one is through with qf and sh
+      for (int c = tid; c < d_k; c += kRowThreads) qf[c] = qrow[c];
+      __syncthreads();
+      ExactRow row{DotCtx{qf, K + (int64_t)kh * k_head + (int64_t)start * k_tok, k_tok, d_k, scale}};
+      uint32_t t, above_cnt, eq_cnt;
+      unsigned long long above_mass;
+      radix_threshold<false>(row, N, 0.f, (unsigned long long)k, sh, t, above_cnt, above_mass, eq_cnt);
+      emit_row(row, N, t, (uint32_t)k - above_cnt, eq_cnt, mask + woff, sh);
+    }
   }
-  // a bracket of this head missed: this row again, exactly
-  const int N = valid_keys(kv_len, r, Hkv, kh, Ncap);
-  if (N <= 0) return;
-  const int k = min(b_step[r * Hq + g], N);
-  if (k <= 0) return;
-  const int grow = (g % G) * S + s;
-  const __nv_bfloat16* qrow = Q + (((int64_t)r * Hkv + kh) * (G * (S + 1)) + grow) * d_k;
-  for (int i = tid; i < d_k; i += kRowThreads) qf[i] = qrow[i];
-  __syncthreads();
-  ExactRow row{DotCtx{qf, K + (int64_t)kh * k_head + (int64_t)start * k_tok, k_tok, d_k, scale}};
-  uint32_t t, above_cnt, eq_cnt;
-  unsigned long long above_mass;
-  radix_threshold<false>(row, N, 0.f, (unsigned long long)k, sh, t, above_cnt, above_mass, eq_cnt);
-  emit_row(row, N, t, (uint32_t)k - above_cnt, eq_cnt, mask + woff, sh);
 }
 
 }  // namespace
@@ -542,14 +564,18 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
 
 int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
                       const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs, int64_t row_words,
-                      uint32_t* mask, const int32_t* kv_len, cudaStream_t st) {
+                      uint32_t* mask, const int32_t* kv_len, bool copy_good, cudaStream_t st) {
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
-  dim3 grid(p->S, Hq, batch);
+  // about two thousand CTAs at most: each walks its share of the (request, KV head) pairs
+  const int64_t pairs = (int64_t)batch * p->n_kv_heads;
+  int64_t z = 2048 / ((int64_t)p->S * G);
+  z = z < 1 ? 1 : (z > pairs ? pairs : z);
+  dim3 grid(p->S, G, (unsigned)z);
   const float scale = (float)(1.0 / sqrt((double)p->d_k));
   {
     LaunchScope scope_("commit_kernel", st);
     launch_on(commit_kernel, grid, dim3(kRowThreads), 0, st, Q, K, k_tok, k_head, cu, Hq, G, p->S, p->d_k, scale, b_step, vs.tmask,
-                                                row_words, mask, vs.head_bad, kv_len);
+              row_words, mask, vs.head_bad, kv_len, (int)pairs, copy_good ? 1 : 0);
   }
   GVOTE_LAUNCH_CHECK("commit_kernel");
   return GVOTE_OK;

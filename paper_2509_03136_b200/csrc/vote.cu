@@ -242,7 +242,7 @@ int32_t launch_resolve(const gvote_params* p, const int32_t* cu, int32_t batch, 
                        const VoteState& vs, int64_t row_words, const int32_t* kv_len, cudaStream_t st);
 int32_t launch_commit(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
                       const int32_t* cu, int32_t batch, const int32_t* b_step, const VoteState& vs, int64_t row_words,
-                      uint32_t* mask, const int32_t* kv_len, cudaStream_t st);
+                      uint32_t* mask, const int32_t* kv_len, bool copy_good, cudaStream_t st);
 int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32_t* cu, int32_t batch, int64_t max_N,
                          const uint32_t* rowmax_part, int n_part, int64_t row_words, uint32_t* mask, int32_t* b_step,
                          const int32_t* kv_len, cudaStream_t st);
@@ -265,7 +265,8 @@ int32_t launch_budget(const gvote_params* p, const uint32_t* mask, const int32_t
 // enqueued) when no tensor map describes the operands.
 int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok, int64_t k_head,
                    const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N, uint32_t* mask,
-                   int32_t* b_step, const WorkspaceMap& m, char* ws, cudaStream_t st, const int32_t* kv_len) {
+                   int32_t* b_step, const WorkspaceMap& m, char* ws, cudaStream_t st, const int32_t* kv_len,
+                   bool defer_merge) {
   VoteState vs;
   vs.sample = reinterpret_cast<uint16_t*>(ws + m.sample);
   vs.bracket = reinterpret_cast<RowBracket*>(ws + m.bracket);
@@ -290,7 +291,7 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
   GVOTE_STEP(launch_score_sweep(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, vs, m.row_words, status, kv_len,
                                 st));
   GVOTE_STEP(launch_resolve(p, cu, batch, max_N, b_step, vs, m.row_words, kv_len, st));
-  GVOTE_STEP(launch_commit(p, Q, K, k_tok, k_head, cu, batch, b_step, vs, m.row_words, mask, kv_len, st));
+  GVOTE_STEP(launch_commit(p, Q, K, k_tok, k_head, cu, batch, b_step, vs, m.row_words, mask, kv_len, !defer_merge, st));
 #undef GVOTE_STEP
   return GVOTE_OK;
 }
@@ -300,14 +301,21 @@ int32_t vote_fused(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfl
 int32_t launch_vote(const gvote_params* p, const __nv_bfloat16* Q, const __nv_bfloat16* K, int64_t k_tok,
                     int64_t k_head, const int32_t* cu, int32_t batch, int64_t total_tokens, int64_t max_N,
                     uint32_t* mask, int32_t* budget, int32_t* b_step, float* dbg_probs, char* ws, size_t ws_bytes,
-                    cudaStream_t st, const int32_t* kv_len) {
+                    cudaStream_t st, const int32_t* kv_len, bool* merge_deferred) {
   const int Hq = p->n_q_heads, Hkv = p->n_kv_heads, G = Hq / Hkv, S1 = p->S + 1, d_k = p->d_k;
+  const bool defer = merge_deferred != nullptr;
+  if (merge_deferred) *merge_deferred = false;
   const float scale = (float)(1.0 / sqrt((double)d_k));
 
   if (!vote_needs_full_rows(p) && dbg_probs == nullptr && max_N > 0) {
     const WorkspaceMap m = workspace_map(p, batch, total_tokens, max_N, false);
-    const int32_t rc = vote_fused(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, mask, b_step, m, ws, st, kv_len);
-    if (rc == GVOTE_OK) return budget ? launch_budget(p, mask, cu, batch, m.row_words, budget, st) : GVOTE_OK;
+    const int32_t rc = vote_fused(p, Q, K, k_tok, k_head, cu, batch, total_tokens, max_N, mask, b_step, m, ws, st, kv_len,
+                                  defer);
+    if (rc == GVOTE_OK) {
+      if (merge_deferred) *merge_deferred = true;
+      // (a caller that defers the merge takes its budgets from the scan that does it)
+      return (budget && !defer) ? launch_budget(p, mask, cu, batch, m.row_words, budget, st) : GVOTE_OK;
+    }
     if (rc != GVOTE_ERR_UNSUPPORTED_SHAPE) return rc;
     // operands no tensor map describes: the route below, if the workspace has room for its fp32 rows
   }
