@@ -1139,3 +1139,48 @@ def test_workspace_queries_are_the_staged_projection(gv, name):
     # the current-query rows do not depend on the fit at all: bit for bit
     cur = slice(G * S, G * (S + 1))
     assert np.array_equal(Q_pass[:, :, cur], Q_staged[:, :, cur])
+
+
+def test_compress_takes_the_exact_route_when_the_sample_misleads(gv):
+    """The whole pass with keys built against the queries it will use (they do not depend on K: a first run
+    leaves them in the workspace): the logits of exactly the sampled tiles are shifted, so the brackets miss,
+    the head is selected again by the exact route, the pruning step's mask scan must not merge the discarded
+    tentative mask, and the result is still the oracle's vote on those queries, compacted bit for bit."""
+    N, d_k, S = 16384, 64, 6
+    cfg = synth.make_small(13, seq_lens=(N,), S=S, d_h=64, n_q_heads=2, n_kv_heads=1, d_k=d_k, p_nuc=0.9)
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg)
+    geom = _geom(cfg)
+    d = pu.upload_layer(li, gv, torch)
+    mask = torch.empty(1, gv.mask_row_words(N, 1), dtype=torch.int32, device="cuda")
+    budget = torch.empty(1, 1, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(1, 2, dtype=torch.int32, device="cuda")
+    ws = gv.alloc_workspace(p, *geom)
+    gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], d["K"].clone(), d["V"].clone(), d["cu"], geom, mask, budget, b_step, ws)
+    Qg = _queries_left_in(gv, p, ws, geom)                 # [1, 1, G (S+1), d_k]
+    e = Qg[0, 0].mean(axis=0)
+    e /= np.linalg.norm(e)
+    rng = np.random.default_rng(7)
+    v = rng.normal(size=N)
+    n_tiles = N // 128
+    want = min(max(n_tiles >> 3, 32), 128)               # the sampling plan of the kernels (vote_geom.cuh)
+    stride = n_tiles // want
+    for j in range(want):
+        t = j * stride + (((j * 2654435761) & 0xFFFFFFFF) >> 15) % stride
+        v[t * 128:(t + 1) * 128] -= 6.0
+    Kbits = synth.f32_to_bf16_bits((v[:, None] * e[None, :] * math.sqrt(d_k)).astype(np.float32)[None])
+    Kd, Vd = gv.bf16_from_bits(Kbits), d["V"].clone()
+    ws2 = gv.alloc_workspace(p, *geom)
+    gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], Kd, Vd, d["cu"], geom, mask, budget, b_step, ws2)
+    assert gv.gvote_poll_status(ws2) == 0
+    assert gv.gvote_exact_heads(ws2) == 1
+    assert np.array_equal(_queries_left_in(gv, p, ws2, geom), Qg)
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    Qr = pu.from_group_major(Qg[0], G)
+    Kr = o.bf16_bits_to_f64(Kbits)
+    gm = np.stack([gv.unpack_mask(mask.cpu().numpy()[0], 0, N)])
+    pu.check_vote_against_oracle(Qr, Kr, float(np.float32(cfg.p_nuc)), "topk", False, gm, b_step.cpu().numpy()[0])
+    n = int(gm[0].sum())
+    assert int(budget[0, 0]) == n
+    Kc, Vc = o.compact(Kbits, li.V, gm)
+    assert np.array_equal(gv.bits_from_bf16(Kd)[0, :n], Kc[0]) and np.array_equal(gv.bits_from_bf16(Vd)[0, :n], Vc[0])
