@@ -1184,3 +1184,42 @@ def test_compress_takes_the_exact_route_when_the_sample_misleads(gv):
     assert int(budget[0, 0]) == n
     Kc, Vc = o.compact(Kbits, li.V, gm)
     assert np.array_equal(gv.bits_from_bf16(Kd)[0, :n], Kc[0]) and np.array_equal(gv.bits_from_bf16(Vd)[0, :n], Vc[0])
+
+
+@pytest.mark.parametrize("name", ["small2", "c1"])
+def test_compress_with_the_current_query_set_in_the_union(gv, name):
+    """include_c0 inside the whole pass: the current query's own top-p set is written into the keep mask by
+    the top-p kernel, the synthetic rows' union reaches it through the tentative mask and the pruning step's
+    scan: both must survive."""
+    cfg = _small_cfgs()[2] if name == "small2" else synth.make_config(name)
+    li = synth.make_layer(cfg, 0)
+    p = gv.params_from_config(cfg, include_c0=True)
+    geom = _geom(cfg)
+    ws = gv.alloc_workspace(p, *geom)
+    d = pu.upload_layer(li, gv, torch)
+    mask = torch.empty(cfg.n_kv_heads, gv.mask_row_words(cfg.total_tokens, cfg.batch), dtype=torch.int32, device="cuda")
+    budget = torch.empty(cfg.batch, cfg.n_kv_heads, dtype=torch.int32, device="cuda")
+    b_step = torch.empty(cfg.batch, cfg.n_q_heads, dtype=torch.int32, device="cuda")
+    gv.gvote_compress(p, d["h"], d["W_q"], d["b_q"], d["K"], d["V"], d["cu"], geom, mask, budget, b_step, ws)
+    assert gv.gvote_poll_status(ws) == 0
+    Qg = _queries_left_in(gv, p, ws, geom)
+    mask, budget, b_step = mask.cpu().numpy(), budget.cpu().numpy(), b_step.cpu().numpy()
+    Kg, Vg = gv.bits_from_bf16(d["K"]), gv.bits_from_bf16(d["V"])
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    pf = float(np.float32(cfg.p_nuc))
+    for r in range(cfg.batch):
+        a, b = int(li.cu_seqlens[r]), int(li.cu_seqlens[r + 1])
+        N = b - a
+        gm = np.stack([gv.unpack_mask(mask[h], gv.mask_word_offset(a, r), N) for h in range(cfg.n_kv_heads)])
+        Kr = o.bf16_bits_to_f64(li.K[:, a:b])
+        Qr = pu.from_group_major(Qg[r], G)
+        pu.check_vote_against_oracle(Qr, Kr, pf, "topk", True, gm, b_step[r])          # 1e-3 bands, C0 in the union
+        om, ob, _, _, _ = o.vote(Qr, Kr, p_nuc=pf, include_c0=True)
+        assert np.all(np.abs(budget[r] - ob) <= max(2, 0.005 * N))
+        without, _, _, _, _ = o.vote(Qr, Kr, p_nuc=pf, include_c0=False)
+        assert (om & ~without).any(), "the case does not exercise include_c0"
+        Kc, Vc = o.compact(li.K[:, a:b], li.V[:, a:b], gm)
+        for h in range(cfg.n_kv_heads):
+            n = int(gm[h].sum())
+            assert budget[r, h] == n
+            assert np.array_equal(Kg[h, a:a + n], Kc[h]) and np.array_equal(Vg[h, a:a + n], Vc[h])
