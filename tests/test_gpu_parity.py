@@ -652,7 +652,8 @@ def test_compress_small(gv, idx):
     _check_compress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx % 2 == 1)))
 
 
-@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c1", "topp"), ("c3", "topk")])
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c1", "topp"), ("c3", "topk"),
+                                       ("c3", "topp")])
 def test_compress_configs(gv, name, mode):
     cfg = synth.make_config(name)
     _check_compress(gv, cfg, synth.make_layer(cfg, 0), mode)
@@ -866,7 +867,7 @@ def test_recompress_small(gv, idx, mode):
     _check_recompress(gv, cfg, synth.make_layer(cfg, 0, with_bias=(idx == 3)), mode)
 
 
-@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk")])
+@pytest.mark.parametrize("name,mode", [("c0", "topk"), ("c0", "topp"), ("c1", "topk"), ("c3", "topk")])
 def test_recompress_configs(gv, name, mode):
     cfg = synth.make_config(name)
     _check_recompress(gv, cfg, synth.make_layer(cfg, 0), mode, n_new=17)
