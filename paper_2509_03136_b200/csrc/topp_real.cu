@@ -2,12 +2,13 @@
 // keys, the smallest set C0 of keys whose weights reach the mass p, and its size B_step = |C0|.
 //
 // There are only n_q_heads such rows per request but each is N long, so a row is shared by a thread-
-// block cluster of eight CTAs, one eighth of the row each, in ONE launch:
+// block cluster of up to eight CTAs (eight for a single request, fewer when a batch brings many rows), an
+// equal part of the row each, in ONE launch:
 //   1. every CTA bins its keys by their distance below the row maximum (512 bins of 1/16 logit; the
 //      maximum comes from the score kernel's read-out) and accumulates per bin a count and the softmax
 //      numerators exp(l - max) in 2^-40 fixed point - integers, so the sums do not depend on the order
 //      of arrival and two runs give the same bits;
-//   2. the cluster's first CTA adds the eight histograms (it reads its peers' shared memory), sums the
+//   2. the cluster's first CTA adds the histograms (it reads its peers' shared memory), sums the
 //      bins into Z and walks them from the top until the mass reaches p * Z;
 //   3. every CTA sends the keys of that crossing bin from its part of the row into a list in the first
 //      CTA's shared memory;
@@ -31,7 +32,6 @@ using namespace sel;
 constexpr int kBins = 512;
 constexpr float kBinsPerLogit = 16.0f;
 constexpr int kThreads = 256;
-constexpr int kClusterCtas = 8;
 constexpr int kListCap = 4096;      // keys of the crossing bin held in shared memory
 constexpr int kRankCap = 256;       // keys ranked pairwise (quadratic work: keep it small; one per thread)
 constexpr int kSubBins = 256;       // one per thread
@@ -115,6 +115,7 @@ __device__ __forceinline__ void block_scan_pair(uint32_t c, unsigned long long m
   m_excl = m_before + m_inc - m;
 }
 
+template <int kClusterCtas>     // CTAs that share a row: 8, 4, 2 or 1
 __global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kThreads)
 real_topp_kernel(const float* __restrict__ logits, const int32_t* __restrict__ cu, int Hq, int G,
                  const uint32_t* __restrict__ rowmax_part, int n_part, float p_nuc, int include_c0, int64_t row_words,
@@ -404,14 +405,21 @@ int32_t launch_real_topp(const gvote_params* p, const float* logits, const int32
   const int Hq = p->n_q_heads, G = Hq / p->n_kv_heads;
   (void)max_N;
   static_assert(kBins == 2 * kThreads && kSubBins == kThreads && kRankCap == kThreads, "bins per thread");
-  GVOTE_CUDA_CHECK(cudaFuncSetAttribute(real_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(ClusterShared)));
-  dim3 grid((unsigned)kClusterCtas, (unsigned)Hq, (unsigned)batch);
-  {
+  // CTAs per row: eight when the rows are few (one request: n_q_heads rows, each max_N long), fewer when a
+  // batch brings many rows, so that the launch stays within a few CTAs per SM - the steps of a cluster cost
+  // the same whether its CTAs have 32 keys each or 4096 (16 ragged requests of 32 heads: 28 us with two CTAs
+  // per row, 37 with four, 69 with eight; one request of 32768 keys: 20, 24 and 34 us with 8, 4 and 2)
+  const int64_t rows = (int64_t)Hq * batch;
+  const int cl = rows * 8 <= 592 ? 8 : (rows * 4 <= 592 ? 4 : 2);
+  auto launch = [&](auto kernel, int n_cta) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ClusterShared));
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)n_cta, (unsigned)Hq, (unsigned)batch);
     LaunchScope scope_("real_topp_kernel", st);
-    launch_on(real_topp_kernel, grid, dim3(kThreads), sizeof(ClusterShared), st, logits, cu, Hq, G, rowmax_part, n_part, p->p_nuc,
-                                                                    p->include_c0, row_words, mask, b_step, kv_len);
-  }
+    return launch_on(kernel, grid, dim3(kThreads), sizeof(ClusterShared), st, logits, cu, Hq, G, rowmax_part, n_part, p->p_nuc,
+                     p->include_c0, row_words, mask, b_step, kv_len);
+  };
+  GVOTE_CUDA_CHECK(cl == 8 ? launch(real_topp_kernel<8>, 8) : (cl == 4 ? launch(real_topp_kernel<4>, 4) : launch(real_topp_kernel<2>, 2)));
   GVOTE_LAUNCH_CHECK("real_topp_kernel");
   return GVOTE_OK;
 }
